@@ -1,0 +1,169 @@
+/*
+ * C ABI of the B200 AlexNet training-step library.
+ *
+ * The calls follow the paper's statement of the problem: identically
+ * initialised model replicas ("Data parallelism": "They are initialized
+ * identically"), a loader that brings the next minibatch to the GPU and
+ * preprocesses it while the current one trains ("Parallel Data Loading" and
+ * its figure), one update per replica on its own minibatch, and the exchange
+ * and average of weights, biases and momentum between two replicas ("Data
+ * parallelism" and its figure), here with both replicas in one GPU's memory.
+ *
+ * Conventions
+ *   - every function returns ALEXNET_OK (0) or a negative error code; nothing
+ *     aborts or throws.  alexnet_last_error() gives a message for the last failure.
+ *   - "host" pointers are ordinary CPU pointers (pinned where stated);
+ *     "device" pointers are CUDA device pointers of the current device.
+ *   - streams are cudaStream_t handles passed as void*.
+ *   - the caller owns the device arena, the host buffers and the streams; the
+ *     library owns only its handle, events and tensor maps.
+ *   - canonical parameter vector (get/set): fp32, concatenated conv1.W
+ *     [96][3][11][11], conv1.b, conv2.W [256][48][5][5], conv2.b, conv3.W
+ *     [384][256][3][3], conv3.b, conv4.W [384][192][3][3], conv4.b, conv5.W
+ *     [256][192][3][3], conv5.b, fc6.W [4096][9216] (input index c*36+h*6+w),
+ *     fc6.b, fc7.W [4096][4096], fc7.b, fc8.W [1000][4096], fc8.b;
+ *     60,965,224 floats.  Grouped filters are [Cout][Cin/groups][kh][kw]; output
+ *     channel co belongs to group co / (Cout/groups).  Convolution is
+ *     cross-correlation (no kernel flip).
+ */
+#ifndef ALEXNET_H
+#define ALEXNET_H
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct alexnet alexnet_t; /* opaque */
+
+enum {
+    ALEXNET_OK = 0,
+    ALEXNET_ERR_ARG = -1,            /* NULL / out-of-range / inconsistent argument */
+    ALEXNET_ERR_CUDA = -2,           /* a CUDA runtime or driver call failed */
+    ALEXNET_ERR_STATE = -3,          /* call out of order (no batch loaded, both slots busy) */
+    ALEXNET_ERR_DEVICE_TIMEOUT = -4, /* a bounded device-side wait expired (latched) */
+    ALEXNET_ERR_NOMEM = -5           /* arena too small */
+};
+
+enum {                                /* alexnet_config_t.flags */
+    ALEXNET_FLAG_LRN_ALPHA_DIV_N = 1, /* s = k + (alpha/n) * sum a^2 instead of alpha * sum a^2 */
+    ALEXNET_FLAG_WD_ON_BIASES = 2,    /* weight decay also on biases */
+    ALEXNET_FLAG_INVERTED_DROPOUT = 4 /* kept units scaled by 1/(1-p) */
+};
+
+typedef struct {
+    int32_t batch;      /* images per replica per step, >= 1 */
+    int32_t replicas;   /* 1 or 2 */
+    uint64_t seed;      /* seeds crop/flip and dropout streams (and the optional init) */
+    float lr, momentum, weight_decay;   /* Krizhevsky et al. 2012: 0.01, 0.9, 5e-4 */
+    int32_t lrn_size;   /* must be 5 */
+    float lrn_alpha, lrn_beta, lrn_k;   /* 1e-4, 0.75, 2 */
+    float dropout_p;    /* 0.5; 0 disables */
+    float init_std;     /* > 0: weights ~ N(0, init_std^2) from the seed, same in all replicas; 0: zeros */
+    uint32_t flags;
+} alexnet_config_t;
+
+/* Number of parameters (60,965,224). */
+size_t alexnet_param_count(void);
+
+/* Bytes of device memory alexnet_create needs for this configuration
+ * (parameters, momentum, gradients, bf16 copies, activations, batch slots,
+ * split-K scratch).  Returns 0 for an invalid configuration. */
+size_t alexnet_workspace_bytes(const alexnet_config_t* cfg);
+
+/* Build `replicas` identically initialised models inside the caller's device
+ * arena (paper: "Data parallelism", first sentences).
+ *   dev_arena        device, >= alexnet_workspace_bytes(cfg), 1024-byte aligned; owned by the caller,
+ *                    must outlive the handle
+ *   host_mean_image  host fp32 [256][256][3] (HWC), or NULL for zeros; copied
+ *   compute_stream   stream of train_step / replica_average
+ *   copy_stream      side stream of load_batch_async (may equal compute_stream: no overlap then)
+ * Errors: ARG (bad cfg / NULL), NOMEM (arena_bytes too small), CUDA. */
+int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_bytes,
+                   const float* host_mean_image, void* compute_stream, void* copy_stream, alexnet_t** out);
+int alexnet_destroy(alexnet_t* h);
+
+/* Loader half of the paper's "Parallel Data Loading": on the copy stream,
+ * copy one uint8 minibatch [B][256][256][3] (HWC) and its int32 labels [B]
+ * (each in [0,1000)) to the device and run the preprocessing gather
+ * (subtract mean image, random 227 crop, random flip; offsets and flip bits
+ * from (seed, replica, step)).  Asynchronous; returns at once.  The source
+ * buffers may be pinned host memory or device memory and must stay unchanged
+ * until the copy has run (alexnet_sync, or the next load into the same slot).
+ * Each replica has two batch slots filled in turn; a third load with none
+ * consumed returns STATE. */
+int alexnet_load_batch_async(alexnet_t* h, int replica, const uint8_t* images, const int32_t* labels, uint64_t step);
+
+/* One SGD step of `replica` on its oldest loaded batch (paper: "they are
+ * updated on different minibatches respectively"): forward, softmax
+ * cross-entropy, backward, momentum update
+ *   v <- momentum*v - lr*weight_decay*w - lr*g ; w <- w + v   (decay on weights only unless flagged).
+ * Runs on the compute stream after the batch's load has finished.  If
+ * host_loss is non-NULL the mean loss is written there and the call
+ * synchronises the compute stream; otherwise it is asynchronous.
+ * Errors: STATE (no loaded batch), DEVICE_TIMEOUT (latched), CUDA. */
+int alexnet_train_step(alexnet_t* h, int replica, float* host_loss);
+
+/* Steps 2 and 3 of the paper's data-parallel figure for two replicas held in
+ * one GPU memory: w_a = w_b = (w_a+w_b)/2 and the same for momentum, over all
+ * weights and biases.  No-op returning OK when replicas == 1. */
+int alexnet_replica_average(alexnet_t* h);
+
+/* Read / write a replica's parameters in the canonical order above.
+ *   which: 0 = parameters, 1 = momentum, 2 = gradient of the last step (read only)
+ *   host buffer of n = alexnet_param_count() floats.  Synchronous. */
+int alexnet_get_params(alexnet_t* h, int replica, int which, float* host_out, size_t n);
+int alexnet_set_params(alexnet_t* h, int replica, int which, const float* host_in, size_t n);
+
+/* Debug / parity access to intermediate tensors of the last step of a replica,
+ * converted to fp32 in canonical NCHW (or [B][N]) order.  alexnet_tensor_size
+ * gives the element count.  set_tensor writes a tensor (rounded to its device
+ * type) so that one operation can be run in isolation by alexnet_run_op. */
+enum {
+    ALEXNET_T_CROPFLIP = 0, /* [B][3]: ox, oy, flip */
+    ALEXNET_T_X0, ALEXNET_T_A1, ALEXNET_T_N1, ALEXNET_T_P1, ALEXNET_T_ARG1,
+    ALEXNET_T_A2, ALEXNET_T_N2, ALEXNET_T_P2, ALEXNET_T_ARG2,
+    ALEXNET_T_A3, ALEXNET_T_A4, ALEXNET_T_A5, ALEXNET_T_P5, ALEXNET_T_ARG5,
+    ALEXNET_T_F6, ALEXNET_T_F7, ALEXNET_T_Z, ALEXNET_T_M6, ALEXNET_T_M7,
+    ALEXNET_T_DZ, ALEXNET_T_DF7, ALEXNET_T_DF6, ALEXNET_T_DP5, ALEXNET_T_DA5, ALEXNET_T_DA4, ALEXNET_T_DA3,
+    ALEXNET_T_DP2, ALEXNET_T_DN2, ALEXNET_T_DA2, ALEXNET_T_DP1, ALEXNET_T_DN1, ALEXNET_T_DA1,
+    ALEXNET_T_LOSS, /* [B] per-sample loss */
+    ALEXNET_T_COUNT
+};
+size_t alexnet_tensor_size(const alexnet_t* h, int tensor_id);
+int alexnet_get_tensor(alexnet_t* h, int replica, int tensor_id, float* host_out, size_t n);
+int alexnet_set_tensor(alexnet_t* h, int replica, int tensor_id, const float* host_in, size_t n);
+
+/* Run one operation of the step `iters` times on the replica's current
+ * tensors (compute stream, asynchronous), for per-layer parity and timing.
+ * Operation ids: ALEXNET_OP_*.  Operations that read a batch slot (conv1,
+ * softmax labels, preprocess) and get/set_tensor of X0 and CROPFLIP use the slot
+ * touched by the most recent load_batch_async or train_step of that replica. */
+enum {
+    ALEXNET_OP_CONV1_FWD = 0, ALEXNET_OP_CONV2_FWD, ALEXNET_OP_CONV3_FWD, ALEXNET_OP_CONV4_FWD, ALEXNET_OP_CONV5_FWD,
+    ALEXNET_OP_CONV2_BWD_DATA, ALEXNET_OP_CONV3_BWD_DATA, ALEXNET_OP_CONV4_BWD_DATA, ALEXNET_OP_CONV5_BWD_DATA,
+    ALEXNET_OP_CONV1_BWD_WEIGHT, ALEXNET_OP_CONV2_BWD_WEIGHT, ALEXNET_OP_CONV3_BWD_WEIGHT,
+    ALEXNET_OP_CONV4_BWD_WEIGHT, ALEXNET_OP_CONV5_BWD_WEIGHT,
+    ALEXNET_OP_FC6_FWD, ALEXNET_OP_FC7_FWD, ALEXNET_OP_FC8_FWD,
+    ALEXNET_OP_FC6_BWD_DATA, ALEXNET_OP_FC7_BWD_DATA, ALEXNET_OP_FC8_BWD_DATA,
+    ALEXNET_OP_FC6_BWD_WEIGHT, ALEXNET_OP_FC7_BWD_WEIGHT, ALEXNET_OP_FC8_BWD_WEIGHT,
+    ALEXNET_OP_LRN1_FWD, ALEXNET_OP_LRN2_FWD, ALEXNET_OP_LRN1_BWD, ALEXNET_OP_LRN2_BWD,
+    ALEXNET_OP_POOL1_FWD, ALEXNET_OP_POOL2_FWD, ALEXNET_OP_POOL5_FWD,
+    ALEXNET_OP_POOL1_BWD, ALEXNET_OP_POOL2_BWD, ALEXNET_OP_POOL5_BWD,
+    ALEXNET_OP_SOFTMAX, ALEXNET_OP_UPDATE, ALEXNET_OP_AVERAGE, ALEXNET_OP_PREPROCESS,
+    ALEXNET_OP_COUNT
+};
+int alexnet_run_op(alexnet_t* h, int replica, int op, int iters);
+
+/* Number of kernels launched by this handle since creation (for accounting). */
+uint64_t alexnet_launch_count(const alexnet_t* h);
+
+/* Wait for both streams; returns a latched DEVICE_TIMEOUT or CUDA error if any. */
+int alexnet_sync(alexnet_t* h);
+const char* alexnet_last_error(const alexnet_t* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,193 @@
+"""Thin Python binding of the C ABI in include/alexnet.h (argument marshalling only).
+
+PyTorch is used for device memory, pinned host memory and streams; every step
+of the training path runs inside the CUDA library.  There is no CPU fallback:
+if the library has not been built, importing a handle fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+
+OK, ERR_ARG, ERR_CUDA, ERR_STATE, ERR_DEVICE_TIMEOUT, ERR_NOMEM = 0, -1, -2, -3, -4, -5
+FLAG_LRN_ALPHA_DIV_N, FLAG_WD_ON_BIASES, FLAG_INVERTED_DROPOUT = 1, 2, 4
+
+TENSORS = ["CROPFLIP", "X0", "A1", "N1", "P1", "ARG1", "A2", "N2", "P2", "ARG2", "A3", "A4", "A5", "P5", "ARG5",
+           "F6", "F7", "Z", "M6", "M7", "DZ", "DF7", "DF6", "DP5", "DA5", "DA4", "DA3", "DP2", "DN2", "DA2",
+           "DP1", "DN1", "DA1", "LOSS"]
+T = {n: i for i, n in enumerate(TENSORS)}
+OPS = ["CONV1_FWD", "CONV2_FWD", "CONV3_FWD", "CONV4_FWD", "CONV5_FWD",
+       "CONV2_BWD_DATA", "CONV3_BWD_DATA", "CONV4_BWD_DATA", "CONV5_BWD_DATA",
+       "CONV1_BWD_WEIGHT", "CONV2_BWD_WEIGHT", "CONV3_BWD_WEIGHT", "CONV4_BWD_WEIGHT", "CONV5_BWD_WEIGHT",
+       "FC6_FWD", "FC7_FWD", "FC8_FWD", "FC6_BWD_DATA", "FC7_BWD_DATA", "FC8_BWD_DATA",
+       "FC6_BWD_WEIGHT", "FC7_BWD_WEIGHT", "FC8_BWD_WEIGHT",
+       "LRN1_FWD", "LRN2_FWD", "LRN1_BWD", "LRN2_BWD", "POOL1_FWD", "POOL2_FWD", "POOL5_FWD",
+       "POOL1_BWD", "POOL2_BWD", "POOL5_BWD", "SOFTMAX", "UPDATE", "AVERAGE", "PREPROCESS"]
+OP = {n: i for i, n in enumerate(OPS)}
+
+EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "alexnet_destroy",
+           "alexnet_load_batch_async", "alexnet_train_step", "alexnet_replica_average", "alexnet_get_params",
+           "alexnet_set_params", "alexnet_tensor_size", "alexnet_get_tensor", "alexnet_set_tensor", "alexnet_run_op",
+           "alexnet_launch_count", "alexnet_sync", "alexnet_last_error"]
+
+
+class Config(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int32), ("replicas", ctypes.c_int32), ("seed", ctypes.c_uint64),
+                ("lr", ctypes.c_float), ("momentum", ctypes.c_float), ("weight_decay", ctypes.c_float),
+                ("lrn_size", ctypes.c_int32), ("lrn_alpha", ctypes.c_float), ("lrn_beta", ctypes.c_float),
+                ("lrn_k", ctypes.c_float), ("dropout_p", ctypes.c_float), ("init_std", ctypes.c_float),
+                ("flags", ctypes.c_uint32)]
+
+
+class AlexNetError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"alexnet error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library():
+    """dlopen the in-tree CUDA library; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_build.LIB):
+        raise RuntimeError(f"{_build.LIB} is missing: run `python -m paper_1412_2302_b200.build` "
+                           "(there is no CPU fallback)")
+    L = ctypes.CDLL(_build.LIB)
+    vp, sz, i32, u64 = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_uint64
+    L.alexnet_param_count.restype = sz
+    L.alexnet_workspace_bytes.restype = sz
+    L.alexnet_workspace_bytes.argtypes = [ctypes.POINTER(Config)]
+    L.alexnet_create.argtypes = [ctypes.POINTER(Config), vp, sz, vp, vp, vp, ctypes.POINTER(vp)]
+    L.alexnet_destroy.argtypes = [vp]
+    L.alexnet_load_batch_async.argtypes = [vp, i32, vp, vp, u64]
+    L.alexnet_train_step.argtypes = [vp, i32, vp]
+    L.alexnet_replica_average.argtypes = [vp]
+    L.alexnet_get_params.argtypes = [vp, i32, i32, vp, sz]
+    L.alexnet_set_params.argtypes = [vp, i32, i32, vp, sz]
+    L.alexnet_tensor_size.restype = sz
+    L.alexnet_tensor_size.argtypes = [vp, i32]
+    L.alexnet_get_tensor.argtypes = [vp, i32, i32, vp, sz]
+    L.alexnet_set_tensor.argtypes = [vp, i32, i32, vp, sz]
+    L.alexnet_run_op.argtypes = [vp, i32, i32, i32]
+    L.alexnet_launch_count.restype = u64
+    L.alexnet_launch_count.argtypes = [vp]
+    L.alexnet_sync.argtypes = [vp]
+    L.alexnet_last_error.restype = ctypes.c_char_p
+    L.alexnet_last_error.argtypes = [vp]
+    _lib = L
+    return L
+
+
+def _ptr(x):
+    """Raw address of a torch tensor or numpy array."""
+    if hasattr(x, "data_ptr"):
+        return ctypes.c_void_p(x.data_ptr())
+    return ctypes.c_void_p(x.ctypes.data)
+
+
+class AlexNet:
+    """One handle = `replicas` identically initialised AlexNets in one GPU's memory."""
+
+    def __init__(self, batch, replicas=1, seed=14122302, lr=0.01, momentum=0.9, weight_decay=5e-4,
+                 lrn_alpha=1e-4, lrn_beta=0.75, lrn_k=2.0, dropout_p=0.5, init_std=0.0, flags=0,
+                 mean_image=None, device="cuda:0", compute_stream=None, copy_stream=None):
+        import torch
+        self._torch = torch
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required (there is no CPU fallback)")
+        self.device = torch.device(device)
+        torch.cuda.set_device(self.device)
+        self.cfg = Config(batch, replicas, seed, lr, momentum, weight_decay, 5, lrn_alpha, lrn_beta, lrn_k,
+                          dropout_p, init_std, flags)
+        self.batch, self.replicas = batch, replicas
+        nbytes = self.lib.alexnet_workspace_bytes(ctypes.byref(self.cfg))
+        if nbytes == 0:
+            raise AlexNetError(ERR_ARG, "invalid configuration")
+        self.arena = torch.empty(nbytes + 1024, dtype=torch.uint8, device=self.device)
+        base = (self.arena.data_ptr() + 1023) // 1024 * 1024
+        self.compute_stream = compute_stream or torch.cuda.Stream(self.device)
+        self.copy_stream = copy_stream or torch.cuda.Stream(self.device)
+        mean = None if mean_image is None else np.ascontiguousarray(mean_image, np.float32)
+        h = ctypes.c_void_p()
+        rc = self.lib.alexnet_create(ctypes.byref(self.cfg), ctypes.c_void_p(base), nbytes,
+                                     None if mean is None else _ptr(mean),
+                                     ctypes.c_void_p(self.compute_stream.cuda_stream),
+                                     ctypes.c_void_p(self.copy_stream.cuda_stream), ctypes.byref(h))
+        if rc != OK:
+            raise AlexNetError(rc, "alexnet_create failed")
+        self.h = h
+        self.param_count = int(self.lib.alexnet_param_count())
+        self._keep = []
+
+    def _ck(self, rc):
+        if rc != OK:
+            raise AlexNetError(rc, self.lib.alexnet_last_error(self.h).decode())
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.alexnet_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- the path
+    def load_batch_async(self, replica, images, labels, step):
+        """images uint8 [B,256,256,3], labels int32 [B]; pinned-host or device torch tensors (or numpy)."""
+        self._keep = self._keep[-8:] + [(images, labels)]
+        self._ck(self.lib.alexnet_load_batch_async(self.h, replica, _ptr(images), _ptr(labels), int(step)))
+
+    def train_step(self, replica=0, want_loss=False):
+        if want_loss:
+            loss = ctypes.c_float()
+            self._ck(self.lib.alexnet_train_step(self.h, replica, ctypes.byref(loss)))
+            return loss.value
+        self._ck(self.lib.alexnet_train_step(self.h, replica, None))
+        return None
+
+    def replica_average(self):
+        self._ck(self.lib.alexnet_replica_average(self.h))
+
+    def sync(self):
+        self._ck(self.lib.alexnet_sync(self.h))
+
+    # ---- parameters, tensors, single operations
+    def get_params(self, replica=0, which=0):
+        out = np.empty(self.param_count, np.float32)
+        self._ck(self.lib.alexnet_get_params(self.h, replica, which, _ptr(out), out.size))
+        return out
+
+    def set_params(self, values, replica=0, which=0):
+        v = np.ascontiguousarray(values, np.float32)
+        self._ck(self.lib.alexnet_set_params(self.h, replica, which, _ptr(v), v.size))
+
+    def tensor_size(self, name):
+        return int(self.lib.alexnet_tensor_size(self.h, T[name]))
+
+    def get_tensor(self, name, replica=0):
+        out = np.empty(self.tensor_size(name), np.float32)
+        self._ck(self.lib.alexnet_get_tensor(self.h, replica, T[name], _ptr(out), out.size))
+        return out
+
+    def set_tensor(self, name, values, replica=0):
+        v = np.ascontiguousarray(values, np.float32).ravel()
+        self._ck(self.lib.alexnet_set_tensor(self.h, replica, T[name], _ptr(v), v.size))
+
+    def run_op(self, name, replica=0, iters=1):
+        self._ck(self.lib.alexnet_run_op(self.h, replica, OP[name], iters))
+
+    @property
+    def launch_count(self):
+        return int(self.lib.alexnet_launch_count(self.h))

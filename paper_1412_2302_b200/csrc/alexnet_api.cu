@@ -1,0 +1,935 @@
+// Host side of the C ABI declared in include/alexnet.h: arena layout, tensor
+// maps and GEMM plans, the two-stream step schedule, parameter / tensor access.
+#include "../../include/alexnet.h"
+
+#include <cudaTypedefs.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "kernels.cuh"
+#include "tc_gemm.cuh"
+
+namespace {
+
+typedef __nv_bfloat16 bf16;
+
+// ------------------------------------------------------------------ geometry
+struct Grid { int Hp, Wp, H, W, C; };
+struct ConvL {
+    int k, pad, cin, cout, groups, cig, cog, taps;
+    Grid gin, gout;
+    long long w_off, b_off, wt_off, canon_w, canon_b;
+    int shift[25];
+};
+struct FcL { int K, N; long long w_off, b_off, canon_w, canon_b; };
+
+struct Layout {
+    ConvL conv[5];
+    FcL fc[3];
+    long long n_weights;   // internal floats holding weights (decay region), multiple of 64
+    long long n_total;     // internal floats in total, multiple of 64
+    long long wt_total;    // bf16 elements of the transposed conv filters
+    kn::ParamSegs segs;
+    kn::TransposeJobs tjobs;
+};
+
+long long align_up(long long x, long long a) { return (x + a - 1) / a * a; }
+
+Layout make_layout() {
+    Layout L;
+    memset(&L, 0, sizeof(L));
+    // conv1 runs as a stride-1 3x3 convolution over the 4x4 space-to-depth input (48 channels on a 57x57 grid)
+    const int spec[5][6] = {  // k, pad, cin, cout, groups, grid
+        {3, 0, 48, 96, 1, 57}, {5, 2, 96, 256, 2, 29}, {3, 1, 256, 384, 1, 14}, {3, 1, 384, 384, 2, 14}, {3, 1, 384, 256, 2, 14}};
+    const int valid[5] = {55, 27, 13, 13, 13};
+    long long off = 0, canon = 0, wt = 0;
+    const long long canon_wcount[5] = {34848, 307200, 884736, 663552, 442368};
+    for (int l = 0; l < 5; ++l) {
+        ConvL& c = L.conv[l];
+        c.k = spec[l][0]; c.pad = spec[l][1]; c.cin = spec[l][2]; c.cout = spec[l][3]; c.groups = spec[l][4];
+        c.cig = c.cin / c.groups; c.cog = c.cout / c.groups; c.taps = c.k * c.k;
+        const int gp = spec[l][5];
+        c.gin = Grid{gp, gp, l == 0 ? 57 : valid[l], l == 0 ? 57 : valid[l], c.cin};
+        c.gout = Grid{gp, gp, valid[l], valid[l], c.cout};
+        for (int t = 0; t < c.taps; ++t) c.shift[t] = (t / c.k - c.pad) * gp + (t % c.k - c.pad);
+        c.w_off = off; off = align_up(off + (long long)c.taps * c.cout * c.cig, 64);
+        c.canon_w = canon; canon += canon_wcount[l];
+        c.canon_b = canon; canon += c.cout;
+        if (l > 0) { c.wt_off = wt; wt = align_up(wt + (long long)c.taps * c.cin * c.cog, 64); }
+    }
+    const int fcs[3][2] = {{9216, 4096}, {4096, 4096}, {4096, 1000}};
+    for (int l = 0; l < 3; ++l) {
+        FcL& f = L.fc[l];
+        f.K = fcs[l][0]; f.N = fcs[l][1];
+        f.w_off = off; off = align_up(off + (long long)f.K * f.N, 64);
+        f.canon_w = canon; canon += (long long)f.K * f.N;
+        f.canon_b = canon; canon += f.N;
+    }
+    L.n_weights = off;
+    for (int l = 0; l < 5; ++l) { L.conv[l].b_off = off; off = align_up(off + L.conv[l].cout, 64); }
+    for (int l = 0; l < 3; ++l) { L.fc[l].b_off = off; off = align_up(off + L.fc[l].N, 64); }
+    L.n_total = off;
+    L.wt_total = wt;
+    // canonical -> internal segments, in canonical order
+    int s = 0;
+    for (int l = 0; l < 5; ++l) {
+        const ConvL& c = L.conv[l];
+        if (l == 0) L.segs.s[s++] = kn::ParamSeg{c.canon_w, c.w_off, 34848, 2, 0, 0, 0};
+        else L.segs.s[s++] = kn::ParamSeg{c.canon_w, c.w_off, canon_wcount[l], 1, c.cout, c.cig, c.k};
+        L.segs.s[s++] = kn::ParamSeg{c.canon_b, c.b_off, c.cout, 0, 0, 0, 0};
+    }
+    for (int l = 0; l < 3; ++l) {
+        const FcL& f = L.fc[l];
+        L.segs.s[s++] = kn::ParamSeg{f.canon_w, f.w_off, (long long)f.K * f.N, l == 0 ? 3 : 0, 0, 0, 0};
+        L.segs.s[s++] = kn::ParamSeg{f.canon_b, f.b_off, f.N, 0, 0, 0, 0};
+    }
+    L.tjobs.n = 4;
+    for (int l = 1; l < 5; ++l) {
+        const ConvL& c = L.conv[l];
+        L.tjobs.j[l - 1] = kn::TransposeJob{c.w_off, c.wt_off, c.taps, c.cout, c.cig, c.groups, (long long)c.taps * c.cin * c.cog};
+    }
+    return L;
+}
+const long long kCanonCount = 60965224;
+
+// ------------------------------------------------------------------- handle
+struct Plan { tc::GemmParams p; int grid; size_t smem; bool valid; };
+
+struct Tensor {  // description of one exportable device tensor
+    void* ptr; int kind; int C, Hp, Wp, H, W; long long N;
+};  // kind: 0 bf16 grid, 1 u8 compact NHWC, 2 bf16 [B][N], 3 f32 [B][N], 4 u8 [B][N], 5 s2d input, 6 int32 [B][3], 7 f32 [B]
+
+struct Replica {
+    float *w, *v, *g;
+    bf16 *shadow, *wt;
+    uint8_t* stage[2]; int32_t* labels[2]; bf16* x0[2]; int32_t* cf[2];
+    bf16 *a1, *n1, *p1, *a2, *n2, *p2, *a3, *a4, *a5, *p5, *f6, *f7;
+    float* z;
+    uint8_t *arg1, *arg2, *arg5, *m6, *m7;
+    bf16 *dz, *df7, *df6, *dp5, *da5, *da4, *da3, *dp2, *dn2, *da2, *dp1, *dn1, *da1;
+    float *loss_n, *loss;
+    // batch slots
+    cudaEvent_t ready[2], consumed[2];
+    bool consumed_valid[2];
+    uint64_t slot_step[2];
+    int next_load, next_train, loaded, last_slot;
+    // plans
+    Plan conv_fwd[5][2], conv_bwd[5], conv_wg[5][2], fc_fwd[3], fc_bwd[3], fc_wg[3];
+};
+
+}  // namespace
+
+struct alexnet {
+    alexnet_config_t cfg;
+    Layout L;
+    int B;
+    cudaStream_t cs, ls;   // compute, loader
+    uint8_t* arena; size_t arena_bytes;
+    Replica rep[2];
+    float* mean; float* ws; float* cs_partial; float* canon_tmp; int* status;
+    size_t ws_floats;
+    std::string err;
+    uint64_t launches;
+    int latched;
+    float alpha_eff, drop_scale; uint32_t thr24;
+    PFN_cuTensorMapEncodeTiled_v12000 encode;
+};
+
+namespace {
+
+int fail(alexnet* h, int code, const std::string& msg) { if (h) h->err = msg; return code; }
+#define CK(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(h, ALEXNET_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); } while (0)
+
+struct Carver {
+    uint8_t* base; size_t off;
+    template <typename T> T* take(size_t count) {
+        off = (off + 1023) / 1024 * 1024;
+        T* p = base ? (T*)(base + off) : nullptr;
+        off += count * sizeof(T);
+        return p;
+    }
+};
+
+int pick_splits(int tiles, int steps, int cap) {
+    int s = (296 + tiles - 1) / tiles;
+    if (s > cap) s = cap;
+    if (s > steps) s = steps;
+    if (s < 1) s = 1;
+    return s;
+}
+int conv_wg_splits(const ConvL& c, int B) {
+    const long long M = (long long)B * c.gin.Hp * c.gin.Wp;
+    const int steps = (int)((M + 63) / 64);
+    const int tiles = ((c.cog + 127) / 128) * c.groups * c.taps;
+    return pick_splits(tiles, steps, 16);
+}
+int fc_fwd_bn(const FcL&) { return 128; }
+int fc_fwd_splits(const FcL& f, int B) {
+    const int tiles = ((B + 127) / 128) * ((f.N + 127) / 128);
+    return pick_splits(tiles, f.K / 64, 16);
+}
+int fc_bwd_splits(const FcL& f, int B) {
+    const int tiles = ((B + 127) / 128) * (f.K / 256);
+    return pick_splits(tiles, (f.N + 63) / 64, 16);
+}
+size_t ws_need(const Layout& L, int B) {
+    size_t need = 0;
+    for (int l = 0; l < 5; ++l) {
+        const ConvL& c = L.conv[l];
+        need = std::max(need, (size_t)conv_wg_splits(c, B) * c.taps * c.cout * c.cig);
+    }
+    for (int l = 0; l < 3; ++l) {
+        need = std::max(need, (size_t)fc_fwd_splits(L.fc[l], B) * B * L.fc[l].N);
+        need = std::max(need, (size_t)fc_bwd_splits(L.fc[l], B) * B * L.fc[l].K);
+    }
+    return need;
+}
+
+// carve the arena; with base == nullptr only the size is computed
+size_t carve(alexnet* h, uint8_t* base) {
+    Carver c{base, 0};
+    const Layout& L = h->L;
+    const int B = h->B;
+    auto rows = [&](const Grid& g) { return (size_t)B * g.Hp * g.Wp; };
+    h->mean = c.take<float>(256 * 256 * 3);
+    h->ws_floats = ws_need(L, B);
+    h->ws = c.take<float>(h->ws_floats);
+    h->cs_partial = c.take<float>(256 * 4096);
+    h->canon_tmp = c.take<float>(kCanonCount);
+    h->status = c.take<int>(16);
+    for (int r = 0; r < h->cfg.replicas; ++r) {
+        Replica& R = h->rep[r];
+        R.w = c.take<float>(L.n_total); R.v = c.take<float>(L.n_total); R.g = c.take<float>(L.n_total);
+        R.shadow = c.take<bf16>(L.n_total); R.wt = c.take<bf16>(L.wt_total);
+        for (int s = 0; s < 2; ++s) {
+            R.stage[s] = c.take<uint8_t>((size_t)B * 196608);
+            R.labels[s] = c.take<int32_t>(B);
+            R.x0[s] = c.take<bf16>(rows(L.conv[0].gin) * 48);
+            R.cf[s] = c.take<int32_t>(3 * B);
+        }
+        const size_t r1 = rows(L.conv[0].gout), r2 = rows(L.conv[1].gout), r3 = rows(L.conv[2].gout);
+        R.a1 = c.take<bf16>(r1 * 96); R.n1 = c.take<bf16>(r1 * 96); R.p1 = c.take<bf16>(r2 * 96);
+        R.a2 = c.take<bf16>(r2 * 256); R.n2 = c.take<bf16>(r2 * 256); R.p2 = c.take<bf16>(r3 * 256);
+        R.a3 = c.take<bf16>(r3 * 384); R.a4 = c.take<bf16>(r3 * 384); R.a5 = c.take<bf16>(r3 * 256);
+        R.p5 = c.take<bf16>((size_t)B * 9216); R.f6 = c.take<bf16>((size_t)B * 4096); R.f7 = c.take<bf16>((size_t)B * 4096);
+        R.z = c.take<float>((size_t)B * 1000);
+        R.arg1 = c.take<uint8_t>((size_t)B * 27 * 27 * 96); R.arg2 = c.take<uint8_t>((size_t)B * 13 * 13 * 256);
+        R.arg5 = c.take<uint8_t>((size_t)B * 9216);
+        R.m6 = c.take<uint8_t>((size_t)B * 4096); R.m7 = c.take<uint8_t>((size_t)B * 4096);
+        R.dz = c.take<bf16>((size_t)B * 1000); R.df7 = c.take<bf16>((size_t)B * 4096); R.df6 = c.take<bf16>((size_t)B * 4096);
+        R.dp5 = c.take<bf16>((size_t)B * 9216);
+        R.da5 = c.take<bf16>(r3 * 256); R.da4 = c.take<bf16>(r3 * 384); R.da3 = c.take<bf16>(r3 * 384);
+        R.dp2 = c.take<bf16>(r3 * 256); R.dn2 = c.take<bf16>(r2 * 256); R.da2 = c.take<bf16>(r2 * 256);
+        R.dp1 = c.take<bf16>(r2 * 96); R.dn1 = c.take<bf16>(r1 * 96); R.da1 = c.take<bf16>(r1 * 96);
+        R.loss_n = c.take<float>(B); R.loss = c.take<float>(16);
+    }
+    return (c.off + 1023) / 1024 * 1024;
+}
+
+int check_cfg(const alexnet_config_t* c) {
+    if (!c) return 0;
+    if (c->batch < 1 || c->batch > 1024) return 0;
+    if (c->replicas < 1 || c->replicas > 2) return 0;
+    if (c->lrn_size != 5) return 0;
+    if (!(c->dropout_p >= 0.f && c->dropout_p < 1.f)) return 0;
+    if (!(c->lrn_k > 0.f)) return 0;
+    return 1;
+}
+
+// ------------------------------------------------------------------- plans
+int make_tm(alexnet* h, CUtensorMap* tm, const void* ptr, uint64_t cols, uint64_t rows, uint64_t pitch_bytes, uint32_t box_rows) {
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {pitch_bytes};
+    cuuint32_t box[2] = {64, box_rows};
+    cuuint32_t es[2] = {1, 1};
+    CUresult r = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)ptr, dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(h, ALEXNET_ERR_CUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+    return ALEXNET_OK;
+}
+
+void finish_plan(Plan& P) {
+    tc::GemmParams& p = P.p;
+    const int stage_bytes = tc::kABytes + tc::b_stage_bytes(p.mode, p.BN);
+    int stages = (227 * 1024 - 2048) / stage_bytes;
+    if (stages > 6) stages = 6;
+    const int per = (p.steps_total + p.splits - 1) / p.splits;
+    if (stages > per) stages = per < 2 ? 2 : per;
+    p.stages = stages;
+    P.smem = tc::smem_bytes(p.mode, p.BN, stages);
+    P.grid = p.m_tiles * p.n_tiles * p.groups * p.taps_grid * p.splits;
+    P.valid = true;
+}
+
+int plan_conv_fwd(alexnet* h, Plan& P, const ConvL& c, const bf16* in, const bf16* wsh, const float* bias, bf16* out) {
+    memset(&P, 0, sizeof(P));
+    tc::GemmParams& p = P.p;
+    const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
+    p.mode = tc::MODE_KK; p.epi = tc::EPI_BF16;
+    p.M_total = (int)M; p.m_tiles = (int)((M + 127) / 128);
+    p.BN = c.cog <= 256 ? c.cog : 192; p.n_tiles = c.cog / p.BN;
+    p.groups = c.groups; p.taps_grid = 1; p.splits = 1;
+    p.kk = c.cig == 48 ? 3 : 4; p.chunks = (c.cig + 63) / 64; p.steps_total = c.taps * p.chunks;
+    p.a_x0 = 0; p.a_gx = c.cig; p.b_tap_rows = c.cout; p.b_g_rows = c.cog;
+    for (int t = 0; t < c.taps; ++t) p.shift[t] = c.shift[t];
+    p.n_valid = c.cog; p.ldo = c.cout; p.out_gx = c.cog;
+    p.Hp = c.gout.Hp; p.Wp = c.gout.Wp; p.H = c.gout.H; p.W = c.gout.W;
+    p.relu = 1; p.mask_scale = 1.f; p.bias = bias; p.mask = nullptr; p.out = out; p.status = h->status;
+    int rc;
+    if ((rc = make_tm(h, &p.tmA, in, c.cin, M, (uint64_t)c.cin * 2, 128))) return rc;
+    if ((rc = make_tm(h, &p.tmB, wsh, c.cig, (uint64_t)c.taps * c.cout, (uint64_t)c.cig * 2, p.BN))) return rc;
+    finish_plan(P);
+    return ALEXNET_OK;
+}
+int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16* wt, const bf16* mask, bf16* dx) {
+    memset(&P, 0, sizeof(P));
+    tc::GemmParams& p = P.p;
+    const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
+    p.mode = tc::MODE_KK; p.epi = tc::EPI_BF16;
+    p.M_total = (int)M; p.m_tiles = (int)((M + 127) / 128);
+    p.BN = c.cig; p.n_tiles = 1; p.groups = c.groups; p.taps_grid = 1; p.splits = 1;
+    p.kk = 4; p.chunks = c.cog / 64; p.steps_total = c.taps * p.chunks;
+    p.a_x0 = 0; p.a_gx = c.cog; p.b_tap_rows = c.cin; p.b_g_rows = c.cig;
+    for (int t = 0; t < c.taps; ++t) p.shift[t] = -c.shift[t];
+    p.n_valid = c.cig; p.ldo = c.cin; p.out_gx = c.cig;
+    p.Hp = c.gin.Hp; p.Wp = c.gin.Wp; p.H = c.gin.H; p.W = c.gin.W;
+    p.relu = 0; p.mask_scale = 1.f; p.bias = nullptr; p.mask = mask; p.out = dx; p.status = h->status;
+    int rc;
+    if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, 128))) return rc;
+    if ((rc = make_tm(h, &p.tmB, wt, c.cog, (uint64_t)c.taps * c.cin, (uint64_t)c.cog * 2, p.BN))) return rc;
+    finish_plan(P);
+    return ALEXNET_OK;
+}
+int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16* xin) {
+    memset(&P, 0, sizeof(P));
+    tc::GemmParams& p = P.p;
+    const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
+    p.mode = tc::MODE_MNMN; p.epi = tc::EPI_F32;
+    p.M_total = c.cog; p.m_tiles = (c.cog + 127) / 128; p.BN = c.cig; p.n_tiles = 1;
+    p.groups = c.groups; p.taps_grid = c.taps; p.steps_total = (int)((M + 63) / 64);
+    p.splits = conv_wg_splits(c, h->B); p.kk = 4; p.chunks = 1;
+    p.a_gx = c.cog; p.b_gx = c.cig;
+    for (int t = 0; t < c.taps; ++t) p.shift[t] = c.shift[t];
+    p.n_valid = c.cig; p.ldo = c.cig; p.out_gx = c.cog;
+    p.tap_stride = (long long)c.cout * c.cig; p.split_stride = (long long)c.taps * c.cout * c.cig;
+    p.out = h->ws; p.status = h->status;
+    int rc;
+    if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, 64))) return rc;
+    if ((rc = make_tm(h, &p.tmB, xin, c.cin, M, (uint64_t)c.cin * 2, 64))) return rc;
+    finish_plan(P);
+    return ALEXNET_OK;
+}
+int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* wsh) {
+    memset(&P, 0, sizeof(P));
+    tc::GemmParams& p = P.p;
+    const int B = h->B;
+    p.mode = tc::MODE_KK; p.epi = tc::EPI_F32;
+    p.M_total = B; p.m_tiles = (B + 127) / 128; p.BN = fc_fwd_bn(f); p.n_tiles = (f.N + p.BN - 1) / p.BN;
+    p.groups = 1; p.taps_grid = 1; p.splits = fc_fwd_splits(f, B);
+    p.kk = 4; p.chunks = f.K / 64; p.steps_total = p.chunks;
+    p.n_valid = f.N; p.ldo = f.N; p.split_stride = (long long)B * f.N;
+    p.out = h->ws; p.status = h->status;
+    int rc;
+    if ((rc = make_tm(h, &p.tmA, x, f.K, B, (uint64_t)f.K * 2, 128))) return rc;
+    if ((rc = make_tm(h, &p.tmB, wsh, f.K, f.N, (uint64_t)f.K * 2, p.BN))) return rc;
+    finish_plan(P);
+    return ALEXNET_OK;
+}
+int plan_fc_bwd(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* wsh) {
+    memset(&P, 0, sizeof(P));
+    tc::GemmParams& p = P.p;
+    const int B = h->B;
+    p.mode = tc::MODE_KMN; p.epi = tc::EPI_F32;
+    p.M_total = B; p.m_tiles = (B + 127) / 128; p.BN = 256; p.n_tiles = f.K / 256;
+    p.groups = 1; p.taps_grid = 1; p.splits = fc_bwd_splits(f, B);
+    p.kk = 4; p.chunks = 1; p.steps_total = (f.N + 63) / 64;
+    p.n_valid = f.K; p.ldo = f.K; p.split_stride = (long long)B * f.K;
+    p.out = h->ws; p.status = h->status;
+    int rc;
+    if ((rc = make_tm(h, &p.tmA, dy, f.N, B, (uint64_t)f.N * 2, 128))) return rc;
+    if ((rc = make_tm(h, &p.tmB, wsh, f.K, f.N, (uint64_t)f.K * 2, 64))) return rc;
+    finish_plan(P);
+    return ALEXNET_OK;
+}
+int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x, float* gout) {
+    memset(&P, 0, sizeof(P));
+    tc::GemmParams& p = P.p;
+    const int B = h->B;
+    p.mode = tc::MODE_MNMN; p.epi = tc::EPI_F32;
+    p.M_total = f.N; p.m_tiles = (f.N + 127) / 128; p.BN = 256; p.n_tiles = f.K / 256;
+    p.groups = 1; p.taps_grid = 1; p.splits = 1; p.kk = 4; p.chunks = 1; p.steps_total = (B + 63) / 64;
+    p.n_valid = f.K; p.ldo = f.K;
+    p.out = gout; p.status = h->status;
+    int rc;
+    if ((rc = make_tm(h, &p.tmA, dy, f.N, B, (uint64_t)f.N * 2, 64))) return rc;
+    if ((rc = make_tm(h, &p.tmB, x, f.K, B, (uint64_t)f.K * 2, 64))) return rc;
+    finish_plan(P);
+    return ALEXNET_OK;
+}
+
+int build_plans(alexnet* h, int r) {
+    Replica& R = h->rep[r];
+    const Layout& L = h->L;
+    const bf16* in[5] = {nullptr, R.p1, R.p2, R.a3, R.a4};
+    bf16* out[5] = {R.a1, R.a2, R.a3, R.a4, R.a5};
+    bf16* dyv[5] = {R.da1, R.da2, R.da3, R.da4, R.da5};
+    bf16* dxv[5] = {nullptr, R.dp1, R.dp2, R.da3, R.da4};
+    const bf16* maskv[5] = {nullptr, nullptr, nullptr, R.a3, R.a4};
+    int rc;
+    for (int l = 0; l < 5; ++l) {
+        const ConvL& c = L.conv[l];
+        for (int s = 0; s < 2; ++s) {
+            const bf16* x = l == 0 ? R.x0[s] : in[l];
+            if ((rc = plan_conv_fwd(h, R.conv_fwd[l][s], c, x, R.shadow + c.w_off, R.w + c.b_off, out[l]))) return rc;
+            if ((rc = plan_conv_wg(h, R.conv_wg[l][s], c, dyv[l], x))) return rc;
+        }
+        if (l > 0 && (rc = plan_conv_bwd(h, R.conv_bwd[l], c, dyv[l], R.wt + c.wt_off, maskv[l], dxv[l]))) return rc;
+    }
+    const bf16* fx[3] = {R.p5, R.f6, R.f7};
+    const bf16* fdy[3] = {R.df6, R.df7, R.dz};
+    for (int l = 0; l < 3; ++l) {
+        const FcL& f = L.fc[l];
+        if ((rc = plan_fc_fwd(h, R.fc_fwd[l], f, fx[l], R.shadow + f.w_off))) return rc;
+        if ((rc = plan_fc_bwd(h, R.fc_bwd[l], f, fdy[l], R.shadow + f.w_off))) return rc;
+        if ((rc = plan_fc_wg(h, R.fc_wg[l], f, fdy[l], fx[l], R.g + f.w_off))) return rc;
+    }
+    return ALEXNET_OK;
+}
+
+// ---------------------------------------------------------------- launches
+inline int nblk(long long n, int t) { return (int)((n + t - 1) / t); }
+
+void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
+    tc::gemm_kernel<<<P.grid, tc::kThreads, P.smem, st>>>(P.p);
+    h->launches++;
+}
+void colsum(alexnet* h, const bf16* dy, long long rows, int C, float* db, cudaStream_t st) {
+    if (C % 8) {
+        kn::colsum_scalar_kernel<<<nblk(C, 128), 128, 0, st>>>(dy, (int)rows, C, db);
+        h->launches++;
+        return;
+    }
+    int splits = (int)std::min<long long>(256, std::max<long long>(1, rows / 256));
+    dim3 grid((C + 63) / 64, splits);
+    kn::colsum_kernel<<<grid, 256, 0, st>>>(dy, rows, C, h->cs_partial);
+    kn::colsum_final_kernel<<<nblk(C, 128), 128, 0, st>>>(h->cs_partial, splits, C, db);
+    h->launches += 2;
+}
+void refresh_shadows(alexnet* h, int r, bool whole, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    if (whole) {
+        kn::shadow_kernel<<<1184, 256, 0, st>>>(R.w, R.shadow, h->L.n_total / 4);
+        h->launches++;
+    }
+    kn::conv_transpose_shadow_kernel<<<592, 256, 0, st>>>(R.shadow, R.wt, h->L.tjobs);
+    h->launches++;
+}
+
+void op_conv_fwd(alexnet* h, int r, int l, int slot, cudaStream_t st) { launch_gemm(h, h->rep[r].conv_fwd[l][slot], st); }
+void op_conv_bwd(alexnet* h, int r, int l, cudaStream_t st) { launch_gemm(h, h->rep[r].conv_bwd[l], st); }
+void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const ConvL& c = h->L.conv[l];
+    const Plan& P = R.conv_wg[l][slot];
+    launch_gemm(h, P, st);
+    const long long total = (long long)c.taps * c.cout * c.cig;
+    kn::wgrad_reduce_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, total, R.g + c.w_off, l == 0);
+    h->launches++;
+    bf16* dyv[5] = {R.da1, R.da2, R.da3, R.da4, R.da5};
+    colsum(h, dyv[l], (long long)h->B * c.gout.Hp * c.gout.Wp, c.cout, R.g + c.b_off, st);
+}
+void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const FcL& f = h->L.fc[l];
+    const Plan& P = R.fc_fwd[l];
+    launch_gemm(h, P, st);
+    const long long total = (long long)h->B * f.N;
+    bf16* outs[3] = {R.f6, R.f7, nullptr};
+    uint8_t* keeps[3] = {R.m6, R.m7, nullptr};
+    const int drop = l < 2 && h->cfg.dropout_p > 0.f;
+    const uint64_t key = kn::stream_key(h->cfg.seed, 2 + l, r, step);
+    kn::fc_reduce_fwd_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, R.w + f.b_off, h->B, f.N,
+                                                                l < 2, drop, key, h->thr24, h->drop_scale, outs[l],
+                                                                l == 2 ? R.z : nullptr, keeps[l]);
+    h->launches++;
+}
+void op_fc_bwd(alexnet* h, int r, int l, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const FcL& f = h->L.fc[l];
+    const Plan& P = R.fc_bwd[l];
+    launch_gemm(h, P, st);
+    const long long total = (long long)h->B * f.K;
+    const bf16* masks[3] = {nullptr, R.f6, R.f7};
+    bf16* outs[3] = {R.dp5, R.df6, R.df7};
+    kn::fc_reduce_bwd_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, masks[l], h->drop_scale, total, outs[l]);
+    h->launches++;
+}
+void op_fc_wg(alexnet* h, int r, int l, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const FcL& f = h->L.fc[l];
+    launch_gemm(h, R.fc_wg[l], st);
+    const bf16* dyv[3] = {R.df6, R.df7, R.dz};
+    colsum(h, dyv[l], h->B, f.N, R.g + f.b_off, st);
+}
+void op_lrn_fwd(alexnet* h, int r, int which, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const Grid& g = h->L.conv[which].gout;
+    const long long rows = (long long)h->B * g.Hp * g.Wp;
+    kn::lrn_fwd_kernel<<<nblk(rows * (g.C / 8), 256), 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.n2 : R.n1, rows, g.C,
+                                                                   h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
+    h->launches++;
+}
+void op_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const Grid& g = h->L.conv[which].gout;
+    const long long rows = (long long)h->B * g.Hp * g.Wp;
+    kn::lrn_bwd_kernel<<<nblk(rows * (g.C / 8), 256), 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.dn2 : R.dn1,
+                                                                   which ? R.da2 : R.da1, rows, g.C, h->alpha_eff,
+                                                                   h->cfg.lrn_beta, h->cfg.lrn_k);
+    h->launches++;
+}
+struct PoolGeo { int C, Hpi, Wpi, Hi, Wi, Ho, Wo, Hpo, Wpo; };
+const PoolGeo kPool[3] = {{96, 57, 57, 55, 55, 27, 27, 29, 29}, {256, 29, 29, 27, 27, 13, 13, 14, 14}, {256, 14, 14, 13, 13, 6, 6, 6, 6}};
+void op_pool_fwd(alexnet* h, int r, int which, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const PoolGeo& g = kPool[which];
+    const bf16* x[3] = {R.n1, R.n2, R.a5};
+    bf16* y[3] = {R.p1, R.p2, R.p5};
+    uint8_t* a[3] = {R.arg1, R.arg2, R.arg5};
+    const long long total = (long long)h->B * g.Ho * g.Wo * (g.C / 8);
+    kn::pool_fwd_kernel<<<nblk(total, 256), 256, 0, st>>>(x[which], y[which], a[which], h->B, g.C, g.Hpi, g.Wpi, g.Ho, g.Wo, g.Hpo, g.Wpo);
+    h->launches++;
+}
+void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const PoolGeo& g = kPool[which];
+    const bf16* dy[3] = {R.dp1, R.dp2, R.dp5};
+    const uint8_t* a[3] = {R.arg1, R.arg2, R.arg5};
+    const bf16* relu[3] = {nullptr, nullptr, R.a5};
+    bf16* dx[3] = {R.dn1, R.dn2, R.da5};
+    const long long total = (long long)h->B * g.Hpi * g.Wpi * (g.C / 8);
+    kn::pool_bwd_kernel<<<nblk(total, 256), 256, 0, st>>>(dy[which], a[which], relu[which], dx[which], h->B, g.C, g.Hpi, g.Wpi,
+                                                          g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo, g.Wpo);
+    h->launches++;
+}
+void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    kn::softmax_xent_kernel<<<h->B, 256, 0, st>>>(R.z, R.labels[slot], R.dz, R.loss_n, h->B, 1000);
+    kn::mean_kernel<<<1, 256, 0, st>>>(R.loss_n, h->B, R.loss);
+    h->launches += 2;
+}
+void op_update(alexnet* h, int r, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const long long nd = (h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES) ? h->L.n_total : h->L.n_weights;
+    kn::sgd_update_kernel<<<1184, 256, 0, st>>>(R.w, R.v, R.g, R.shadow, h->L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum,
+                                                h->cfg.weight_decay);
+    h->launches++;
+    refresh_shadows(h, r, false, st);
+}
+void op_average(alexnet* h, cudaStream_t st) {
+    Replica &A = h->rep[0], &Bq = h->rep[1];
+    kn::replica_average_kernel<<<1184, 256, 0, st>>>(A.w, Bq.w, A.v, Bq.v, A.shadow, Bq.shadow, h->L.n_total / 4);
+    h->launches++;
+    refresh_shadows(h, 0, false, st);
+    refresh_shadows(h, 1, false, st);
+}
+void op_preprocess(alexnet* h, int r, int slot, uint64_t step, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const long long total = (long long)h->B * 57 * 57 * 4;
+    kn::preprocess_kernel<<<nblk(total, 256), 256, 0, st>>>(R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
+                                                            kn::stream_key(h->cfg.seed, 1, r, step));
+    h->launches++;
+}
+
+void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const uint64_t step = R.slot_step[slot];
+    op_conv_fwd(h, r, 0, slot, st); op_lrn_fwd(h, r, 0, st); op_pool_fwd(h, r, 0, st);
+    op_conv_fwd(h, r, 1, slot, st); op_lrn_fwd(h, r, 1, st); op_pool_fwd(h, r, 1, st);
+    op_conv_fwd(h, r, 2, slot, st); op_conv_fwd(h, r, 3, slot, st); op_conv_fwd(h, r, 4, slot, st);
+    op_pool_fwd(h, r, 2, st);
+    op_fc_fwd(h, r, 0, step, st); op_fc_fwd(h, r, 1, step, st); op_fc_fwd(h, r, 2, step, st);
+    op_softmax(h, r, slot, st);
+    op_fc_wg(h, r, 2, st); op_fc_bwd(h, r, 2, st);
+    op_fc_wg(h, r, 1, st); op_fc_bwd(h, r, 1, st);
+    op_fc_wg(h, r, 0, st); op_fc_bwd(h, r, 0, st);
+    op_pool_bwd(h, r, 2, st);
+    op_conv_wg(h, r, 4, slot, st); op_conv_bwd(h, r, 4, st);
+    op_conv_wg(h, r, 3, slot, st); op_conv_bwd(h, r, 3, st);
+    op_conv_wg(h, r, 2, slot, st); op_conv_bwd(h, r, 2, st);
+    op_pool_bwd(h, r, 1, st); op_lrn_bwd(h, r, 1, st);
+    op_conv_wg(h, r, 1, slot, st); op_conv_bwd(h, r, 1, st);
+    op_pool_bwd(h, r, 0, st); op_lrn_bwd(h, r, 0, st);
+    op_conv_wg(h, r, 0, slot, st);
+}
+
+int check_status(alexnet* h) {
+    if (h->latched) return h->latched;
+    return ALEXNET_OK;
+}
+int poll_status(alexnet* h) {  // after a synchronisation
+    int st = 0;
+    cudaError_t e = cudaMemcpy(&st, h->status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail(h, ALEXNET_ERR_CUDA, std::string("status read: ") + cudaGetErrorString(e));
+    if (st) { h->latched = ALEXNET_ERR_DEVICE_TIMEOUT; return fail(h, ALEXNET_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired"); }
+    return ALEXNET_OK;
+}
+
+// N(0, std^2) init from the hash (stream 6), identical in every replica; written at internal positions
+__global__ void init_kernel(float* arena, const kn::ParamSegs segs, uint64_t key, float std_) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    const long long total = 60965224;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        int s = 0;
+        while (s < 15 && i >= segs.s[s + 1].canon_off) ++s;
+        float val = 0.f;
+        if ((s & 1) == 0) {  // weight segments
+            const uint64_t r = kn::draw(key, (uint64_t)i);
+            const float u1 = ((float)(r >> 40) + 1.f) * (1.f / 16777216.f);
+            const float u2 = (float)((r >> 16) & 0xFFFFFF) * (1.f / 16777216.f);
+            val = std_ * sqrtf(-2.f * logf(u1)) * cospif(2.f * u2);
+        }
+        arena[kn::canon_to_internal(segs.s[s], i - segs.s[s].canon_off)] = val;
+    }
+}
+
+// -------------------------------------------------------------- tensor table
+bool tensor_desc(alexnet* h, int r, int id, Tensor* T) {
+    Replica& R = h->rep[r];
+    const int ls = R.last_slot;
+    auto grid = [&](void* p, const Grid& g, int C) { *T = Tensor{p, 0, C, g.Hp, g.Wp, g.H, g.W, 0}; };
+    const Grid g1 = h->L.conv[0].gout, g2 = h->L.conv[1].gout, g3 = h->L.conv[2].gout;
+    const Grid gp5 = Grid{6, 6, 6, 6, 256};
+    switch (id) {
+        case ALEXNET_T_CROPFLIP: *T = Tensor{R.cf[ls], 6, 0, 0, 0, 0, 0, 3}; return true;
+        case ALEXNET_T_X0: *T = Tensor{R.x0[ls], 5, 3, 57, 57, 227, 227, 0}; return true;
+        case ALEXNET_T_A1: grid(R.a1, g1, 96); return true;
+        case ALEXNET_T_N1: grid(R.n1, g1, 96); return true;
+        case ALEXNET_T_P1: grid(R.p1, g2, 96); return true;
+        case ALEXNET_T_ARG1: *T = Tensor{R.arg1, 1, 96, 27, 27, 27, 27, 0}; return true;
+        case ALEXNET_T_A2: grid(R.a2, g2, 256); return true;
+        case ALEXNET_T_N2: grid(R.n2, g2, 256); return true;
+        case ALEXNET_T_P2: grid(R.p2, g3, 256); return true;
+        case ALEXNET_T_ARG2: *T = Tensor{R.arg2, 1, 256, 13, 13, 13, 13, 0}; return true;
+        case ALEXNET_T_A3: grid(R.a3, g3, 384); return true;
+        case ALEXNET_T_A4: grid(R.a4, g3, 384); return true;
+        case ALEXNET_T_A5: grid(R.a5, g3, 256); return true;
+        case ALEXNET_T_P5: grid(R.p5, gp5, 256); return true;
+        case ALEXNET_T_ARG5: *T = Tensor{R.arg5, 1, 256, 6, 6, 6, 6, 0}; return true;
+        case ALEXNET_T_F6: *T = Tensor{R.f6, 2, 0, 0, 0, 0, 0, 4096}; return true;
+        case ALEXNET_T_F7: *T = Tensor{R.f7, 2, 0, 0, 0, 0, 0, 4096}; return true;
+        case ALEXNET_T_Z: *T = Tensor{R.z, 3, 0, 0, 0, 0, 0, 1000}; return true;
+        case ALEXNET_T_M6: *T = Tensor{R.m6, 4, 0, 0, 0, 0, 0, 4096}; return true;
+        case ALEXNET_T_M7: *T = Tensor{R.m7, 4, 0, 0, 0, 0, 0, 4096}; return true;
+        case ALEXNET_T_DZ: *T = Tensor{R.dz, 2, 0, 0, 0, 0, 0, 1000}; return true;
+        case ALEXNET_T_DF7: *T = Tensor{R.df7, 2, 0, 0, 0, 0, 0, 4096}; return true;
+        case ALEXNET_T_DF6: *T = Tensor{R.df6, 2, 0, 0, 0, 0, 0, 4096}; return true;
+        case ALEXNET_T_DP5: grid(R.dp5, gp5, 256); return true;
+        case ALEXNET_T_DA5: grid(R.da5, g3, 256); return true;
+        case ALEXNET_T_DA4: grid(R.da4, g3, 384); return true;
+        case ALEXNET_T_DA3: grid(R.da3, g3, 384); return true;
+        case ALEXNET_T_DP2: grid(R.dp2, g3, 256); return true;
+        case ALEXNET_T_DN2: grid(R.dn2, g2, 256); return true;
+        case ALEXNET_T_DA2: grid(R.da2, g2, 256); return true;
+        case ALEXNET_T_DP1: grid(R.dp1, g2, 96); return true;
+        case ALEXNET_T_DN1: grid(R.dn1, g1, 96); return true;
+        case ALEXNET_T_DA1: grid(R.da1, g1, 96); return true;
+        case ALEXNET_T_LOSS: *T = Tensor{R.loss_n, 7, 0, 0, 0, 0, 0, 1}; return true;
+    }
+    return false;
+}
+size_t tensor_elems(const Tensor& T, int B) {  // canonical element count
+    switch (T.kind) {
+        case 0: case 1: return (size_t)B * T.C * T.H * T.W;
+        case 5: return (size_t)B * 3 * 227 * 227;
+        default: return (size_t)B * T.N;
+    }
+}
+size_t tensor_dev_bytes(const Tensor& T, int B) {
+    switch (T.kind) {
+        case 0: return (size_t)B * T.Hp * T.Wp * T.C * 2;
+        case 1: return (size_t)B * T.H * T.W * T.C;
+        case 2: return (size_t)B * T.N * 2;
+        case 3: case 7: return (size_t)B * T.N * 4;
+        case 4: return (size_t)B * T.N;
+        case 5: return (size_t)B * 57 * 57 * 48 * 2;
+        case 6: return (size_t)B * 3 * 4;
+    }
+    return 0;
+}
+inline float bf2f(uint16_t b) { uint32_t u = (uint32_t)b << 16; float f; memcpy(&f, &u, 4); return f; }
+inline uint16_t f2bf(float f) {
+    uint32_t u; memcpy(&u, &f, 4);
+    u = u + 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(u >> 16);
+}
+
+}  // namespace
+
+// =========================================================================== C ABI
+extern "C" {
+
+size_t alexnet_param_count(void) { return (size_t)kCanonCount; }
+
+size_t alexnet_workspace_bytes(const alexnet_config_t* cfg) {
+    if (!check_cfg(cfg)) return 0;
+    alexnet tmp;
+    tmp.cfg = *cfg; tmp.B = cfg->batch; tmp.L = make_layout();
+    return carve(&tmp, nullptr);
+}
+
+int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_bytes, const float* host_mean_image,
+                   void* compute_stream, void* copy_stream, alexnet_t** out) {
+    if (!out) return ALEXNET_ERR_ARG;
+    *out = nullptr;
+    if (!check_cfg(cfg) || !dev_arena || ((uintptr_t)dev_arena & 1023)) return ALEXNET_ERR_ARG;
+    alexnet* h = new alexnet();
+    h->cfg = *cfg; h->B = cfg->batch; h->L = make_layout();
+    h->cs = (cudaStream_t)compute_stream; h->ls = (cudaStream_t)copy_stream;
+    h->launches = 0; h->latched = 0;
+    h->alpha_eff = (cfg->flags & ALEXNET_FLAG_LRN_ALPHA_DIV_N) ? cfg->lrn_alpha / 5.f : cfg->lrn_alpha;
+    h->drop_scale = ((cfg->flags & ALEXNET_FLAG_INVERTED_DROPOUT) && cfg->dropout_p > 0.f) ? 1.f / (1.f - cfg->dropout_p) : 1.f;
+    h->thr24 = (uint32_t)floor((double)cfg->dropout_p * 16777216.0);
+    const size_t need = carve(h, nullptr);
+    if (arena_bytes < need) { delete h; return ALEXNET_ERR_NOMEM; }
+    h->arena = (uint8_t*)dev_arena; h->arena_bytes = arena_bytes;
+    carve(h, h->arena);
+#define CKC(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { fprintf(stderr, "alexnet_create: %s: %s\n", #call, cudaGetErrorString(e_)); delete h; return ALEXNET_ERR_CUDA; } } while (0)
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CKC(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) { delete h; return ALEXNET_ERR_CUDA; }
+    h->encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+    CKC(cudaFuncSetAttribute(tc::gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    // pad positions of every grid must be zero from the start; gradients and momentum start at zero
+    CKC(cudaMemsetAsync(h->arena, 0, need, h->cs));
+    if (host_mean_image) CKC(cudaMemcpyAsync(h->mean, host_mean_image, 256 * 256 * 3 * sizeof(float), cudaMemcpyHostToDevice, h->cs));
+    for (int r = 0; r < cfg->replicas; ++r) {
+        Replica& R = h->rep[r];
+        R.next_load = R.next_train = R.loaded = R.last_slot = 0;
+        for (int s = 0; s < 2; ++s) {
+            CKC(cudaEventCreateWithFlags(&R.ready[s], cudaEventDisableTiming));
+            CKC(cudaEventCreateWithFlags(&R.consumed[s], cudaEventDisableTiming));
+            R.consumed_valid[s] = false; R.slot_step[s] = 0;
+        }
+        if (cfg->init_std > 0.f) {
+            init_kernel<<<1184, 256, 0, h->cs>>>(R.w, h->L.segs, kn::stream_key(cfg->seed, 6, 0, 0), cfg->init_std);
+            h->launches++;
+        }
+        refresh_shadows(h, r, true, h->cs);
+        int rc = build_plans(h, r);
+        if (rc) { fprintf(stderr, "alexnet_create: %s\n", h->err.c_str()); delete h; return rc; }
+    }
+    CKC(cudaStreamSynchronize(h->cs));
+    CKC(cudaGetLastError());
+    *out = h;
+    return ALEXNET_OK;
+}
+
+int alexnet_destroy(alexnet_t* h) {
+    if (!h) return ALEXNET_ERR_ARG;
+    cudaStreamSynchronize(h->cs);
+    cudaStreamSynchronize(h->ls);
+    for (int r = 0; r < h->cfg.replicas; ++r)
+        for (int s = 0; s < 2; ++s) { cudaEventDestroy(h->rep[r].ready[s]); cudaEventDestroy(h->rep[r].consumed[s]); }
+    delete h;
+    return ALEXNET_OK;
+}
+
+int alexnet_load_batch_async(alexnet_t* h, int replica, const uint8_t* images, const int32_t* labels, uint64_t step) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas || !images || !labels) return fail(h, ALEXNET_ERR_ARG, "load_batch_async: bad argument");
+    if (int rc = check_status(h)) return rc;
+    Replica& R = h->rep[replica];
+    if (R.loaded == 2) return fail(h, ALEXNET_ERR_STATE, "load_batch_async: both batch slots hold unconsumed batches");
+    const int s = R.next_load;
+    if (R.consumed_valid[s]) CK(cudaStreamWaitEvent(h->ls, R.consumed[s], 0));
+    CK(cudaMemcpyAsync(R.stage[s], images, (size_t)h->B * 196608, cudaMemcpyDefault, h->ls));
+    CK(cudaMemcpyAsync(R.labels[s], labels, (size_t)h->B * sizeof(int32_t), cudaMemcpyDefault, h->ls));
+    op_preprocess(h, replica, s, step, h->ls);
+    CK(cudaEventRecord(R.ready[s], h->ls));
+    R.slot_step[s] = step;
+    R.last_slot = s; R.next_load ^= 1; R.loaded++;
+    return ALEXNET_OK;
+}
+
+int alexnet_train_step(alexnet_t* h, int replica, float* host_loss) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas) return fail(h, ALEXNET_ERR_ARG, "train_step: bad replica");
+    if (int rc = check_status(h)) return rc;
+    Replica& R = h->rep[replica];
+    if (R.loaded == 0) return fail(h, ALEXNET_ERR_STATE, "train_step: no loaded batch");
+    const int s = R.next_train;
+    CK(cudaStreamWaitEvent(h->cs, R.ready[s], 0));
+    forward_backward(h, replica, s, h->cs);
+    CK(cudaEventRecord(R.consumed[s], h->cs));
+    R.consumed_valid[s] = true;
+    op_update(h, replica, h->cs);
+    R.last_slot = s; R.next_train ^= 1; R.loaded--;
+    CK(cudaGetLastError());
+    if (host_loss) {
+        CK(cudaMemcpyAsync(host_loss, R.loss, sizeof(float), cudaMemcpyDeviceToHost, h->cs));
+        CK(cudaStreamSynchronize(h->cs));
+        return poll_status(h);
+    }
+    return ALEXNET_OK;
+}
+
+int alexnet_replica_average(alexnet_t* h) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (int rc = check_status(h)) return rc;
+    if (h->cfg.replicas < 2) return ALEXNET_OK;
+    op_average(h, h->cs);
+    CK(cudaGetLastError());
+    return ALEXNET_OK;
+}
+
+int alexnet_get_params(alexnet_t* h, int replica, int which, float* host_out, size_t n) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas || which < 0 || which > 2 || !host_out || n != (size_t)kCanonCount)
+        return fail(h, ALEXNET_ERR_ARG, "get_params: bad argument");
+    Replica& R = h->rep[replica];
+    const float* src = which == 0 ? R.w : which == 1 ? R.v : R.g;
+    kn::params_gather_kernel<<<1184, 256, 0, h->cs>>>(src, h->canon_tmp, h->L.segs, kCanonCount);
+    h->launches++;
+    CK(cudaMemcpyAsync(host_out, h->canon_tmp, n * sizeof(float), cudaMemcpyDeviceToHost, h->cs));
+    CK(cudaStreamSynchronize(h->cs));
+    return poll_status(h);
+}
+
+int alexnet_set_params(alexnet_t* h, int replica, int which, const float* host_in, size_t n) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas || which < 0 || which > 1 || !host_in || n != (size_t)kCanonCount)
+        return fail(h, ALEXNET_ERR_ARG, "set_params: bad argument");
+    Replica& R = h->rep[replica];
+    float* dst = which == 0 ? R.w : R.v;
+    CK(cudaMemcpyAsync(h->canon_tmp, host_in, n * sizeof(float), cudaMemcpyHostToDevice, h->cs));
+    CK(cudaMemsetAsync(dst, 0, h->L.n_total * sizeof(float), h->cs));
+    kn::params_scatter_kernel<<<1184, 256, 0, h->cs>>>(dst, h->canon_tmp, h->L.segs, kCanonCount);
+    h->launches++;
+    if (which == 0) refresh_shadows(h, replica, true, h->cs);
+    CK(cudaStreamSynchronize(h->cs));
+    return ALEXNET_OK;
+}
+
+size_t alexnet_tensor_size(const alexnet_t* h, int tensor_id) {
+    if (!h) return 0;
+    Tensor T;
+    if (!tensor_desc((alexnet*)h, 0, tensor_id, &T)) return 0;
+    return tensor_elems(T, h->B);
+}
+
+int alexnet_get_tensor(alexnet_t* h, int replica, int tensor_id, float* out, size_t n) {
+    if (!h) return ALEXNET_ERR_ARG;
+    Tensor T;
+    if (replica < 0 || replica >= h->cfg.replicas || !out || !tensor_desc(h, replica, tensor_id, &T) || n != tensor_elems(T, h->B))
+        return fail(h, ALEXNET_ERR_ARG, "get_tensor: bad argument");
+    const int B = h->B;
+    std::vector<uint8_t> raw(tensor_dev_bytes(T, B));
+    CK(cudaStreamSynchronize(h->cs));
+    CK(cudaStreamSynchronize(h->ls));
+    CK(cudaMemcpy(raw.data(), T.ptr, raw.size(), cudaMemcpyDeviceToHost));
+    const uint16_t* hb = (const uint16_t*)raw.data();
+    switch (T.kind) {
+        case 0:
+            for (int b = 0; b < B; ++b) for (int c = 0; c < T.C; ++c) for (int y = 0; y < T.H; ++y) for (int x = 0; x < T.W; ++x)
+                out[(((size_t)b * T.C + c) * T.H + y) * T.W + x] = bf2f(hb[(((size_t)b * T.Hp + y) * T.Wp + x) * T.C + c]);
+            break;
+        case 1:
+            for (int b = 0; b < B; ++b) for (int c = 0; c < T.C; ++c) for (int y = 0; y < T.H; ++y) for (int x = 0; x < T.W; ++x)
+                out[(((size_t)b * T.C + c) * T.H + y) * T.W + x] = (float)raw[(((size_t)b * T.H + y) * T.W + x) * T.C + c];
+            break;
+        case 2: for (size_t i = 0; i < n; ++i) out[i] = bf2f(hb[i]); break;
+        case 3: case 7: memcpy(out, raw.data(), n * 4); break;
+        case 4: for (size_t i = 0; i < n; ++i) out[i] = (float)raw[i]; break;
+        case 5:
+            for (int b = 0; b < B; ++b) for (int c = 0; c < 3; ++c) for (int y = 0; y < 227; ++y) for (int x = 0; x < 227; ++x)
+                out[(((size_t)b * 3 + c) * 227 + y) * 227 + x] =
+                    bf2f(hb[(((size_t)b * 57 + y / 4) * 57 + x / 4) * 48 + ((y % 4) * 4 + x % 4) * 3 + c]);
+            break;
+        case 6: for (size_t i = 0; i < n; ++i) out[i] = (float)((const int32_t*)raw.data())[i]; break;
+    }
+    return ALEXNET_OK;
+}
+
+int alexnet_set_tensor(alexnet_t* h, int replica, int tensor_id, const float* in, size_t n) {
+    if (!h) return ALEXNET_ERR_ARG;
+    Tensor T;
+    if (replica < 0 || replica >= h->cfg.replicas || !in || !tensor_desc(h, replica, tensor_id, &T) || n != tensor_elems(T, h->B))
+        return fail(h, ALEXNET_ERR_ARG, "set_tensor: bad argument");
+    const int B = h->B;
+    std::vector<uint8_t> raw(tensor_dev_bytes(T, B), 0);
+    uint16_t* hb = (uint16_t*)raw.data();
+    switch (T.kind) {
+        case 0:
+            for (int b = 0; b < B; ++b) for (int c = 0; c < T.C; ++c) for (int y = 0; y < T.H; ++y) for (int x = 0; x < T.W; ++x)
+                hb[(((size_t)b * T.Hp + y) * T.Wp + x) * T.C + c] = f2bf(in[(((size_t)b * T.C + c) * T.H + y) * T.W + x]);
+            break;
+        case 1:
+            for (int b = 0; b < B; ++b) for (int c = 0; c < T.C; ++c) for (int y = 0; y < T.H; ++y) for (int x = 0; x < T.W; ++x)
+                raw[(((size_t)b * T.H + y) * T.W + x) * T.C + c] = (uint8_t)in[(((size_t)b * T.C + c) * T.H + y) * T.W + x];
+            break;
+        case 2: for (size_t i = 0; i < n; ++i) hb[i] = f2bf(in[i]); break;
+        case 3: case 7: memcpy(raw.data(), in, n * 4); break;
+        case 4: for (size_t i = 0; i < n; ++i) raw[i] = (uint8_t)in[i]; break;
+        case 5:
+            for (int b = 0; b < B; ++b) for (int c = 0; c < 3; ++c) for (int y = 0; y < 227; ++y) for (int x = 0; x < 227; ++x)
+                hb[(((size_t)b * 57 + y / 4) * 57 + x / 4) * 48 + ((y % 4) * 4 + x % 4) * 3 + c] =
+                    f2bf(in[(((size_t)b * 3 + c) * 227 + y) * 227 + x]);
+            break;
+        case 6: for (size_t i = 0; i < n; ++i) ((int32_t*)raw.data())[i] = (int32_t)in[i]; break;
+    }
+    CK(cudaStreamSynchronize(h->cs));
+    CK(cudaStreamSynchronize(h->ls));
+    CK(cudaMemcpy(T.ptr, raw.data(), raw.size(), cudaMemcpyHostToDevice));
+    return ALEXNET_OK;
+}
+
+int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas || op < 0 || op >= ALEXNET_OP_COUNT || iters < 1)
+        return fail(h, ALEXNET_ERR_ARG, "run_op: bad argument");
+    if (op == ALEXNET_OP_AVERAGE && h->cfg.replicas < 2) return fail(h, ALEXNET_ERR_ARG, "run_op: average needs two replicas");
+    if (int rc = check_status(h)) return rc;
+    Replica& R = h->rep[replica];
+    const int slot = R.last_slot;
+    cudaStream_t st = h->cs;
+    for (int it = 0; it < iters; ++it) {
+        if (op <= ALEXNET_OP_CONV5_FWD) op_conv_fwd(h, replica, op - ALEXNET_OP_CONV1_FWD, slot, st);
+        else if (op <= ALEXNET_OP_CONV5_BWD_DATA) op_conv_bwd(h, replica, op - ALEXNET_OP_CONV2_BWD_DATA + 1, st);
+        else if (op <= ALEXNET_OP_CONV5_BWD_WEIGHT) op_conv_wg(h, replica, op - ALEXNET_OP_CONV1_BWD_WEIGHT, slot, st);
+        else if (op <= ALEXNET_OP_FC8_FWD) op_fc_fwd(h, replica, op - ALEXNET_OP_FC6_FWD, R.slot_step[slot], st);
+        else if (op <= ALEXNET_OP_FC8_BWD_DATA) op_fc_bwd(h, replica, op - ALEXNET_OP_FC6_BWD_DATA, st);
+        else if (op <= ALEXNET_OP_FC8_BWD_WEIGHT) op_fc_wg(h, replica, op - ALEXNET_OP_FC6_BWD_WEIGHT, st);
+        else if (op <= ALEXNET_OP_LRN2_FWD) op_lrn_fwd(h, replica, op - ALEXNET_OP_LRN1_FWD, st);
+        else if (op <= ALEXNET_OP_LRN2_BWD) op_lrn_bwd(h, replica, op - ALEXNET_OP_LRN1_BWD, st);
+        else if (op <= ALEXNET_OP_POOL5_FWD) op_pool_fwd(h, replica, op - ALEXNET_OP_POOL1_FWD, st);
+        else if (op <= ALEXNET_OP_POOL5_BWD) op_pool_bwd(h, replica, op - ALEXNET_OP_POOL1_BWD, st);
+        else if (op == ALEXNET_OP_SOFTMAX) op_softmax(h, replica, slot, st);
+        else if (op == ALEXNET_OP_UPDATE) op_update(h, replica, st);
+        else if (op == ALEXNET_OP_AVERAGE) op_average(h, st);
+        else if (op == ALEXNET_OP_PREPROCESS) op_preprocess(h, replica, slot, R.slot_step[slot], st);
+    }
+    CK(cudaGetLastError());
+    return ALEXNET_OK;
+}
+
+uint64_t alexnet_launch_count(const alexnet_t* h) { return h ? h->launches : 0; }
+
+int alexnet_sync(alexnet_t* h) {
+    if (!h) return ALEXNET_ERR_ARG;
+    CK(cudaStreamSynchronize(h->ls));
+    CK(cudaStreamSynchronize(h->cs));
+    if (int rc = check_status(h)) return rc;
+    return poll_status(h);
+}
+
+const char* alexnet_last_error(const alexnet_t* h) { return h ? h->err.c_str() : "null handle"; }
+
+}  // extern "C"

@@ -1,0 +1,464 @@
+// HBM-bound kernels of the AlexNet training step: preprocessing gather, LRN,
+// max-pool, split-K reductions with fused bias/ReLU/dropout, softmax
+// cross-entropy, bias gradients, momentum update, replica average, layout
+// permutations.  Activations are bf16 in a zero-padded flat NHWC grid
+// [B][Hp][Wp][C] whose valid region is the top-left H x W of every image; pad
+// positions always hold zero.  All accesses are 16-byte vectors along C.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace kn {
+
+// ---------------------------------------------------------------- counter hash
+// SplitMix64 finaliser over key + golden*(idx+1); key = finalise(seed ^ stream<<56 ^ replica<<48 ^ step).
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t z) {
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+    return z ^ (z >> 31);
+}
+__host__ __device__ __forceinline__ uint64_t stream_key(uint64_t seed, uint64_t stream, uint64_t replica, uint64_t step) {
+    return mix64(seed ^ (stream << 56) ^ (replica << 48) ^ step);
+}
+__host__ __device__ __forceinline__ uint64_t draw(uint64_t key, uint64_t idx) {
+    return mix64(key + 0x9E3779B97F4A7C15ULL * (idx + 1));
+}
+
+__device__ __forceinline__ void unpack8(const uint4& u, float* f) {
+    const __nv_bfloat162* h = (const __nv_bfloat162*)&u;
+    #pragma unroll
+    for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+    uint4 u;
+    __nv_bfloat162* h = (__nv_bfloat162*)&u;
+    #pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    return u;
+}
+
+// ------------------------------------------------------------- preprocessing
+// Per image: crop offset (ox, oy) in [0,29]^2 and flip bit from the hash
+// (stream 1, idx = image).  out = u8[sy][sx][c] - mean[sy][sx][c] with
+// sy = oy + Y, sx = ox + (flip ? 226 - X : X), written as bf16 in the 4x4
+// space-to-depth layout [B][57][57][48], channel = ((Y%4)*4 + X%4)*3 + c,
+// with row/column 227 of the 228-padded image set to zero.
+__global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* __restrict__ mean,
+                                  __nv_bfloat16* __restrict__ out, int32_t* __restrict__ cf_out,
+                                  int B, uint64_t key) {
+    // one thread per (n, by, bx, dy): 12 output values (4 dx * 3 colours) = 24 bytes
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long total = (long long)B * 57 * 57 * 4;
+    if (t >= total) return;
+    const int dy = (int)(t & 3);
+    long long cell = t >> 2;
+    const int bx = (int)(cell % 57); cell /= 57;
+    const int by = (int)(cell % 57);
+    const int n = (int)(cell / 57);
+    const uint64_t r = draw(key, (uint64_t)n);
+    const int ox = (int)((r & 0xFFFF) % 30), oy = (int)(((r >> 16) & 0xFFFF) % 30), flip = (int)((r >> 32) & 1);
+    if (cf_out && by == 0 && bx == 0 && dy == 0) { cf_out[3 * n] = ox; cf_out[3 * n + 1] = oy; cf_out[3 * n + 2] = flip; }
+    const int Y = by * 4 + dy;
+    float v[12];
+    #pragma unroll
+    for (int dx = 0; dx < 4; ++dx) {
+        const int X = bx * 4 + dx;
+        if (Y < 227 && X < 227) {
+            const int sy = oy + Y, sx = ox + (flip ? 226 - X : X);
+            const size_t s = ((size_t)sy * 256 + sx) * 3;
+            const uint8_t* ip = img + (size_t)n * 196608 + s;
+            #pragma unroll
+            for (int c = 0; c < 3; ++c) v[dx * 3 + c] = (float)ip[c] - mean[s + c];
+        } else {
+            v[dx * 3] = v[dx * 3 + 1] = v[dx * 3 + 2] = 0.f;
+        }
+    }
+    __nv_bfloat162* o = (__nv_bfloat162*)(out + ((size_t)(n * 57 + by) * 57 + bx) * 48 + dy * 12);
+    #pragma unroll
+    for (int i = 0; i < 6; ++i) o[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+}
+
+// ----------------------------------------------------------------------- LRN
+__device__ __forceinline__ float pow_neg(float s, float beta) {
+    if (beta == 0.75f) { float r = rsqrtf(s); return r * sqrtf(r); }
+    return exp2f(-beta * log2f(s));
+}
+// b_c = a_c * (k + alpha * sum_{c' in [c-2,c+2] clipped} a_c'^2)^(-beta); one thread = 8 channels of one pixel.
+__global__ void lrn_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ b,
+                               long long rows, int C, float alpha, float beta, float k) {
+    const int cpr = C >> 3;
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows * cpr) return;
+    const int ch = (int)(t % cpr);
+    const uint4* ap = (const uint4*)a + t;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    float f[24];
+    unpack8(ch > 0 ? ap[-1] : zero, f);
+    unpack8(ap[0], f + 8);
+    unpack8(ch < cpr - 1 ? ap[1] : zero, f + 16);
+    float o[8];
+    #pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float ss = 0.f;
+        #pragma unroll
+        for (int j = -2; j <= 2; ++j) ss += f[8 + i + j] * f[8 + i + j];
+        o[i] = f[8 + i] * pow_neg(k + alpha * ss, beta);
+    }
+    ((uint4*)b)[t] = pack8(o);
+}
+// da_m = [a_m > 0] * ( g_m s_m^-beta - 2 alpha beta a_m sum_{c in [m-2,m+2]} g_c a_c s_c^(-beta-1) )
+// (the ReLU mask of the convolution that produced a is applied here).
+__global__ void lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ g,
+                               __nv_bfloat16* __restrict__ da, long long rows, int C, float alpha, float beta, float k) {
+    const int cpr = C >> 3;
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows * cpr) return;
+    const int ch = (int)(t % cpr);
+    const uint4* ap = (const uint4*)a + t;
+    const uint4* gp = (const uint4*)g + t;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    float fa[24], fg[24];
+    unpack8(ch > 0 ? ap[-1] : zero, fa);
+    unpack8(ap[0], fa + 8);
+    unpack8(ch < cpr - 1 ? ap[1] : zero, fa + 16);
+    unpack8(ch > 0 ? gp[-1] : zero, fg);
+    unpack8(gp[0], fg + 8);
+    unpack8(ch < cpr - 1 ? gp[1] : zero, fg + 16);
+    float sp[12], tt[12];   // channels c0-2 .. c0+9
+    #pragma unroll
+    for (int i = 0; i < 12; ++i) {
+        const int c = 6 + i;
+        float ss = 0.f;
+        #pragma unroll
+        for (int j = -2; j <= 2; ++j) ss += fa[c + j] * fa[c + j];
+        const float s = k + alpha * ss;
+        sp[i] = pow_neg(s, beta);
+        tt[i] = fg[c] * fa[c] * sp[i] / s;
+    }
+    float o[8];
+    #pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float acc = tt[i] + tt[i + 1] + tt[i + 2] + tt[i + 3] + tt[i + 4];
+        const float am = fa[8 + i];
+        const float v = fg[8 + i] * sp[i + 2] - 2.f * alpha * beta * am * acc;
+        o[i] = am > 0.f ? v : 0.f;
+    }
+    ((uint4*)da)[t] = pack8(o);
+}
+
+// ------------------------------------------------------------------ max pool
+// 3x3 stride 2, no padding; first maximum in (ky,kx) row-major order wins; argmax = ky*3+kx.
+__global__ void pool_fwd_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
+                                uint8_t* __restrict__ arg, int B, int C, int Hpi, int Wpi,
+                                int Ho, int Wo, int Hpo, int Wpo) {
+    const int cpr = C >> 3;
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (long long)B * Ho * Wo * cpr) return;
+    const int ch = (int)(t % cpr);
+    long long r = t / cpr;
+    const int ox = (int)(r % Wo); r /= Wo;
+    const int oy = (int)(r % Ho);
+    const int n = (int)(r / Ho);
+    float best[8]; int bi[8];
+    #pragma unroll
+    for (int ky = 0; ky < 3; ++ky)
+        #pragma unroll
+        for (int kx = 0; kx < 3; ++kx) {
+            const uint4 u = ((const uint4*)x)[((size_t)(n * Hpi + 2 * oy + ky) * Wpi + 2 * ox + kx) * cpr + ch];
+            float f[8];
+            unpack8(u, f);
+            #pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if ((ky == 0 && kx == 0) || f[i] > best[i]) { best[i] = f[i]; bi[i] = ky * 3 + kx; }
+        }
+    ((uint4*)y)[((size_t)(n * Hpo + oy) * Wpo + ox) * cpr + ch] = pack8(best);
+    uint2 ab;
+    ab.x = bi[0] | (bi[1] << 8) | (bi[2] << 16) | (bi[3] << 24);
+    ab.y = bi[4] | (bi[5] << 8) | (bi[6] << 16) | (bi[7] << 24);
+    ((uint2*)arg)[t] = ab;
+}
+// dx[y][x] = sum over the (up to 4) windows containing (y,x) whose argmax points at it; optional ReLU mask.
+__global__ void pool_bwd_kernel(const __nv_bfloat16* __restrict__ dy, const uint8_t* __restrict__ arg,
+                                const __nv_bfloat16* __restrict__ relu_src, __nv_bfloat16* __restrict__ dx,
+                                int B, int C, int Hpi, int Wpi, int Hi, int Wi, int Ho, int Wo, int Hpo, int Wpo) {
+    const int cpr = C >> 3;
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (long long)B * Hpi * Wpi * cpr) return;
+    const int ch = (int)(t % cpr);
+    long long r = t / cpr;
+    const int x = (int)(r % Wpi); r /= Wpi;
+    const int y = (int)(r % Hpi);
+    const int n = (int)(r / Hpi);
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (y < Hi && x < Wi) {
+        const int oy_lo = max(0, (y - 1) >> 1), oy_hi = min(Ho - 1, y >> 1);
+        const int ox_lo = max(0, (x - 1) >> 1), ox_hi = min(Wo - 1, x >> 1);
+        for (int oy = oy_lo; oy <= oy_hi; ++oy)
+            for (int ox = ox_lo; ox <= ox_hi; ++ox) {
+                const int code = (y - 2 * oy) * 3 + (x - 2 * ox);
+                const uint2 ab = ((const uint2*)arg)[((size_t)(n * Ho + oy) * Wo + ox) * cpr + ch];
+                float f[8];
+                unpack8(((const uint4*)dy)[((size_t)(n * Hpo + oy) * Wpo + ox) * cpr + ch], f);
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int a = (int)(((i < 4 ? ab.x : ab.y) >> (8 * (i & 3))) & 0xFF);
+                    if (a == code) acc[i] += f[i];
+                }
+            }
+        if (relu_src) {
+            float m[8];
+            unpack8(((const uint4*)relu_src)[t], m);
+            #pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = m[i] > 0.f ? acc[i] : 0.f;
+        }
+    }
+    ((uint4*)dx)[t] = pack8(acc);
+}
+
+// ------------------------------------------------- split-K reductions (FC, wgrad)
+// y[b][n] = act( sum_z ws[z][b][n] + bias[n] ) * keep(b*N + n) * scale -> bf16, or fp32 logits when out_f32.
+__global__ void fc_reduce_fwd_kernel(const float* __restrict__ ws, int splits, long long split_stride,
+                                     const float* __restrict__ bias, int B, int N, int relu,
+                                     int use_dropout, uint64_t key, uint32_t thr24, float scale,
+                                     __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32,
+                                     uint8_t* __restrict__ keep_out) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (long long)B * N) return;
+    const int n = (int)(t % N);
+    float v = 0.f;
+    for (int z = 0; z < splits; ++z) v += ws[z * split_stride + t];
+    v += bias[n];
+    if (relu) v = fmaxf(v, 0.f);
+    if (use_dropout) {
+        const bool keep = (uint32_t)(draw(key, (uint64_t)t) >> 40) >= thr24;
+        if (keep_out) keep_out[t] = keep ? 1 : 0;
+        v = keep ? v * scale : 0.f;
+    } else if (keep_out) {
+        keep_out[t] = 1;
+    }
+    if (out_f32) out_f32[t] = v; else out_bf16[t] = __float2bfloat16_rn(v);
+}
+// dx[b][k] = [mask[b][k] > 0] * scale * sum_z ws[z][b][k] -> bf16 (mask = the layer input, post ReLU and dropout)
+__global__ void fc_reduce_bwd_kernel(const float* __restrict__ ws, int splits, long long split_stride,
+                                     const __nv_bfloat16* __restrict__ mask, float scale, long long total,
+                                     __nv_bfloat16* __restrict__ out) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= total) return;
+    float v = 0.f;
+    for (int z = 0; z < splits; ++z) v += ws[z * split_stride + t];
+    if (mask) v = __bfloat162float(mask[t]) > 0.f ? v * scale : 0.f;
+    out[t] = __float2bfloat16_rn(v);
+}
+// g[i] = sum_z ws[z][i]; conv1: entries of the 12x12 zero-padded filter outside 11x11 stay zero.
+__global__ void wgrad_reduce_kernel(const float* __restrict__ ws, int splits, long long split_stride,
+                                    long long total, float* __restrict__ g, int conv1_pad_mask) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= total) return;
+    float v = 0.f;
+    for (int z = 0; z < splits; ++z) v += ws[z * split_stride + t];
+    if (conv1_pad_mask) {
+        const int ch = (int)(t % 48), tap = (int)(t / (48 * 96));
+        const int ky = (tap / 3) * 4 + (ch / 3) / 4, kx = (tap % 3) * 4 + (ch / 3) % 4;
+        if (ky > 10 || kx > 10) v = 0.f;
+    }
+    g[t] = v;
+}
+
+// db[c] = sum over rows of dy[row][c] (bf16 in, fp32 out), two stages: grid (ceil(C/64), row_splits)
+// writes partial[split][C]; colsum_final_kernel adds the splits in a fixed order.
+__global__ void colsum_kernel(const __nv_bfloat16* __restrict__ dy, long long rows, int C, float* __restrict__ partial) {
+    // block: 256 threads = 32 row-lanes x 8 column-chunks (8 channels each) -> 64 columns per block
+    __shared__ float red[32][65];
+    const int cc = threadIdx.x & 7, rl = threadIdx.x >> 3;
+    const int c0 = blockIdx.x * 64 + cc * 8;
+    const long long per = (rows + gridDim.y - 1) / gridDim.y;
+    const long long r0 = (long long)blockIdx.y * per, r1 = min(rows, r0 + per);
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (c0 < C) {
+        for (long long r = r0 + rl; r < r1; r += 32) {
+            float f[8];
+            unpack8(*(const uint4*)(dy + r * C + c0), f);
+            #pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] += f[i];
+        }
+    }
+    #pragma unroll
+    for (int i = 0; i < 8; ++i) red[rl][cc * 8 + i] = acc[i];
+    __syncthreads();
+    if (threadIdx.x < 64) {
+        float s = 0.f;
+        for (int r = 0; r < 32; ++r) s += red[r][threadIdx.x];
+        const int c = blockIdx.x * 64 + threadIdx.x;
+        if (c < C) partial[(size_t)blockIdx.y * C + c] = s;
+    }
+}
+__global__ void colsum_final_kernel(const float* __restrict__ partial, int splits, int C, float* __restrict__ db) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    float s = 0.f;
+    for (int z = 0; z < splits; ++z) s += partial[(size_t)z * C + c];
+    db[c] = s;
+}
+// same for a row pitch that is not a multiple of 8 elements (the 1000-wide logits gradient)
+__global__ void colsum_scalar_kernel(const __nv_bfloat16* __restrict__ dy, int rows, int C, float* __restrict__ db) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    float s = 0.f;
+    for (int r = 0; r < rows; ++r) s += __bfloat162float(dy[(size_t)r * C + c]);
+    db[c] = s;
+}
+
+// ------------------------------------------------------ softmax cross-entropy
+// one block per sample: p = softmax(z), loss_n = -log p[label], dz = (p - onehot)/B as bf16
+__global__ void softmax_xent_kernel(const float* __restrict__ z, const int32_t* __restrict__ labels,
+                                    __nv_bfloat16* __restrict__ dz, float* __restrict__ loss_n, int B, int N) {
+    __shared__ float red[32];
+    const int n = blockIdx.x, tid = threadIdx.x;
+    const float* zr = z + (size_t)n * N;
+    float mx = -INFINITY;
+    for (int j = tid; j < N; j += blockDim.x) mx = fmaxf(mx, zr[j]);
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(~0u, mx, o));
+    if ((tid & 31) == 0) red[tid >> 5] = mx;
+    __syncthreads();
+    mx = red[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) mx = fmaxf(mx, red[w]);
+    __syncthreads();
+    float sum = 0.f;
+    for (int j = tid; j < N; j += blockDim.x) sum += expf(zr[j] - mx);
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(~0u, sum, o);
+    if ((tid & 31) == 0) red[tid >> 5] = sum;
+    __syncthreads();
+    sum = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); ++w) sum += red[w];
+    const int lab = labels[n];
+    const float inv = 1.f / sum, invB = 1.f / (float)B;
+    for (int j = tid; j < N; j += blockDim.x) {
+        const float pj = expf(zr[j] - mx) * inv;
+        dz[(size_t)n * N + j] = __float2bfloat16_rn((pj - (j == lab ? 1.f : 0.f)) * invB);
+    }
+    if (tid == 0) loss_n[n] = -(zr[lab] - mx - logf(sum));
+}
+__global__ void mean_kernel(const float* __restrict__ v, int n, float* __restrict__ out) {
+    __shared__ float red[32];
+    float s = 0.f;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) s += v[i];
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(~0u, s, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
+        *out = t / (float)n;
+    }
+}
+
+// ------------------------------------------------ momentum update and average
+// v <- mu v - lr wd w [i < n_decay] - lr g ; w <- w + v ; bf16 shadow of w.  22 bytes per parameter.
+__global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g,
+                                  __nv_bfloat16* __restrict__ shadow, long long n4, long long n_decay4,
+                                  float lr, float mu, float wd) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 wv = ((float4*)w)[i], vv = ((float4*)v)[i];
+        const float4 gv = ((const float4*)g)[i];
+        const float d = i < n_decay4 ? lr * wd : 0.f;
+        vv.x = mu * vv.x - d * wv.x - lr * gv.x; wv.x += vv.x;
+        vv.y = mu * vv.y - d * wv.y - lr * gv.y; wv.y += vv.y;
+        vv.z = mu * vv.z - d * wv.z - lr * gv.z; wv.z += vv.z;
+        vv.w = mu * vv.w - d * wv.w - lr * gv.w; wv.w += vv.w;
+        ((float4*)w)[i] = wv;
+        ((float4*)v)[i] = vv;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(wv.x, wv.y), hi = __floats2bfloat162_rn(wv.z, wv.w);
+        ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
+    }
+}
+// exchange-and-average with both replicas in one HBM: w_a = w_b = (w_a+w_b)/2, same for momentum; refresh both shadows.
+__global__ void replica_average_kernel(float* __restrict__ wa, float* __restrict__ wb, float* __restrict__ va,
+                                       float* __restrict__ vb, __nv_bfloat16* __restrict__ sa,
+                                       __nv_bfloat16* __restrict__ sb, long long n4) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        const float4 a = ((float4*)wa)[i], b = ((float4*)wb)[i];
+        const float4 c = ((float4*)va)[i], d = ((float4*)vb)[i];
+        const float4 w = make_float4(0.5f * (a.x + b.x), 0.5f * (a.y + b.y), 0.5f * (a.z + b.z), 0.5f * (a.w + b.w));
+        const float4 v = make_float4(0.5f * (c.x + d.x), 0.5f * (c.y + d.y), 0.5f * (c.z + d.z), 0.5f * (c.w + d.w));
+        ((float4*)wa)[i] = w; ((float4*)wb)[i] = w;
+        ((float4*)va)[i] = v; ((float4*)vb)[i] = v;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+        const uint2 s = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
+        ((uint2*)sa)[i] = s; ((uint2*)sb)[i] = s;
+    }
+}
+__global__ void shadow_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ shadow, long long n4) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        const float4 wv = ((const float4*)w)[i];
+        __nv_bfloat162 lo = __floats2bfloat162_rn(wv.x, wv.y), hi = __floats2bfloat162_rn(wv.z, wv.w);
+        ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
+    }
+}
+
+// transposed bf16 copies of the grouped conv filters for the backward-data pass:
+// wt[tap][g*cig + ci][co'] = wf[tap][g*cog + co'][ci]
+struct TransposeJob { long long src_off, dst_off; int taps, cout, cig, groups; long long count; };
+struct TransposeJobs { TransposeJob j[4]; int n; };
+__global__ void conv_transpose_shadow_kernel(const __nv_bfloat16* __restrict__ shadow, __nv_bfloat16* __restrict__ wt,
+                                             const TransposeJobs jobs) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (int q = 0; q < jobs.n; ++q) {
+        const TransposeJob J = jobs.j[q];
+        const int cog = J.cout / J.groups;
+        for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < J.count; i += stride) {
+            // i indexes dst [tap][cin][cog]
+            const int co_ = (int)(i % cog);
+            long long r = i / cog;
+            const int cin = (int)(r % (J.cig * J.groups));
+            const int tap = (int)(r / (J.cig * J.groups));
+            const int grp = cin / J.cig, ci = cin % J.cig;
+            wt[J.dst_off + i] = shadow[J.src_off + ((long long)tap * J.cout + grp * cog + co_) * J.cig + ci];
+        }
+    }
+}
+
+// ------------------------------------------- canonical <-> internal parameter order
+struct ParamSeg { long long canon_off, int_off, count; int kind, a, b, c; };  // kind 0 copy, 1 conv [co][ci][k][k], 2 conv1 s2d, 3 fc6
+struct ParamSegs { ParamSeg s[16]; };
+__device__ __forceinline__ long long canon_to_internal(const ParamSeg& S, long long i) {
+    if (S.kind == 0) return S.int_off + i;
+    if (S.kind == 1) {          // a = cout, b = cig, c = k : canonical ((co*cig+ci)*k+ky)*k+kx -> (tap*cout+co)*cig+ci
+        const int kk2 = S.c * S.c;
+        const int tap = (int)(i % kk2);
+        long long r = i / kk2;
+        const int ci = (int)(r % S.b), co = (int)(r / S.b);
+        return S.int_off + ((long long)tap * S.a + co) * S.b + ci;
+    }
+    if (S.kind == 2) {          // conv1: [96][3][11][11] -> [tap 3x3][96][48], channel ((ky%4)*4 + kx%4)*3 + c
+        const int kx = (int)(i % 11), ky = (int)((i / 11) % 11), c = (int)((i / 121) % 3), co = (int)(i / 363);
+        const int tap = (ky >> 2) * 3 + (kx >> 2), ch = ((ky & 3) * 4 + (kx & 3)) * 3 + c;
+        return S.int_off + ((long long)tap * 96 + co) * 48 + ch;
+    }
+    // fc6: [4096][c*36 + hw] -> [4096][hw*256 + c]
+    const int k = (int)(i % 9216), n = (int)(i / 9216);
+    return S.int_off + (long long)n * 9216 + (k % 36) * 256 + k / 36;
+}
+__global__ void params_gather_kernel(const float* __restrict__ arena, float* __restrict__ canon, const ParamSegs segs,
+                                     long long total) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        int s = 0;
+        while (s < 15 && i >= segs.s[s + 1].canon_off) ++s;
+        canon[i] = arena[canon_to_internal(segs.s[s], i - segs.s[s].canon_off)];
+    }
+}
+__global__ void params_scatter_kernel(float* __restrict__ arena, const float* __restrict__ canon, const ParamSegs segs,
+                                      long long total) {
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        int s = 0;
+        while (s < 15 && i >= segs.s[s + 1].canon_off) ++s;
+        arena[canon_to_internal(segs.s[s], i - segs.s[s].canon_off)] = canon[i];
+    }
+}
+
+}  // namespace kn
