@@ -159,6 +159,13 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters);
 /* Number of kernels launched by this handle since creation (for accounting). */
 uint64_t alexnet_launch_count(const alexnet_t* h);
 
+/* Optional timing of the tensor-core GEMM kernel: while enabled, every launch
+ * of it is bracketed by a CUDA event pair on its stream.  profile_read waits for
+ * both streams, returns the summed device time (ms) and the number of launches
+ * recorded since the last read, and clears the record. */
+int alexnet_profile(alexnet_t* h, int enable);
+int alexnet_profile_read(alexnet_t* h, double* gemm_ms, uint64_t* gemm_launches);
+
 /* Wait for both streams; returns a latched DEVICE_TIMEOUT or CUDA error if any. */
 int alexnet_sync(alexnet_t* h);
 const char* alexnet_last_error(const alexnet_t* h);

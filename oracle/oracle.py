@@ -327,23 +327,42 @@ class OracleNet:
         a = c.lrn_alpha / c.lrn_size if c.lrn_alpha_div_n else c.lrn_alpha
         return dict(size=c.lrn_size, alpha=a, beta=c.lrn_beta, k=c.lrn_k)
 
-    def forward_backward(self, img_u8, labels, mean, step):
+    def forward_backward(self, img_u8, labels, mean, step, cf=None, m6=None, m7=None, mean_over=None,
+                         gates=None, args=None):
         """One forward + backward pass.  Returns a dict with every intermediate
-        (canonical NCHW fp64), the flat canonical gradient 'g' and 'loss'."""
+        (canonical NCHW fp64), the flat canonical gradient 'g' and 'loss'.
+        cf / m6 / m7 override the hashed crop-flip triples and dropout masks and
+        mean_over the batch size of the loss mean, so that a few images of a
+        larger batch can be evaluated on their own.
+
+        gates / args: the discrete decisions of the backward pass (which units
+        pass gradient through ReLU and dropout; which window element receives a
+        pool gradient) are by default the oracle's own, taken in fp64.  A caller
+        comparing against an implementation that stores bf16 activations passes
+        that implementation's decisions here (dicts keyed a1..a5, f6, f7 and
+        arg1, arg2, arg5) after checking them valid, so that both sides take
+        each decision in the same precision; the forward pass is unaffected."""
         c = self.cfg
         q = self._q
         P = unpack(self.w)
         Pq = {k: q(a) if k.endswith(".W") else a for k, a in P.items()}
         B = img_u8.shape[0]
         T = {}
-        T["cf"] = crop_flip(c.seed, self.replica, step, B)
+        T["cf"] = crop_flip(c.seed, self.replica, step, B) if cf is None else np.asarray(cf, np.int32)
         T["x0"] = q(preprocess(img_u8, mean, T["cf"]))
         la = self._lrn_args()
 
         def conv_block(name, x):
             cc = CONV[name]
             z = conv_fwd(x, Pq[name + ".W"], P[name + ".b"], cc["s"], cc["p"], cc["g"])
+            T["pre_a" + name[-1]] = z
             return q(np.maximum(z, 0.0))
+
+        def gate(k):
+            return np.asarray(gates[k], bool) if gates is not None else (T[k] > 0)
+
+        def arg(k):
+            return np.asarray(args[k], np.uint8) if args is not None else T[k]
 
         T["a1"] = conv_block("conv1", T["x0"])
         T["n1"] = q(lrn_fwd(T["a1"], **la))
@@ -357,29 +376,35 @@ class OracleNet:
         T["p5"], T["arg5"] = pool_fwd(T["a5"])
         flat = T["p5"].reshape(B, 9216)  # C,H,W order
         scale = 1.0 / (1.0 - c.dropout_p) if (c.inverted_dropout and c.dropout_p > 0) else 1.0
-        if c.dropout_p > 0:
+        if m6 is not None:
+            T["m6"], T["m7"] = np.asarray(m6, np.uint8), np.asarray(m7, np.uint8)
+        elif c.dropout_p > 0:
             T["m6"] = dropout_mask(c.seed, 2, self.replica, step, B, 4096, c.dropout_p)
             T["m7"] = dropout_mask(c.seed, 3, self.replica, step, B, 4096, c.dropout_p)
         else:
             T["m6"] = np.ones((B, 4096), np.uint8)
             T["m7"] = np.ones((B, 4096), np.uint8)
-        T["f6"] = q(np.maximum(fc_fwd(flat, Pq["fc6.W"], P["fc6.b"]), 0.0) * T["m6"] * scale)
-        T["f7"] = q(np.maximum(fc_fwd(T["f6"], Pq["fc7.W"], P["fc7.b"]), 0.0) * T["m7"] * scale)
+        T["pre_f6"] = fc_fwd(flat, Pq["fc6.W"], P["fc6.b"])
+        T["f6"] = q(np.maximum(T["pre_f6"], 0.0) * T["m6"] * scale)
+        T["pre_f7"] = fc_fwd(T["f6"], Pq["fc7.W"], P["fc7.b"])
+        T["f7"] = q(np.maximum(T["pre_f7"], 0.0) * T["m7"] * scale)
         T["z"] = fc_fwd(T["f7"], Pq["fc8.W"], P["fc8.b"])
         T["prob"], T["loss"], dz = softmax_xent(T["z"], labels)
+        if mean_over is not None:
+            dz = dz * (B / float(mean_over))
         T["dz"] = q(dz)
 
         # ---- backward
         G = {}
         d7, G["fc8.W"], G["fc8.b"] = fc_bwd(T["f7"], Pq["fc8.W"], T["dz"])
-        d7 = q(d7 * (T["f7"] > 0) * scale)          # dropout mask and ReLU: f7 > 0 iff kept and positive
+        d7 = q(d7 * gate("f7") * scale)          # dropout mask and ReLU: f7 > 0 iff kept and positive
         T["df7"] = d7
         d6, G["fc7.W"], G["fc7.b"] = fc_bwd(T["f6"], Pq["fc7.W"], d7)
-        d6 = q(d6 * (T["f6"] > 0) * scale)
+        d6 = q(d6 * gate("f6") * scale)
         T["df6"] = d6
         dp5, G["fc6.W"], G["fc6.b"] = fc_bwd(flat, Pq["fc6.W"], d6)
         T["dp5"] = q(dp5).reshape(T["p5"].shape)
-        da5 = pool_bwd(T["dp5"], T["arg5"], T["a5"].shape) * (T["a5"] > 0)
+        da5 = pool_bwd(T["dp5"], arg("arg5"), T["a5"].shape) * gate("a5")
         T["da5"] = q(da5)
 
         def conv_back(name, x, dy, need_dx=True):
@@ -390,14 +415,14 @@ class OracleNet:
                 return None
             return conv_bwd_data(dy, Pq[name + ".W"], x.shape, cc["s"], cc["p"], cc["g"])
 
-        T["da4"] = q(conv_back("conv5", T["a4"], T["da5"]) * (T["a4"] > 0))
-        T["da3"] = q(conv_back("conv4", T["a3"], T["da4"]) * (T["a3"] > 0))
+        T["da4"] = q(conv_back("conv5", T["a4"], T["da5"]) * gate("a4"))
+        T["da3"] = q(conv_back("conv4", T["a3"], T["da4"]) * gate("a3"))
         T["dp2"] = q(conv_back("conv3", T["p2"], T["da3"]))
-        T["dn2"] = pool_bwd(T["dp2"], T["arg2"], T["n2"].shape)
-        T["da2"] = q(lrn_bwd(T["a2"], T["dn2"], **la) * (T["a2"] > 0))
+        T["dn2"] = pool_bwd(T["dp2"], arg("arg2"), T["n2"].shape)
+        T["da2"] = q(lrn_bwd(T["a2"], T["dn2"], **la) * gate("a2"))
         T["dp1"] = q(conv_back("conv2", T["p1"], T["da2"]))
-        T["dn1"] = pool_bwd(T["dp1"], T["arg1"], T["n1"].shape)
-        T["da1"] = q(lrn_bwd(T["a1"], T["dn1"], **la) * (T["a1"] > 0))
+        T["dn1"] = pool_bwd(T["dp1"], arg("arg1"), T["n1"].shape)
+        T["da1"] = q(lrn_bwd(T["a1"], T["dn1"], **la) * gate("a1"))
         conv_back("conv1", T["x0"], T["da1"], need_dx=False)
 
         off, tot = param_offsets()
@@ -407,9 +432,9 @@ class OracleNet:
         T["g"] = g
         return T
 
-    def train_step(self, img_u8, labels, mean, step):
+    def train_step(self, img_u8, labels, mean, step, **kw):
         c = self.cfg
-        T = self.forward_backward(img_u8, labels, mean, step)
+        T = self.forward_backward(img_u8, labels, mean, step, **kw)
         self.w, self.v = sgd_momentum(self.w, self.v, T["g"], c.lr, c.momentum, c.weight_decay,
                                       decay_mask(c.wd_on_biases))
         return T
@@ -421,19 +446,21 @@ def average_replicas(a: OracleNet, b: OracleNet):
     a.v, b.v = replica_average(a.v, b.v)
 
 
-def conv1_block(img_u8, mean, cf, w1, b1, upstream, cfg: OracleConfig = None):
+def conv1_block(img_u8, mean, cf, w1, b1, upstream, cfg: OracleConfig = None, gates=None, args=None):
     """The conv1 block alone: preprocess -> conv1 -> ReLU -> LRN -> pool, with
-    loss = sum(pooled * upstream); returns intermediates and dW1, db1."""
+    loss = sum(pooled * upstream); returns intermediates and dW1, db1.
+    gates / args as in OracleNet.forward_backward."""
     cfg = cfg or OracleConfig()
     la = dict(size=cfg.lrn_size, alpha=cfg.lrn_alpha, beta=cfg.lrn_beta, k=cfg.lrn_k)
     T = {}
     T["x0"] = preprocess(img_u8, mean, cf)
     cc = CONV["conv1"]
-    T["a1"] = np.maximum(conv_fwd(T["x0"], w1, b1, cc["s"], cc["p"], cc["g"]), 0.0)
+    T["pre_a1"] = conv_fwd(T["x0"], w1, b1, cc["s"], cc["p"], cc["g"])
+    T["a1"] = np.maximum(T["pre_a1"], 0.0)
     T["n1"] = lrn_fwd(T["a1"], **la)
     T["p1"], T["arg1"] = pool_fwd(T["n1"])
     T["loss"] = float((T["p1"] * upstream).sum())
-    T["dn1"] = pool_bwd(_f64(upstream), T["arg1"], T["n1"].shape)
-    T["da1"] = lrn_bwd(T["a1"], T["dn1"], **la) * (T["a1"] > 0)
+    T["dn1"] = pool_bwd(_f64(upstream), T["arg1"] if args is None else np.asarray(args["arg1"], np.uint8), T["n1"].shape)
+    T["da1"] = lrn_bwd(T["a1"], T["dn1"], **la) * ((T["a1"] > 0) if gates is None else np.asarray(gates["a1"], bool))
     T["dW1"], T["db1"] = conv_bwd_weight(T["x0"], T["da1"], w1.shape, cc["s"], cc["p"], cc["g"])
     return T

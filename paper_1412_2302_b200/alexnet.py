@@ -32,7 +32,7 @@ OP = {n: i for i, n in enumerate(OPS)}
 EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "alexnet_destroy",
            "alexnet_load_batch_async", "alexnet_train_step", "alexnet_replica_average", "alexnet_get_params",
            "alexnet_set_params", "alexnet_tensor_size", "alexnet_get_tensor", "alexnet_set_tensor", "alexnet_run_op",
-           "alexnet_launch_count", "alexnet_sync", "alexnet_last_error"]
+           "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error"]
 
 
 class Config(ctypes.Structure):
@@ -79,6 +79,8 @@ def load_library():
     L.alexnet_run_op.argtypes = [vp, i32, i32, i32]
     L.alexnet_launch_count.restype = u64
     L.alexnet_launch_count.argtypes = [vp]
+    L.alexnet_profile.argtypes = [vp, i32]
+    L.alexnet_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(u64)]
     L.alexnet_sync.argtypes = [vp]
     L.alexnet_last_error.restype = ctypes.c_char_p
     L.alexnet_last_error.argtypes = [vp]
@@ -187,6 +189,15 @@ class AlexNet:
 
     def run_op(self, name, replica=0, iters=1):
         self._ck(self.lib.alexnet_run_op(self.h, replica, OP[name], iters))
+
+    def profile(self, enable):
+        self._ck(self.lib.alexnet_profile(self.h, 1 if enable else 0))
+
+    def profile_read(self):
+        """(summed GEMM-kernel device time in ms, launches) since the last read."""
+        ms, n = ctypes.c_double(), ctypes.c_uint64()
+        self._ck(self.lib.alexnet_profile_read(self.h, ctypes.byref(ms), ctypes.byref(n)))
+        return ms.value, int(n.value)
 
     @property
     def launch_count(self):

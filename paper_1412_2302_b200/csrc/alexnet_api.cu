@@ -138,6 +138,10 @@ struct alexnet {
     int latched;
     float alpha_eff, drop_scale; uint32_t thr24;
     PFN_cuTensorMapEncodeTiled_v12000 encode;
+    // optional per-launch timing of the GEMM kernel (event pairs on the launching stream)
+    bool prof;
+    std::vector<cudaEvent_t> prof_ev;
+    size_t prof_used;
 };
 
 namespace {
@@ -406,7 +410,16 @@ int build_plans(alexnet* h, int r) {
 inline int nblk(long long n, int t) { return (int)((n + t - 1) / t); }
 
 void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
+    if (h->prof) {
+        while (h->prof_ev.size() < h->prof_used + 2) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) { h->prof = false; break; }
+            h->prof_ev.push_back(e);
+        }
+    }
+    if (h->prof) cudaEventRecord(h->prof_ev[h->prof_used], st);
     tc::gemm_kernel<<<P.grid, tc::kThreads, P.smem, st>>>(P.p);
+    if (h->prof) { cudaEventRecord(h->prof_ev[h->prof_used + 1], st); h->prof_used += 2; }
     h->launches++;
 }
 void colsum(alexnet* h, const bf16* dy, long long rows, int C, float* db, cudaStream_t st) {
@@ -692,7 +705,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     alexnet* h = new alexnet();
     h->cfg = *cfg; h->B = cfg->batch; h->L = make_layout();
     h->cs = (cudaStream_t)compute_stream; h->ls = (cudaStream_t)copy_stream;
-    h->launches = 0; h->latched = 0;
+    h->launches = 0; h->latched = 0; h->prof = false; h->prof_used = 0;
     h->alpha_eff = (cfg->flags & ALEXNET_FLAG_LRN_ALPHA_DIV_N) ? cfg->lrn_alpha / 5.f : cfg->lrn_alpha;
     h->drop_scale = ((cfg->flags & ALEXNET_FLAG_INVERTED_DROPOUT) && cfg->dropout_p > 0.f) ? 1.f / (1.f - cfg->dropout_p) : 1.f;
     h->thr24 = (uint32_t)floor((double)cfg->dropout_p * 16777216.0);
@@ -736,6 +749,7 @@ int alexnet_destroy(alexnet_t* h) {
     if (!h) return ALEXNET_ERR_ARG;
     cudaStreamSynchronize(h->cs);
     cudaStreamSynchronize(h->ls);
+    for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
     for (int r = 0; r < h->cfg.replicas; ++r)
         for (int s = 0; s < 2; ++s) { cudaEventDestroy(h->rep[r].ready[s]); cudaEventDestroy(h->rep[r].consumed[s]); }
     delete h;
@@ -921,6 +935,28 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
 }
 
 uint64_t alexnet_launch_count(const alexnet_t* h) { return h ? h->launches : 0; }
+
+int alexnet_profile(alexnet_t* h, int enable) {
+    if (!h) return ALEXNET_ERR_ARG;
+    h->prof = enable != 0;
+    return ALEXNET_OK;
+}
+
+int alexnet_profile_read(alexnet_t* h, double* gemm_ms, uint64_t* gemm_launches) {
+    if (!h || !gemm_ms || !gemm_launches) return ALEXNET_ERR_ARG;
+    CK(cudaStreamSynchronize(h->ls));
+    CK(cudaStreamSynchronize(h->cs));
+    double ms = 0.0;
+    for (size_t i = 0; i + 1 < h->prof_used; i += 2) {
+        float t = 0.f;
+        CK(cudaEventElapsedTime(&t, h->prof_ev[i], h->prof_ev[i + 1]));
+        ms += t;
+    }
+    *gemm_ms = ms;
+    *gemm_launches = h->prof_used / 2;
+    h->prof_used = 0;
+    return ALEXNET_OK;
+}
 
 int alexnet_sync(alexnet_t* h) {
     if (!h) return ALEXNET_ERR_ARG;
