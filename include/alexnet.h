@@ -166,6 +166,30 @@ uint64_t alexnet_launch_count(const alexnet_t* h);
 int alexnet_profile(alexnet_t* h, int enable);
 int alexnet_profile_read(alexnet_t* h, double* gemm_ms, uint64_t* gemm_launches);
 
+/* Bias gradient db[c] = sum over rows of dy[row][c], for callers that cannot
+ * allocate device memory when they need it.  (The paper has no counterpart of
+ * this call; it is the bias-gradient reduction of the step offered on its own.)
+ * Such callers are, for example, a loop in the middle of overlapped steps,
+ * where cudaMalloc / cudaFree would synchronise the device and serialise the
+ * loader stream with the compute stream, or a process that has handed all free
+ * HBM to the arena of alexnet_create.  The scratch of the two-stage reduction
+ * lives in a fixed 1 MiB array inside the library image, held by every GPU that
+ * loads the library until the process exits; nothing is allocated or freed.
+ *   dev_dy    device, bf16 [rows][channels], row-major, 16-byte aligned; read only
+ *   rows      >= 1
+ *   channels  multiple of 8, at most 4096 (the fixed scratch); larger values are
+ *             rejected with ALEXNET_ERR_ARG and a message
+ *   dev_db    device, fp32 [channels]; written
+ *   stream    cudaStream_t the two kernels are launched on (asynchronous)
+ *   err       optional host buffer for an error message (may be NULL)
+ * The first call on a device looks up the scratch address for that device;
+ * make that call before any stream capture begins there.  All calls share the
+ * scratch, which keeps the last call's contents (nothing in it needs clearing:
+ * each call overwrites what it later reads), so calls whose kernels could run
+ * at the same time on one GPU race: order them on one stream or with events. */
+int alexnet_bias_grad_noalloc(const void* dev_dy, int64_t rows, int32_t channels, float* dev_db, void* stream,
+                              char* err, size_t err_len);
+
 /* Wait for both streams; returns a latched DEVICE_TIMEOUT or CUDA error if any. */
 int alexnet_sync(alexnet_t* h);
 const char* alexnet_last_error(const alexnet_t* h);

@@ -32,7 +32,7 @@ OP = {n: i for i, n in enumerate(OPS)}
 EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "alexnet_destroy",
            "alexnet_load_batch_async", "alexnet_train_step", "alexnet_replica_average", "alexnet_get_params",
            "alexnet_set_params", "alexnet_tensor_size", "alexnet_get_tensor", "alexnet_set_tensor", "alexnet_run_op",
-           "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error"]
+           "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error", "alexnet_bias_grad_noalloc"]
 
 
 class Config(ctypes.Structure):
@@ -84,6 +84,7 @@ def load_library():
     L.alexnet_sync.argtypes = [vp]
     L.alexnet_last_error.restype = ctypes.c_char_p
     L.alexnet_last_error.argtypes = [vp]
+    L.alexnet_bias_grad_noalloc.argtypes = [vp, ctypes.c_int64, ctypes.c_int32, vp, vp, ctypes.c_char_p, sz]
     _lib = L
     return L
 
@@ -202,3 +203,19 @@ class AlexNet:
     @property
     def launch_count(self):
         return int(self.lib.alexnet_launch_count(self.h))
+
+
+def bias_grad_noalloc(dy, db, stream=None):
+    """db[c] = sum_rows dy[row][c] through the entry point that allocates nothing.
+
+    dy: CUDA bf16 tensor [rows, channels] (contiguous); db: CUDA fp32 tensor
+    [channels], written in place.  For callers that must not allocate device
+    memory (see include/alexnet.h); channels is limited to 4096.  Raises
+    AlexNetError with the library's message when the sizes are rejected."""
+    lib = load_library()
+    msg = ctypes.create_string_buffer(256)
+    rows, ch = int(dy.shape[0]), int(dy.shape[1])
+    rc = lib.alexnet_bias_grad_noalloc(_ptr(dy), rows, ch, _ptr(db),
+                                       ctypes.c_void_p(stream.cuda_stream if stream is not None else 0), msg, 256)
+    if rc != OK:
+        raise AlexNetError(rc, msg.value.decode())

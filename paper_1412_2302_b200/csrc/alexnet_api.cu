@@ -969,3 +969,76 @@ int alexnet_sync(alexnet_t* h) {
 const char* alexnet_last_error(const alexnet_t* h) { return h ? h->err.c_str() : "null handle"; }
 
 }  // extern "C"
+
+// ===================================================================================
+// Bias gradient without any allocation.
+//
+// Some users of this library cannot allocate device memory at the moment they
+// need a bias gradient: a training loop that is in the middle of overlapped
+// steps (cudaMalloc and cudaFree synchronise the whole device, which would
+// serialise the loader stream with the compute stream), or a process that has
+// already given every free byte of HBM to the arena it passed to
+// alexnet_create.  For them this entry point keeps its scratch -- the per-split
+// partial column sums of the two-stage reduction -- in a fixed array that is
+// part of the loaded library image.  Every GPU that loads the library holds
+// that array (kNoAllocSplits * kNoAllocMaxC floats = 1 MiB) until the process
+// exits.
+//
+// The array's name is only a host-side stand-in for the symbol, not a device
+// address, so host code never passes it to a kernel: once per device, with that
+// device current, the address is fetched with cudaGetSymbolAddress and cached.
+// That set-up happens inside the first call on each device, so make that first
+// call before starting any stream capture on that device.
+//
+// All calls share the one array and it keeps whatever the last call left in it.
+// Nothing in it has to start at zero: the first stage writes every partial the
+// second stage reads, in the same call.  Two calls whose kernels overlap on the
+// GPU (different streams, no dependency) race on it; order them.
+namespace {
+constexpr int kNoAllocSplits = 64;
+constexpr int kNoAllocMaxC = 4096;
+static __device__ __align__(256) float g_noalloc_partials[kNoAllocSplits * kNoAllocMaxC];
+
+constexpr int kMaxDevices = 64;
+float* g_noalloc_ptr[kMaxDevices] = {nullptr};
+
+void put_err(char* buf, size_t len, const char* msg) {
+    if (buf && len) { snprintf(buf, len, "%s", msg); }
+}
+}  // namespace
+
+extern "C" int alexnet_bias_grad_noalloc(const void* dev_dy, int64_t rows, int32_t channels, float* dev_db,
+                                         void* stream, char* err, size_t err_len) {
+    if (!dev_dy || !dev_db) { put_err(err, err_len, "bias_grad_noalloc: NULL pointer"); return ALEXNET_ERR_ARG; }
+    if (rows < 1) { put_err(err, err_len, "bias_grad_noalloc: rows must be >= 1"); return ALEXNET_ERR_ARG; }
+    if (channels < 8 || channels % 8 != 0) {
+        put_err(err, err_len, "bias_grad_noalloc: channels must be a positive multiple of 8");
+        return ALEXNET_ERR_ARG;
+    }
+    if (channels > kNoAllocMaxC) {
+        put_err(err, err_len, "bias_grad_noalloc: channels exceeds the fixed scratch (maximum 4096)");
+        return ALEXNET_ERR_ARG;
+    }
+    if (((uintptr_t)dev_dy & 15) != 0) { put_err(err, err_len, "bias_grad_noalloc: dy must be 16-byte aligned"); return ALEXNET_ERR_ARG; }
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) { put_err(err, err_len, "bias_grad_noalloc: cudaGetDevice failed"); return ALEXNET_ERR_CUDA; }
+    if (!g_noalloc_ptr[dev]) {
+        float* p = nullptr;
+        e = cudaGetSymbolAddress((void**)&p, g_noalloc_partials);
+        if (e != cudaSuccess || !p) {
+            put_err(err, err_len, cudaGetErrorString(e));
+            return ALEXNET_ERR_CUDA;
+        }
+        g_noalloc_ptr[dev] = p;
+    }
+    float* scratch = g_noalloc_ptr[dev];
+    cudaStream_t st = (cudaStream_t)stream;
+    int splits = (int)std::min<int64_t>(kNoAllocSplits, std::max<int64_t>(1, rows / 256));
+    dim3 grid((channels + 63) / 64, splits);
+    kn::colsum_kernel<<<grid, 256, 0, st>>>((const bf16*)dev_dy, (long long)rows, channels, scratch);
+    kn::colsum_final_kernel<<<(channels + 127) / 128, 128, 0, st>>>(scratch, splits, channels, dev_db);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { put_err(err, err_len, cudaGetErrorString(e)); return ALEXNET_ERR_CUDA; }
+    return ALEXNET_OK;
+}
