@@ -137,6 +137,7 @@ struct alexnet {
     uint64_t launches;
     int latched;
     float alpha_eff, drop_scale; uint32_t thr24;
+    int sm_count;
     PFN_cuTensorMapEncodeTiled_v12000 encode;
     // optional per-launch timing of the GEMM kernel (event pairs on the launching stream)
     bool prof;
@@ -258,16 +259,19 @@ int make_tm(alexnet* h, CUtensorMap* tm, const void* ptr, uint64_t cols, uint64_
     return ALEXNET_OK;
 }
 
-void finish_plan(Plan& P) {
+void finish_plan(const alexnet* h, Plan& P) {
     tc::GemmParams& p = P.p;
     const int stage_bytes = tc::kABytes + tc::b_stage_bytes(p.mode, p.BN);
     int stages = (227 * 1024 - 2048) / stage_bytes;
-    if (stages > 6) stages = 6;
-    const int per = (p.steps_total + p.splits - 1) / p.splits;
-    if (stages > per) stages = per < 2 ? 2 : per;
+    if (stages > tc::kMaxStages) stages = tc::kMaxStages;
     p.stages = stages;
+    // every split gets at least one k-step
+    const int per = (p.steps_total + p.splits - 1) / p.splits;
+    p.splits = (p.steps_total + per - 1) / per;
+    p.steps_per_split = per;
+    p.tiles_total = p.m_tiles * p.n_tiles * p.groups * p.taps_grid * p.splits;
     P.smem = tc::smem_bytes(p.mode, p.BN, stages);
-    P.grid = p.m_tiles * p.n_tiles * p.groups * p.taps_grid * p.splits;
+    P.grid = std::min(p.tiles_total, h->sm_count);   // persistent: one CTA per SM walks the tile list
     P.valid = true;
 }
 
@@ -288,7 +292,7 @@ int plan_conv_fwd(alexnet* h, Plan& P, const ConvL& c, const bf16* in, const bf1
     int rc;
     if ((rc = make_tm(h, &p.tmA, in, c.cin, M, (uint64_t)c.cin * 2, 128))) return rc;
     if ((rc = make_tm(h, &p.tmB, wsh, c.cig, (uint64_t)c.taps * c.cout, (uint64_t)c.cig * 2, p.BN))) return rc;
-    finish_plan(P);
+    finish_plan(h, P);
     return ALEXNET_OK;
 }
 int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16* wt, const bf16* mask, bf16* dx) {
@@ -307,7 +311,7 @@ int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf1
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, 128))) return rc;
     if ((rc = make_tm(h, &p.tmB, wt, c.cog, (uint64_t)c.taps * c.cin, (uint64_t)c.cog * 2, p.BN))) return rc;
-    finish_plan(P);
+    finish_plan(h, P);
     return ALEXNET_OK;
 }
 int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16* xin) {
@@ -326,7 +330,7 @@ int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, 64))) return rc;
     if ((rc = make_tm(h, &p.tmB, xin, c.cin, M, (uint64_t)c.cin * 2, 64))) return rc;
-    finish_plan(P);
+    finish_plan(h, P);
     return ALEXNET_OK;
 }
 int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* wsh) {
@@ -342,7 +346,7 @@ int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* ws
     int rc;
     if ((rc = make_tm(h, &p.tmA, x, f.K, B, (uint64_t)f.K * 2, 128))) return rc;
     if ((rc = make_tm(h, &p.tmB, wsh, f.K, f.N, (uint64_t)f.K * 2, p.BN))) return rc;
-    finish_plan(P);
+    finish_plan(h, P);
     return ALEXNET_OK;
 }
 int plan_fc_bwd(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* wsh) {
@@ -358,7 +362,7 @@ int plan_fc_bwd(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* w
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, f.N, B, (uint64_t)f.N * 2, 128))) return rc;
     if ((rc = make_tm(h, &p.tmB, wsh, f.K, f.N, (uint64_t)f.K * 2, 64))) return rc;
-    finish_plan(P);
+    finish_plan(h, P);
     return ALEXNET_OK;
 }
 int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x, float* gout) {
@@ -373,7 +377,7 @@ int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x,
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, f.N, B, (uint64_t)f.N * 2, 64))) return rc;
     if ((rc = make_tm(h, &p.tmB, x, f.K, B, (uint64_t)f.K * 2, 64))) return rc;
-    finish_plan(P);
+    finish_plan(h, P);
     return ALEXNET_OK;
 }
 
@@ -720,6 +724,11 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     if (!fn || qres != cudaDriverEntryPointSuccess) { delete h; return ALEXNET_ERR_CUDA; }
     h->encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
     CKC(cudaFuncSetAttribute(tc::gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    {
+        int dev = 0;
+        CKC(cudaGetDevice(&dev));
+        CKC(cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev));
+    }
     // pad positions of every grid must be zero from the start; gradients and momentum start at zero
     CKC(cudaMemsetAsync(h->arena, 0, need, h->cs));
     if (host_mean_image) CKC(cudaMemcpyAsync(h->mean, host_mean_image, 256 * 256 * 3 * sizeof(float), cudaMemcpyHostToDevice, h->cs));

@@ -1,10 +1,14 @@
 // tcgen05 / TMEM / TMA GEMM core for sm_100a.
 //
-// One CTA computes one 128 x BN fp32 accumulator tile in tensor memory from
-// bf16 operands staged in shared memory by TMA (128-byte swizzle), through a
-// ring of STAGES buffers.  Warp roles: warp 0 = TMA producer, warp 1 = MMA
-// issuer (one elected lane) and TMEM owner, warps 2..5 = epilogue (each reads
-// the 32 TMEM lanes of its quadrant).  Three operand arrangements:
+// A persistent kernel: each CTA (one per SM) walks a strided list of 128 x BN
+// output tiles.  bf16 operands are staged in shared memory by TMA (128-byte
+// swizzle) through a ring of `stages` buffers; fp32 accumulators live in tensor
+// memory, double buffered, so the epilogue of tile i overlaps the main loop of
+// tile i+1.  Warp roles: warp 0 = TMA producer (one lane), warp 1 = MMA issuer
+// (one lane) and TMEM owner, warps 2..5 = epilogue (each reads the 32 TMEM
+// lanes of its quadrant).  The single-lane loops carry no division or modulo:
+// stage, phase, tap and chunk counters advance incrementally.
+// Three operand arrangements:
 //   MODE_KK   A K-major, B K-major   conv fwd, conv bwd-data, FC fwd
 //   MODE_KMN  A K-major, B MN-major  FC bwd-data (weights read untransposed)
 //   MODE_MNMN A MN-major, B MN-major weight gradients (reduction over rows)
@@ -24,16 +28,19 @@ enum { MODE_KK = 0, MODE_KMN = 1, MODE_MNMN = 2 };
 enum { EPI_BF16 = 0, EPI_F32 = 1 };
 constexpr int kThreads = 192;
 constexpr int kMaxTaps = 25;
+constexpr int kMaxStages = 8;
 constexpr long long kWaitBudgetCycles = 400000000LL;  // ~0.2 s at 2 GHz
 
 struct GemmParams {
     CUtensorMap tmA, tmB;
     int mode, epi;
-    int m_tiles, n_tiles, groups, taps_grid, splits;  // grid decomposition (m fastest)
+    int m_tiles, n_tiles, groups, taps_grid, splits;  // tile decomposition (m fastest)
+    int tiles_total;
     int BN;            // MMA N (multiple of 16, <= 256)
     int kk;            // K=16 MMAs per stage (<= 4)
     int chunks;        // MODE_KK: 64-element K chunks per tap
     int steps_total;   // k-steps over the whole reduction (split evenly over `splits`)
+    int steps_per_split;
     int stages;        // smem ring depth
     int a_x0, a_gx;    // A column origin and per-group column stride
     int b_gx;          // MODE_MNMN: B per-group column stride
@@ -63,6 +70,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -74,10 +84,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // bounded wait: returns false when the cycle budget ran out or another role aborted
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    long long t0 = clock64();
+    #pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
     while (true) {
-        for (int i = 0; i < 64; ++i)
+        #pragma unroll 1
+        for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (clock64() - t0 > kWaitBudgetCycles) { *abort_flag = 1; return false; }
@@ -87,6 +100,9 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
@@ -147,73 +163,113 @@ inline size_t smem_bytes(int mode, int BN, int stages) {
     return 1024 + (size_t)stages * (kABytes + b_stage_bytes(mode, BN)) + 256;
 }
 
+// position of a CTA in the tile list; tiles are numbered with m fastest, then
+// n tile, group, tap (weight gradients), k split
+struct TileCursor {
+    int m_tile, rest;          // rest = tile / m_tiles
+    int n_tile, g, tap_g, z;   // decoded from rest
+    __device__ __forceinline__ void decode(const GemmParams& p) {
+        int r = rest;
+        n_tile = r % p.n_tiles; r /= p.n_tiles;
+        g = r % p.groups; r /= p.groups;
+        tap_g = r % p.taps_grid;
+        z = r / p.taps_grid;
+    }
+    __device__ __forceinline__ void init(const GemmParams& p) {
+        m_tile = blockIdx.x % p.m_tiles;
+        rest = blockIdx.x / p.m_tiles;
+        decode(p);
+    }
+    __device__ __forceinline__ void next(const GemmParams& p) {
+        m_tile += gridDim.x;
+        if (m_tile >= p.m_tiles) {
+            do { m_tile -= p.m_tiles; ++rest; } while (m_tile >= p.m_tiles);
+            decode(p);
+        }
+    }
+};
+
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     const int bbytes = b_stage_bytes(p.mode, p.BN);
     const int stage_bytes = kABytes + bbytes;
-    const uint32_t bar_base = base + p.stages * stage_bytes;       // full[8], empty[8], accum, tmem slot
-    uint8_t* gen = smem_raw + (base - raw) + p.stages * stage_bytes;
-    volatile int* abort_flag = (volatile int*)(gen + 160);
-    volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 144);
-    auto full_bar = [&](int s) { return bar_base + 8u * s; };
-    auto empty_bar = [&](int s) { return bar_base + 64u + 8u * s; };
-    const uint32_t accum_bar = bar_base + 128u;
+    const int stages = p.stages;
+    // barriers: full[8] @0, empty[8] @64, acc_full[2] @128, acc_empty[2] @144, tmem slot @160, abort flag @168
+    const uint32_t bar_base = base + stages * stage_bytes;
+    uint8_t* gen = smem_raw + (base - raw) + stages * stage_bytes;
+    volatile int* abort_flag = (volatile int*)(gen + 168);
+    volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 160);
+    const uint32_t full0 = bar_base, empty0 = bar_base + 64u, accf0 = bar_base + 128u, acce0 = bar_base + 144u;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // tile decode (m fastest)
-    int idx = blockIdx.x;
-    const int m_tile = idx % p.m_tiles; idx /= p.m_tiles;
-    const int n_tile = idx % p.n_tiles; idx /= p.n_tiles;
-    const int g = idx % p.groups; idx /= p.groups;
-    const int tap_g = idx % p.taps_grid; idx /= p.taps_grid;
-    const int z = idx;
-    const int m0 = m_tile * 128, n0 = n_tile * p.BN;
-    const int per = (p.steps_total + p.splits - 1) / p.splits;
-    const int s_begin = z * per;
-    const int s_end = min(p.steps_total, s_begin + per);
-    const int nsteps = max(0, s_end - s_begin);
-
     uint32_t ncols = 32;
-    while ((int)ncols < p.BN) ncols <<= 1;
+    while ((int)ncols < 2 * p.BN) ncols <<= 1;
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        for (int s = 0; s < p.stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        mbar_init(accum_bar, 1);
+        for (int s = 0; s < stages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(accf0 + 8u * s, 1); mbar_init(acce0 + 8u * s, 128); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&p.tmA);
+        tma_prefetch_desc(&p.tmB);
     }
     if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), ncols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    const int per = p.steps_per_split;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             const uint32_t tx = (uint32_t)stage_bytes;
-            for (int i = 0; i < nsteps; ++i) {
-                const int s = s_begin + i, st = i % p.stages;
-                if (!mbar_wait(empty_bar(st), ((i / p.stages) & 1) ^ 1, abort_flag)) break;
-                const uint32_t sa = base + st * stage_bytes, sb = sa + kABytes;
-                mbar_expect_tx(full_bar(st), tx);
+            const int nb = (p.BN + 63) >> 6;
+            TileCursor tc; tc.init(p);
+            int st = 0; uint32_t ph = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
+                const int m0 = tc.m_tile * 128, n0 = tc.n_tile * p.BN;
+                const int s_begin = tc.z * per;
+                const int nsteps = min(p.steps_total, s_begin + per) - s_begin;
                 if (p.mode == MODE_KK) {
-                    const int tap = s / p.chunks, ch = s - tap * p.chunks;
-                    tma_load_2d(sa, &p.tmA, p.a_x0 + g * p.a_gx + ch * 64, m0 + p.shift[tap], full_bar(st));
-                    tma_load_2d(sb, &p.tmB, ch * 64, tap * p.b_tap_rows + g * p.b_g_rows + n0, full_bar(st));
+                    int tap = 0, ch = s_begin;
+                    if (p.chunks < p.steps_total && s_begin > 0) { tap = s_begin / p.chunks; ch = s_begin - tap * p.chunks; }
+                    const int xa = p.a_x0 + tc.g * p.a_gx, yb = tc.g * p.b_g_rows + n0;
+                    for (int i = 0; i < nsteps; ++i) {
+                        if (!(ok = mbar_wait(empty0 + 8u * st, ph ^ 1u, abort_flag))) break;
+                        const uint32_t sa = base + st * stage_bytes, fb = full0 + 8u * st;
+                        mbar_expect_tx(fb, tx);
+                        tma_load_2d(sa, &p.tmA, xa + ch * 64, m0 + p.shift[tap], fb);
+                        tma_load_2d(sa + kABytes, &p.tmB, ch * 64, tap * p.b_tap_rows + yb, fb);
+                        if (++ch == p.chunks) { ch = 0; ++tap; }
+                        if (++st == stages) { st = 0; ph ^= 1u; }
+                    }
                 } else if (p.mode == MODE_KMN) {
-                    tma_load_2d(sa, &p.tmA, s * 64, m0, full_bar(st));
-                    for (int j = 0; j < (p.BN + 63) / 64; ++j)
-                        tma_load_2d(sb + j * 8192, &p.tmB, n0 + 64 * j, s * 64, full_bar(st));
+                    for (int i = 0; i < nsteps; ++i) {
+                        if (!(ok = mbar_wait(empty0 + 8u * st, ph ^ 1u, abort_flag))) break;
+                        const uint32_t sa = base + st * stage_bytes, fb = full0 + 8u * st;
+                        const int q = (s_begin + i) * 64;
+                        mbar_expect_tx(fb, tx);
+                        tma_load_2d(sa, &p.tmA, q, m0, fb);
+                        for (int j = 0; j < nb; ++j) tma_load_2d(sa + kABytes + j * 8192, &p.tmB, n0 + 64 * j, q, fb);
+                        if (++st == stages) { st = 0; ph ^= 1u; }
+                    }
                 } else {
-                    const int q = s * 64;
-                    for (int j = 0; j < 2; ++j)
-                        tma_load_2d(sa + j * 8192, &p.tmA, g * p.a_gx + m0 + 64 * j, q, full_bar(st));
-                    for (int j = 0; j < (p.BN + 63) / 64; ++j)
-                        tma_load_2d(sb + j * 8192, &p.tmB, g * p.b_gx + n0 + 64 * j, q + p.shift[tap_g], full_bar(st));
+                    const int xa = tc.g * p.a_gx + m0, xb = tc.g * p.b_gx + n0, sh = p.shift[tc.tap_g];
+                    for (int i = 0; i < nsteps; ++i) {
+                        if (!(ok = mbar_wait(empty0 + 8u * st, ph ^ 1u, abort_flag))) break;
+                        const uint32_t sa = base + st * stage_bytes, fb = full0 + 8u * st;
+                        const int q = (s_begin + i) * 64;
+                        mbar_expect_tx(fb, tx);
+                        tma_load_2d(sa, &p.tmA, xa, q, fb);
+                        tma_load_2d(sa + 8192, &p.tmA, xa + 64, q, fb);
+                        for (int j = 0; j < nb; ++j) tma_load_2d(sa + kABytes + j * 8192, &p.tmB, xb + 64 * j, q + sh, fb);
+                        if (++st == stages) { st = 0; ph ^= 1u; }
+                    }
                 }
             }
         }
@@ -224,32 +280,49 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             const uint32_t idesc = instr_desc(p.BN, a_mn, b_mn);
             const uint32_t a_adv = a_mn ? 2048u : 32u, b_adv = b_mn ? 2048u : 32u;
             const uint32_t a_lbo = a_mn ? 8192u : 16u, b_lbo = b_mn ? 8192u : 16u;
+            const int kk = p.kk;
+            TileCursor tc; tc.init(p);
+            int st = 0; uint32_t ph = 0;
+            int ab = 0; uint32_t aph = 0;
             bool ok = true;
-            for (int i = 0; i < nsteps && ok; ++i) {
-                const int st = i % p.stages;
-                ok = mbar_wait(full_bar(st), (i / p.stages) & 1, abort_flag);
-                if (!ok) break;
+            for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
+                const int s_begin = tc.z * per;
+                const int nsteps = min(p.steps_total, s_begin + per) - s_begin;
+                if (!(ok = mbar_wait(acce0 + 8u * ab, aph ^ 1u, abort_flag))) break;
                 tc_fence_after();
-                const uint32_t sa = base + st * stage_bytes, sb = sa + kABytes;
-                for (int j = 0; j < p.kk; ++j)
-                    umma(tmem, smem_desc(sa + j * a_adv, a_lbo, 1024), smem_desc(sb + j * b_adv, b_lbo, 1024),
-                         idesc, (i > 0 || j > 0) ? 1u : 0u);
-                umma_commit(empty_bar(st));
+                const uint32_t d = tmem + (uint32_t)(ab * p.BN);
+                for (int i = 0; i < nsteps; ++i) {
+                    if (!(ok = mbar_wait(full0 + 8u * st, ph, abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t sa = base + st * stage_bytes, sb = sa + kABytes;
+                    #pragma unroll 4
+                    for (int j = 0; j < kk; ++j)
+                        umma(d, smem_desc(sa + j * a_adv, a_lbo, 1024), smem_desc(sb + j * b_adv, b_lbo, 1024),
+                             idesc, (i > 0 || j > 0) ? 1u : 0u);
+                    umma_commit(empty0 + 8u * st);
+                    if (++st == stages) { st = 0; ph ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(accf0 + 8u * ab);
+                if (++ab == 2) { ab = 0; aph ^= 1u; }
             }
-            umma_commit(accum_bar);
         }
     } else {
         // ------------------------------------------------------------ epilogue
         const int quad = warp & 3;
         const int r = quad * 32 + lane;          // row within the tile = TMEM lane
-        bool ok = mbar_wait(accum_bar, 0, abort_flag);
-        tc_fence_after();
-        if (ok) {
+        TileCursor tc; tc.init(p);
+        int ab = 0; uint32_t aph = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
+            const int m0 = tc.m_tile * 128, n0 = tc.n_tile * p.BN, g = tc.g;
+            const int s_begin = tc.z * per;
+            const int nsteps = min(p.steps_total, s_begin + per) - s_begin;
             bool row_ok, pad_row = false;
             long long row_off;
             if (p.mode == MODE_MNMN) {
                 row_ok = (m0 + r) < p.M_total;
-                row_off = (long long)z * p.split_stride + (long long)tap_g * p.tap_stride +
+                row_off = (long long)tc.z * p.split_stride + (long long)tc.tap_g * p.tap_stride +
                           (long long)(g * p.out_gx + m0 + r) * p.ldo;
             } else {
                 const int row = m0 + r;
@@ -258,15 +331,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     const int x = row % p.Wp, y = (row / p.Wp) % p.Hp;
                     pad_row = (x >= p.W) || (y >= p.H);
                 }
-                row_off = (long long)z * p.split_stride + (long long)row * p.ldo + g * p.out_gx;
+                row_off = (long long)tc.z * p.split_stride + (long long)row * p.ldo + g * p.out_gx;
             }
+            if (!(ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag))) break;
+            tc_fence_after();
+            const uint32_t t0 = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * p.BN);
             for (int c = 0; c < p.BN; c += 16) {
                 uint32_t v[16];
-                tmem_ld16(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)c, v);
+                tmem_ld16(t0 + (uint32_t)c, v);
                 tmem_ld_wait();
                 if (!row_ok) continue;
                 const int col0 = n0 + c;
-                if (nsteps == 0) {
+                if (nsteps <= 0) {
                     #pragma unroll
                     for (int k = 0; k < 16; ++k) v[k] = 0u;
                 }
@@ -323,6 +399,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     }
                 }
             }
+            // this accumulator buffer may be overwritten by the next tile but one
+            tc_fence_before();
+            mbar_arrive(acce0 + 8u * ab);
+            if (++ab == 2) { ab = 0; aph ^= 1u; }
         }
     }
     tc_fence_before();
