@@ -98,7 +98,7 @@ Layout make_layout() {
 const long long kCanonCount = 60965224;
 
 // ------------------------------------------------------------------- handle
-struct Plan { tc::GemmParams p; int grid; size_t smem; bool valid; };
+struct Plan { tc::GemmParams p; tc::ConvParams c; bool conv; int grid; size_t smem; bool valid; };
 
 struct Tensor {  // description of one exportable device tensor
     void* ptr; int kind; int C, Hp, Wp, H, W; long long N;
@@ -275,43 +275,107 @@ void finish_plan(const alexnet* h, Plan& P) {
     P.valid = true;
 }
 
+// Tile shape of the convolution kernel for a problem of M rows, N output channels per group, `groups`
+// groups, a kh x kw filter over `chunks` 64-channel chunks: the (row halves, BN) pair with the lowest
+// modelled time.  Per weight stage the tensor pipe needs MH*kk*BN/2 cycles; TMA brings about 64 bytes
+// per cycle per SM from L2; tiles are dealt to the SMs in rounds.
+struct ConvShape { int MH, BN, acc_stages; };
+ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, int kh, int kw, int chunks, int kk) {
+    ConvShape best{1, N <= 256 ? N : 128, 1};
+    double best_t = 1e30;
+    const int a_rows = kw > 1 ? 136 : 128;
+    const size_t budget = 227 * 1024 - 2048;
+    for (int MH = 1; MH <= 4; MH *= 2) {
+        for (int BN = 16; BN <= 256 && BN <= N; BN += 16) {
+            if (N % BN) continue;
+            if (MH * BN > 512) continue;
+            if (2 * (size_t)MH * a_rows * 128 + 4 * (size_t)BN * 128 > budget) continue;
+            const int acc = 2 * MH * BN <= 512 ? 2 : 1;
+            const long long tiles = ((M + 128 * MH - 1) / (128 * MH)) * (N / BN) * groups;
+            const long long rounds = (tiles + h->sm_count - 1) / h->sm_count;
+            // per weight stage: the pipe needs MH*kk*BN/2 cycles, each issuer about 105 cycles per instruction
+            const double mma = kw * kk * std::max(MH * BN / 2.0, 105.0);
+            const double tma = ((double)MH * a_rows * 128 + (double)kw * BN * 128) / 72.0;
+            double tile_t = (double)kh * chunks * std::max(mma, tma) + 800.0;
+            const double epi = MH * (BN / 16) * 170.0;
+            if (acc == 1) tile_t += epi; else tile_t = std::max(tile_t, epi + 300.0);
+            const double t = rounds * tile_t;
+            if (t < best_t) { best_t = t; best = ConvShape{MH, BN, acc}; }
+        }
+    }
+    return best;
+}
+
+void finish_conv_plan(const alexnet* h, Plan& P) {
+    tc::ConvParams& c = P.c;
+    const int per = (c.asteps_total + c.splits - 1) / c.splits;
+    c.splits = (c.asteps_total + per - 1) / per;
+    c.asteps_per_split = per;
+    c.tiles_total = c.m_tiles * c.n_tiles * c.groups * c.splits;
+    const size_t a_bytes = (size_t)c.MH * c.a_box_rows * 128, b_bytes = (size_t)c.BN * 128;
+    const size_t budget = 227 * 1024 - 2048;
+    if (c.kw == 1) {
+        int st = (int)(budget / (a_bytes + b_bytes));
+        st = std::min(st, 8);
+        c.a_stages = c.b_stages = st;
+    } else {
+        c.a_stages = 3;
+        if (budget < 3 * a_bytes + 4 * b_bytes) c.a_stages = 2;
+        c.b_stages = (int)std::min<size_t>(8, (budget - c.a_stages * a_bytes) / b_bytes);
+    }
+    P.conv = true;
+    P.smem = tc::conv_smem_bytes(c);
+    P.grid = std::min(c.tiles_total, h->sm_count);
+    P.valid = true;
+}
+
 int plan_conv_fwd(alexnet* h, Plan& P, const ConvL& c, const bf16* in, const bf16* wsh, const float* bias, bf16* out) {
     memset(&P, 0, sizeof(P));
-    tc::GemmParams& p = P.p;
+    tc::ConvParams& p = P.c;
     const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
-    p.mode = tc::MODE_KK; p.epi = tc::EPI_BF16;
-    p.M_total = (int)M; p.m_tiles = (int)((M + 127) / 128);
-    p.BN = c.cog <= 256 ? c.cog : 192; p.n_tiles = c.cog / p.BN;
-    p.groups = c.groups; p.taps_grid = 1; p.splits = 1;
-    p.kk = c.cig == 48 ? 3 : 4; p.chunks = (c.cig + 63) / 64; p.steps_total = c.taps * p.chunks;
+    const int gp = c.gin.Wp;
+    p.kh = p.kw = c.k; p.chunks = (c.cig + 63) / 64; p.kk = c.cig == 48 ? 3 : 4;
+    const ConvShape sh = choose_conv_shape(h, M, c.cog, c.groups, p.kh, p.kw, p.chunks, p.kk);
+    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages;
+    p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH - 1) / (128 * p.MH));
+    p.n_tiles = c.cog / p.BN; p.groups = c.groups; p.splits = 1;
+    p.asteps_total = p.kh * p.chunks;
+    p.a_box_rows = p.kw > 1 ? 136 : 128;
     p.a_x0 = 0; p.a_gx = c.cig; p.b_tap_rows = c.cout; p.b_g_rows = c.cog;
-    for (int t = 0; t < c.taps; ++t) p.shift[t] = c.shift[t];
-    p.n_valid = c.cog; p.ldo = c.cout; p.out_gx = c.cog;
+    for (int ky = 0; ky < c.k; ++ky) p.halo_shift[ky] = (ky - c.pad) * gp - c.pad;
+    for (int kx = 0; kx < c.k; ++kx) p.tap_off[kx] = kx;
+    p.epi = tc::EPI_BF16; p.n_valid = c.cog; p.ldo = c.cout; p.out_gx = c.cog;
     p.Hp = c.gout.Hp; p.Wp = c.gout.Wp; p.H = c.gout.H; p.W = c.gout.W;
     p.relu = 1; p.mask_scale = 1.f; p.bias = bias; p.mask = nullptr; p.out = out; p.status = h->status;
     int rc;
-    if ((rc = make_tm(h, &p.tmA, in, c.cin, M, (uint64_t)c.cin * 2, 128))) return rc;
+    if ((rc = make_tm(h, &p.tmA, in, c.cin, M, (uint64_t)c.cin * 2, p.a_box_rows))) return rc;
     if ((rc = make_tm(h, &p.tmB, wsh, c.cig, (uint64_t)c.taps * c.cout, (uint64_t)c.cig * 2, p.BN))) return rc;
-    finish_plan(h, P);
+    finish_conv_plan(h, P);
     return ALEXNET_OK;
 }
 int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16* wt, const bf16* mask, bf16* dx) {
     memset(&P, 0, sizeof(P));
-    tc::GemmParams& p = P.p;
+    tc::ConvParams& p = P.c;
     const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
-    p.mode = tc::MODE_KK; p.epi = tc::EPI_BF16;
-    p.M_total = (int)M; p.m_tiles = (int)((M + 127) / 128);
-    p.BN = c.cig; p.n_tiles = 1; p.groups = c.groups; p.taps_grid = 1; p.splits = 1;
-    p.kk = 4; p.chunks = c.cog / 64; p.steps_total = c.taps * p.chunks;
+    const int gp = c.gin.Wp;
+    p.kh = p.kw = c.k; p.chunks = c.cog / 64; p.kk = 4;
+    const ConvShape sh = choose_conv_shape(h, M, c.cig, c.groups, p.kh, p.kw, p.chunks, p.kk);
+    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages;
+    p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH - 1) / (128 * p.MH));
+    p.n_tiles = c.cig / p.BN; p.groups = c.groups; p.splits = 1;
+    p.asteps_total = p.kh * p.chunks;
+    p.a_box_rows = p.kw > 1 ? 136 : 128;
     p.a_x0 = 0; p.a_gx = c.cog; p.b_tap_rows = c.cin; p.b_g_rows = c.cig;
-    for (int t = 0; t < c.taps; ++t) p.shift[t] = -c.shift[t];
-    p.n_valid = c.cig; p.ldo = c.cin; p.out_gx = c.cig;
+    // the gradient at input row m gathers dy at m - shift(ky,kx): per filter row the taps read descending rows
+    for (int ky = 0; ky < c.k; ++ky) p.halo_shift[ky] = -(ky - c.pad) * gp + c.pad - (c.k - 1);
+    for (int kx = 0; kx < c.k; ++kx) p.tap_off[kx] = c.k - 1 - kx;
+    p.epi = tc::EPI_BF16; p.n_valid = c.cig; p.ldo = c.cin; p.out_gx = c.cig;
     p.Hp = c.gin.Hp; p.Wp = c.gin.Wp; p.H = c.gin.H; p.W = c.gin.W;
     p.relu = 0; p.mask_scale = 1.f; p.bias = nullptr; p.mask = mask; p.out = dx; p.status = h->status;
     int rc;
-    if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, 128))) return rc;
+    if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, p.a_box_rows))) return rc;
     if ((rc = make_tm(h, &p.tmB, wt, c.cog, (uint64_t)c.taps * c.cin, (uint64_t)c.cog * 2, p.BN))) return rc;
-    finish_plan(h, P);
+    finish_conv_plan(h, P);
     return ALEXNET_OK;
 }
 int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16* xin) {
@@ -335,18 +399,21 @@ int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16
 }
 int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* wsh) {
     memset(&P, 0, sizeof(P));
-    tc::GemmParams& p = P.p;
+    tc::ConvParams& p = P.c;
     const int B = h->B;
-    p.mode = tc::MODE_KK; p.epi = tc::EPI_F32;
-    p.M_total = B; p.m_tiles = (B + 127) / 128; p.BN = fc_fwd_bn(f); p.n_tiles = (f.N + p.BN - 1) / p.BN;
-    p.groups = 1; p.taps_grid = 1; p.splits = fc_fwd_splits(f, B);
-    p.kk = 4; p.chunks = f.K / 64; p.steps_total = p.chunks;
-    p.n_valid = f.N; p.ldo = f.N; p.split_stride = (long long)B * f.N;
-    p.out = h->ws; p.status = h->status;
+    p.kh = p.kw = 1; p.chunks = f.K / 64; p.kk = 4;
+    p.MH = 1; p.BN = fc_fwd_bn(f); p.acc_stages = 2;
+    p.M_total = B; p.m_tiles = (B + 127) / 128; p.n_tiles = (f.N + p.BN - 1) / p.BN;
+    p.groups = 1; p.splits = fc_fwd_splits(f, B);
+    p.asteps_total = p.chunks;
+    p.a_box_rows = 128;
+    p.halo_shift[0] = 0; p.tap_off[0] = 0;
+    p.epi = tc::EPI_F32; p.n_valid = f.N; p.ldo = f.N; p.split_stride = (long long)B * f.N;
+    p.mask_scale = 1.f; p.out = h->ws; p.status = h->status;
     int rc;
     if ((rc = make_tm(h, &p.tmA, x, f.K, B, (uint64_t)f.K * 2, 128))) return rc;
     if ((rc = make_tm(h, &p.tmB, wsh, f.K, f.N, (uint64_t)f.K * 2, p.BN))) return rc;
-    finish_plan(h, P);
+    finish_conv_plan(h, P);
     return ALEXNET_OK;
 }
 int plan_fc_bwd(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* wsh) {
@@ -422,7 +489,8 @@ void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
         }
     }
     if (h->prof) cudaEventRecord(h->prof_ev[h->prof_used], st);
-    tc::gemm_kernel<<<P.grid, tc::kThreads, P.smem, st>>>(P.p);
+    if (P.conv) tc::conv_kernel<<<P.grid, tc::conv_threads(P.c), P.smem, st>>>(P.c);
+    else tc::gemm_kernel<<<P.grid, tc::kThreads, P.smem, st>>>(P.p);
     if (h->prof) { cudaEventRecord(h->prof_ev[h->prof_used + 1], st); h->prof_used += 2; }
     h->launches++;
 }
@@ -471,7 +539,7 @@ void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st) {
     uint8_t* keeps[3] = {R.m6, R.m7, nullptr};
     const int drop = l < 2 && h->cfg.dropout_p > 0.f;
     const uint64_t key = kn::stream_key(h->cfg.seed, 2 + l, r, step);
-    kn::fc_reduce_fwd_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, R.w + f.b_off, h->B, f.N,
+    kn::fc_reduce_fwd_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.c.splits, P.c.split_stride, R.w + f.b_off, h->B, f.N,
                                                                 l < 2, drop, key, h->thr24, h->drop_scale, outs[l],
                                                                 l == 2 ? R.z : nullptr, keeps[l]);
     h->launches++;
@@ -724,6 +792,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     if (!fn || qres != cudaDriverEntryPointSuccess) { delete h; return ALEXNET_ERR_CUDA; }
     h->encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
     CKC(cudaFuncSetAttribute(tc::gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CKC(cudaFuncSetAttribute(tc::conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     {
         int dev = 0;
         CKC(cudaGetDevice(&dev));

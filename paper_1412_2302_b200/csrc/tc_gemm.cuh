@@ -154,6 +154,68 @@ __device__ __forceinline__ uint32_t instr_desc(int N, int a_mn, int b_mn) {
     return d;
 }
 
+// One 16-column slice of an accumulator row: bias, ReLU, pad-row zeroing, ReLU/dropout
+// mask, conversion and store.  P is a parameter struct with the epilogue fields.
+template <typename P>
+__device__ __forceinline__ void epi_chunk(const P& p, uint32_t* v, bool zero, bool pad_row, long long row_off, int col0, int g) {
+    if (zero) {
+        #pragma unroll
+        for (int k = 0; k < 16; ++k) v[k] = 0u;
+    }
+    if (p.epi == EPI_F32) {
+        float* o = (float*)p.out + row_off + col0;
+        if (col0 + 16 <= p.n_valid) {
+            #pragma unroll
+            for (int k = 0; k < 16; k += 4)
+                *(float4*)(o + k) = make_float4(__uint_as_float(v[k]), __uint_as_float(v[k + 1]),
+                                                __uint_as_float(v[k + 2]), __uint_as_float(v[k + 3]));
+        } else {
+            for (int k = 0; k < 16; ++k)
+                if (col0 + k < p.n_valid) o[k] = __uint_as_float(v[k]);
+        }
+        return;
+    }
+    __nv_bfloat16* o = (__nv_bfloat16*)p.out + row_off + col0;
+    float f[16];
+    #pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        float t = __uint_as_float(v[k]);
+        if (p.bias) t += p.bias[g * p.out_gx + min(col0 + k, p.n_valid - 1)];
+        if (p.relu) t = fmaxf(t, 0.f);
+        f[k] = pad_row ? 0.f : t;
+    }
+    if (p.mask) {
+        const __nv_bfloat16* mk = p.mask + row_off + col0;
+        if (col0 + 16 <= p.n_valid) {
+            uint4 m0v = *(const uint4*)mk, m1v = *(const uint4*)(mk + 8);
+            const __nv_bfloat16* mm = (const __nv_bfloat16*)&m0v;
+            const __nv_bfloat16* mn = (const __nv_bfloat16*)&m1v;
+            #pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                f[k] = __bfloat162float(mm[k]) > 0.f ? f[k] * p.mask_scale : 0.f;
+                f[k + 8] = __bfloat162float(mn[k]) > 0.f ? f[k + 8] * p.mask_scale : 0.f;
+            }
+        } else {
+            for (int k = 0; k < 16; ++k)
+                if (col0 + k < p.n_valid)
+                    f[k] = __bfloat162float(mk[k]) > 0.f ? f[k] * p.mask_scale : 0.f;
+        }
+    }
+    if (col0 + 16 <= p.n_valid) {
+        uint32_t w[8];
+        #pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);
+            w[k] = *(uint32_t*)&h;
+        }
+        *(uint4*)o = make_uint4(w[0], w[1], w[2], w[3]);
+        *(uint4*)(o + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+    } else {
+        for (int k = 0; k < 16; ++k)
+            if (col0 + k < p.n_valid) o[k] = __float2bfloat16_rn(f[k]);
+    }
+}
+
 constexpr int kABytes = 128 * 128;  // 128 rows x 64 bf16, or 2 boxes of 64 x 64
 
 __host__ __device__ inline int b_stage_bytes(int mode, int BN) {
@@ -341,63 +403,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 tmem_ld16(t0 + (uint32_t)c, v);
                 tmem_ld_wait();
                 if (!row_ok) continue;
-                const int col0 = n0 + c;
-                if (nsteps <= 0) {
-                    #pragma unroll
-                    for (int k = 0; k < 16; ++k) v[k] = 0u;
-                }
-                if (p.epi == EPI_F32) {
-                    float* o = (float*)p.out + row_off + col0;
-                    if (col0 + 16 <= p.n_valid) {
-                        #pragma unroll
-                        for (int k = 0; k < 16; k += 4)
-                            *(float4*)(o + k) = make_float4(__uint_as_float(v[k]), __uint_as_float(v[k + 1]),
-                                                            __uint_as_float(v[k + 2]), __uint_as_float(v[k + 3]));
-                    } else {
-                        for (int k = 0; k < 16; ++k)
-                            if (col0 + k < p.n_valid) o[k] = __uint_as_float(v[k]);
-                    }
-                } else {
-                    __nv_bfloat16* o = (__nv_bfloat16*)p.out + row_off + col0;
-                    float f[16];
-                    #pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        float t = __uint_as_float(v[k]);
-                        if (p.bias) t += p.bias[g * p.out_gx + min(col0 + k, p.n_valid - 1)];
-                        if (p.relu) t = fmaxf(t, 0.f);
-                        f[k] = pad_row ? 0.f : t;
-                    }
-                    if (p.mask) {
-                        const __nv_bfloat16* mk = p.mask + row_off + col0;
-                        if (col0 + 16 <= p.n_valid) {
-                            uint4 m0v = *(const uint4*)mk, m1v = *(const uint4*)(mk + 8);
-                            const __nv_bfloat16* mm = (const __nv_bfloat16*)&m0v;
-                            const __nv_bfloat16* mn = (const __nv_bfloat16*)&m1v;
-                            #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                f[k] = __bfloat162float(mm[k]) > 0.f ? f[k] * p.mask_scale : 0.f;
-                                f[k + 8] = __bfloat162float(mn[k]) > 0.f ? f[k + 8] * p.mask_scale : 0.f;
-                            }
-                        } else {
-                            for (int k = 0; k < 16; ++k)
-                                if (col0 + k < p.n_valid)
-                                    f[k] = __bfloat162float(mk[k]) > 0.f ? f[k] * p.mask_scale : 0.f;
-                        }
-                    }
-                    if (col0 + 16 <= p.n_valid) {
-                        uint32_t w[8];
-                        #pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * k], f[2 * k + 1]);
-                            w[k] = *(uint32_t*)&h;
-                        }
-                        *(uint4*)o = make_uint4(w[0], w[1], w[2], w[3]);
-                        *(uint4*)(o + 8) = make_uint4(w[4], w[5], w[6], w[7]);
-                    } else {
-                        for (int k = 0; k < 16; ++k)
-                            if (col0 + k < p.n_valid) o[k] = __float2bfloat16_rn(f[k]);
-                    }
-                }
+                epi_chunk(p, v, nsteps <= 0, pad_row, row_off, n0 + c, g);
             }
             // this accumulator buffer may be overwritten by the next tile but one
             tc_fence_before();
@@ -409,6 +415,246 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     __syncthreads();
     if (*abort_flag) {
         // a wait expired: give in-flight copies time to land before the block retires
+        if (threadIdx.x == 0 && p.status) atomicExch(p.status, 1);
+        long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) { }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, ncols);
+    }
+}
+
+// ===========================================================================
+// Convolution / FC-forward kernel (both operands K-major) with operand reuse.
+//
+// One tile = MH x 128 output rows by BN output channels (MH = 1, 2 or 4).  For
+// each filter row ky and each 64-channel chunk the producer loads ONE "halo" of
+// activation rows (MH boxes of a_box_rows rows, covering MH*128 + kw - 1
+// consecutive rows of the flat grid); the kw taps of that filter row read it at
+// row offsets tap_off[kx] through shared-memory descriptors whose start address
+// is advanced by whole 128-byte rows.  Every weight tile (BN rows x 64 channels
+// of one tap) is used by the MH row halves.  Activations and weights therefore
+// travel in separate rings: an A stage lives for kw B stages.
+// One thread issues a tcgen05.mma roughly every 100 cycles, which is slower
+// than the tensor pipe for N < 192; so each 128-row half has its own issuer
+// warp (they write disjoint accumulators) and the pipe stays fed.
+// Warps: 0 = TMA producer, 1..MH = MMA issuers, MH+1..MH+4 = epilogue.
+// Accumulators: MH x BN columns per buffer, two buffers when they fit in the
+// 512 TMEM columns.
+struct ConvParams {
+    CUtensorMap tmA, tmB;
+    int m_tiles, n_tiles, groups, splits;   // tile decomposition (m fastest, then n, group, k split)
+    int tiles_total;
+    int MH;             // 128-row halves per tile (1, 2 or 4)
+    int BN, kk;         // MMA N (multiple of 16, <= 256); K=16 MMAs per weight stage (<= 4)
+    int kh, kw;         // filter rows; taps per filter row
+    int chunks;         // 64-channel chunks
+    int asteps_total;   // kh * chunks, split evenly over `splits`
+    int asteps_per_split;
+    int a_stages, b_stages, acc_stages;
+    int a_box_rows;     // rows per activation box (128, or 136 when kw > 1)
+    int a_x0, a_gx;     // A column origin and per-group column stride
+    int b_tap_rows, b_g_rows;   // B row = (ky*kw+kx)*b_tap_rows + g*b_g_rows + n0
+    int halo_shift[5];  // per ky: first halo row relative to the tile's first output row
+    int tap_off[5];     // per kx: row offset of the tap inside the halo
+    // epilogue (same meaning as in GemmParams)
+    int epi, M_total, n_valid, ldo, out_gx;
+    long long split_stride;
+    int Hp, Wp, H, W, relu;
+    float mask_scale;
+    const float* bias;
+    const __nv_bfloat16* mask;
+    void* out;
+    int* status;
+};
+
+constexpr int kConvMaxThreads = 32 * 9;
+inline int conv_threads(const ConvParams& p) { return 32 * (5 + p.MH); }
+inline size_t conv_smem_bytes(const ConvParams& p) {
+    return 1024 + (size_t)p.a_stages * p.MH * p.a_box_rows * 128 + (size_t)p.b_stages * p.BN * 128 + 512;
+}
+
+// tile cursor shared by the roles (m fastest, then n tile, group, split)
+struct ConvCursor {
+    int m_tile, rest, n_tile, g, z;
+    __device__ __forceinline__ void decode(const ConvParams& q) {
+        int r = rest;
+        n_tile = r % q.n_tiles; r /= q.n_tiles;
+        g = r % q.groups;
+        z = r / q.groups;
+    }
+    __device__ __forceinline__ void init(const ConvParams& q) {
+        m_tile = blockIdx.x % q.m_tiles; rest = blockIdx.x / q.m_tiles; decode(q);
+    }
+    __device__ __forceinline__ void next(const ConvParams& q) {
+        m_tile += gridDim.x;
+        if (m_tile >= q.m_tiles) {
+            do { m_tile -= q.m_tiles; ++rest; } while (m_tile >= q.m_tiles);
+            decode(q);
+        }
+    }
+};
+
+__global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_constant__ ConvParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const int MH = p.MH, BN = p.BN;
+    const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * 128u, a_bytes = a_box_bytes * MH, b_bytes = (uint32_t)BN * 128u;
+    const int a_stages = p.a_stages, b_stages = p.b_stages;
+    const uint32_t ring_a = base, ring_b = base + a_stages * a_bytes;
+    // barriers: fullA[8] @0, emptyA[8] @64, fullB[8] @128, emptyB[8] @192, acc_full[2] @256, acc_empty[2] @272,
+    // tmem slot @288, abort flag @296
+    const uint32_t bar_base = ring_b + b_stages * b_bytes;
+    uint8_t* gen = smem_raw + (bar_base - raw);
+    volatile int* abort_flag = (volatile int*)(gen + 296);
+    volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 288);
+    const uint32_t fullA = bar_base, emptyA = bar_base + 64u, fullB = bar_base + 128u, emptyB = bar_base + 192u;
+    const uint32_t accf0 = bar_base + 256u, acce0 = bar_base + 272u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int acc_stages = p.acc_stages, acc_cols = MH * BN;
+    uint32_t ncols = 32;
+    while ((int)ncols < acc_stages * acc_cols) ncols <<= 1;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < a_stages; ++s) { mbar_init(fullA + 8u * s, 1); mbar_init(emptyA + 8u * s, MH); }
+        for (int s = 0; s < b_stages; ++s) { mbar_init(fullB + 8u * s, 1); mbar_init(emptyB + 8u * s, MH); }
+        for (int s = 0; s < 2; ++s) { mbar_init(accf0 + 8u * s, MH); mbar_init(acce0 + 8u * s, 128); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&p.tmA);
+        tma_prefetch_desc(&p.tmB);
+    }
+    if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), ncols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    const int per = p.asteps_per_split, kw = p.kw;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            ConvCursor tc; tc.init(p);
+            int sa = 0, sb = 0; uint32_t pha = 0, phb = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
+                const int m0 = tc.m_tile * (128 * MH), n0 = tc.n_tile * BN;
+                const int a_begin = tc.z * per;
+                const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
+                int ky = 0, ch = a_begin;
+                if (p.chunks < p.asteps_total && a_begin > 0) { ky = a_begin / p.chunks; ch = a_begin - ky * p.chunks; }
+                const int xa = p.a_x0 + tc.g * p.a_gx, yb = tc.g * p.b_g_rows + n0;
+                for (int i = 0; i < nsteps && ok; ++i) {
+                    if (!(ok = mbar_wait(emptyA + 8u * sa, pha ^ 1u, abort_flag))) break;
+                    {
+                        const uint32_t dst = ring_a + sa * a_bytes, fb = fullA + 8u * sa;
+                        const int y = m0 + p.halo_shift[ky];
+                        mbar_expect_tx(fb, a_bytes);
+                        for (int h = 0; h < MH; ++h)
+                            tma_load_2d(dst + h * a_box_bytes, &p.tmA, xa + ch * 64, y + h * p.a_box_rows, fb);
+                    }
+                    if (++sa == a_stages) { sa = 0; pha ^= 1u; }
+                    int brow = ky * kw * p.b_tap_rows + yb;
+                    for (int kx = 0; kx < kw; ++kx, brow += p.b_tap_rows) {
+                        if (!(ok = mbar_wait(emptyB + 8u * sb, phb ^ 1u, abort_flag))) break;
+                        const uint32_t fb = fullB + 8u * sb;
+                        mbar_expect_tx(fb, b_bytes);
+                        tma_load_2d(ring_b + sb * b_bytes, &p.tmB, ch * 64, brow, fb);
+                        if (++sb == b_stages) { sb = 0; phb ^= 1u; }
+                    }
+                    if (++ch == p.chunks) { ch = 0; ++ky; }
+                }
+            }
+        }
+    } else if (warp <= MH) {
+        // ------------------------------------------------------------ MMA issuer of row half h
+        if (lane == 0) {
+            const int h = warp - 1;
+            const uint32_t idesc = instr_desc(BN, 0, 0);
+            const uint64_t dbase = smem_desc(0, 16, 1024);
+            const int kk = p.kk;
+            int sa = 0, sb = 0; uint32_t pha = 0, phb = 0;
+            int ab = 0; uint32_t aph = 0;
+            bool ok = true;
+            int z = blockIdx.x / (p.m_tiles * p.n_tiles * p.groups);     // only the split index matters here
+            int in_split = blockIdx.x - z * (p.m_tiles * p.n_tiles * p.groups);
+            const int tiles_per_split = p.m_tiles * p.n_tiles * p.groups;
+            for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x) {
+                const int a_begin = z * per;
+                const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
+                if (!(ok = mbar_wait(acce0 + 8u * ab, aph ^ 1u, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t d = tmem + (uint32_t)(ab * acc_cols + h * BN);
+                uint32_t accum = 0;
+                for (int i = 0; i < nsteps && ok; ++i) {
+                    if (!(ok = mbar_wait(fullA + 8u * sa, pha, abort_flag))) break;
+                    const uint32_t a_half = ring_a + sa * a_bytes + (uint32_t)h * 16384u;
+                    for (int kx = 0; kx < kw; ++kx) {
+                        if (!(ok = mbar_wait(fullB + 8u * sb, phb, abort_flag))) break;
+                        tc_fence_after();
+                        const uint64_t bd = dbase + (uint64_t)((ring_b + sb * b_bytes) >> 4);
+                        const uint64_t ad = dbase + (uint64_t)((a_half + (uint32_t)p.tap_off[kx] * 128u) >> 4);
+                        #pragma unroll 4
+                        for (int j = 0; j < kk; ++j)
+                            umma(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), idesc, accum | (uint32_t)j);
+                        accum = 1;
+                        umma_commit(emptyB + 8u * sb);
+                        if (++sb == b_stages) { sb = 0; phb ^= 1u; }
+                    }
+                    if (!ok) break;
+                    umma_commit(emptyA + 8u * sa);
+                    if (++sa == a_stages) { sa = 0; pha ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(accf0 + 8u * ab);
+                if (++ab == acc_stages) { ab = 0; aph ^= 1u; }
+                in_split += gridDim.x;
+                while (in_split >= tiles_per_split) { in_split -= tiles_per_split; ++z; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;          // row within a 128-row half = TMEM lane
+        ConvCursor tc; tc.init(p);
+        int ab = 0; uint32_t aph = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
+            const int m0 = tc.m_tile * (128 * MH), n0 = tc.n_tile * BN, g = tc.g;
+            const int a_begin = tc.z * per;
+            const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
+            if (!(ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag))) break;
+            tc_fence_after();
+            #pragma unroll 1
+            for (int h = 0; h < MH; ++h) {
+                const int row = m0 + h * 128 + r;
+                const bool row_ok = row < p.M_total;
+                bool pad_row = false;
+                if (p.Hp > 0) {
+                    const int x = row % p.Wp, y = (row / p.Wp) % p.Hp;
+                    pad_row = (x >= p.W) || (y >= p.H);
+                }
+                const long long row_off = (long long)tc.z * p.split_stride + (long long)row * p.ldo + g * p.out_gx;
+                const uint32_t t0 = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * acc_cols + h * BN);
+                for (int c = 0; c < BN; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(t0 + (uint32_t)c, v);
+                    tmem_ld_wait();
+                    if (!row_ok) continue;
+                    epi_chunk(p, v, nsteps <= 0, pad_row, row_off, n0 + c, g);
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acce0 + 8u * ab);
+            if (++ab == acc_stages) { ab = 0; aph ^= 1u; }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
         if (threadIdx.x == 0 && p.status) atomicExch(p.status, 1);
         long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) { }
