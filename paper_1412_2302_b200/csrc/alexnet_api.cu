@@ -98,7 +98,7 @@ Layout make_layout() {
 const long long kCanonCount = 60965224;
 
 // ------------------------------------------------------------------- handle
-struct Plan { tc::GemmParams p; tc::ConvParams c; bool conv; int grid; size_t smem; bool valid; };
+struct Plan { tc::GemmParams p; tc::ConvParams c; tc::WgradParams w; bool conv, wgrad; int grid; size_t smem; bool valid; };
 
 struct Tensor {  // description of one exportable device tensor
     void* ptr; int kind; int C, Hp, Wp, H, W; long long N;
@@ -167,11 +167,15 @@ int pick_splits(int tiles, int steps, int cap) {
     if (s < 1) s = 1;
     return s;
 }
-int conv_wg_splits(const ConvL& c, int B) {
+int conv_wg_splits(const ConvL& c, int B, int sm_count = 148) {
+    // one wave: (filter rows x 64-channel input blocks x 128-channel output blocks x groups) units times the row splits
     const long long M = (long long)B * c.gin.Hp * c.gin.Wp;
     const int steps = (int)((M + 63) / 64);
-    const int tiles = ((c.cog + 127) / 128) * c.groups * c.taps;
-    return pick_splits(tiles, steps, 16);
+    const int units = ((c.cog + 127) / 128) * ((c.cig + 63) / 64) * c.groups * c.k;
+    int s = sm_count / units;
+    if (s > steps) s = steps;
+    if (s < 1) s = 1;
+    return s;
 }
 int fc_fwd_bn(const FcL&) { return 128; }
 int fc_fwd_splits(const FcL& f, int B) {
@@ -380,21 +384,30 @@ int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf1
 }
 int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16* xin) {
     memset(&P, 0, sizeof(P));
-    tc::GemmParams& p = P.p;
+    tc::WgradParams& p = P.w;
     const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
-    p.mode = tc::MODE_MNMN; p.epi = tc::EPI_F32;
-    p.M_total = c.cog; p.m_tiles = (c.cog + 127) / 128; p.BN = c.cig; p.n_tiles = 1;
-    p.groups = c.groups; p.taps_grid = c.taps; p.steps_total = (int)((M + 63) / 64);
-    p.splits = conv_wg_splits(c, h->B); p.kk = 4; p.chunks = 1;
+    p.m_tiles = (c.cog + 127) / 128; p.n_tiles = (c.cig + 63) / 64; p.groups = c.groups; p.kh = c.k; p.kw = c.k;
+    p.steps_total = (int)((M + 63) / 64);
+    p.splits = conv_wg_splits(c, h->B, std::min(h->sm_count, 148));   // never more than the workspace was sized for
+    p.steps_per_split = (p.steps_total + p.splits - 1) / p.splits;
+    p.splits = (p.steps_total + p.steps_per_split - 1) / p.steps_per_split;
+    p.tiles_total = p.m_tiles * p.n_tiles * p.groups * p.kh * p.splits;
+    if (c.k <= 4) { p.NI = 1; p.acc_kx0[0] = 0; p.acc_taps[0] = c.k; }
+    else { p.NI = 2; p.acc_kx0[0] = 0; p.acc_taps[0] = 3; p.acc_kx0[1] = 3; p.acc_taps[1] = c.k - 3; }
+    p.stages = std::min(8, (int)((227 * 1024 - 2048) / (tc::kWgABytes + tc::kWgBBytes)));
     p.a_gx = c.cog; p.b_gx = c.cig;
-    for (int t = 0; t < c.taps; ++t) p.shift[t] = c.shift[t];
-    p.n_valid = c.cig; p.ldo = c.cig; p.out_gx = c.cog;
+    for (int ky = 0; ky < c.k; ++ky) p.halo_shift[ky] = (ky - c.pad) * c.gin.Wp - c.pad;
+    p.M_total = c.cog; p.n_valid = c.cig; p.ldo = c.cig; p.out_gx = c.cog;
     p.tap_stride = (long long)c.cout * c.cig; p.split_stride = (long long)c.taps * c.cout * c.cig;
+    p.epi = tc::EPI_F32; p.mask_scale = 1.f;
     p.out = h->ws; p.status = h->status;
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, 64))) return rc;
-    if ((rc = make_tm(h, &p.tmB, xin, c.cin, M, (uint64_t)c.cin * 2, 64))) return rc;
-    finish_plan(h, P);
+    if ((rc = make_tm(h, &p.tmB, xin, c.cin, M, (uint64_t)c.cin * 2, 72))) return rc;
+    P.wgrad = true;
+    P.smem = tc::wgrad_smem_bytes(p);
+    P.grid = p.tiles_total;
+    P.valid = true;
     return ALEXNET_OK;
 }
 int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* wsh) {
@@ -489,7 +502,8 @@ void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
         }
     }
     if (h->prof) cudaEventRecord(h->prof_ev[h->prof_used], st);
-    if (P.conv) tc::conv_kernel<<<P.grid, tc::conv_threads(P.c), P.smem, st>>>(P.c);
+    if (P.wgrad) tc::wgrad_kernel<<<P.grid, tc::wgrad_threads(P.w), P.smem, st>>>(P.w);
+    else if (P.conv) tc::conv_kernel<<<P.grid, tc::conv_threads(P.c), P.smem, st>>>(P.c);
     else tc::gemm_kernel<<<P.grid, tc::kThreads, P.smem, st>>>(P.p);
     if (h->prof) { cudaEventRecord(h->prof_ev[h->prof_used + 1], st); h->prof_used += 2; }
     h->launches++;
@@ -524,7 +538,7 @@ void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
     const Plan& P = R.conv_wg[l][slot];
     launch_gemm(h, P, st);
     const long long total = (long long)c.taps * c.cout * c.cig;
-    kn::wgrad_reduce_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, total, R.g + c.w_off, l == 0);
+    kn::wgrad_reduce_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.w.splits, P.w.split_stride, total, R.g + c.w_off, l == 0);
     h->launches++;
     bf16* dyv[5] = {R.da1, R.da2, R.da3, R.da4, R.da5};
     colsum(h, dyv[l], (long long)h->B * c.gout.Hp * c.gout.Wp, c.cout, R.g + c.b_off, st);
@@ -566,7 +580,8 @@ void op_lrn_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
     const Grid& g = h->L.conv[which].gout;
     const long long rows = (long long)h->B * g.Hp * g.Wp;
-    kn::lrn_fwd_kernel<<<nblk(rows * (g.C / 8), 256), 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.n2 : R.n1, rows, g.C,
+    kn::lrn_fwd_kernel<<<nblk(rows * (g.C / 8), 256), 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.n2 : R.n1,
+                                                                   (unsigned)(rows * (g.C / 8)), (unsigned)(g.C / 8),
                                                                    h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
     h->launches++;
 }
@@ -575,8 +590,8 @@ void op_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     const Grid& g = h->L.conv[which].gout;
     const long long rows = (long long)h->B * g.Hp * g.Wp;
     kn::lrn_bwd_kernel<<<nblk(rows * (g.C / 8), 256), 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.dn2 : R.dn1,
-                                                                   which ? R.da2 : R.da1, rows, g.C, h->alpha_eff,
-                                                                   h->cfg.lrn_beta, h->cfg.lrn_k);
+                                                                   which ? R.da2 : R.da1, (unsigned)(rows * (g.C / 8)),
+                                                                   (unsigned)(g.C / 8), h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
     h->launches++;
 }
 struct PoolGeo { int C, Hpi, Wpi, Hi, Wi, Ho, Wo, Hpo, Wpo; };
@@ -587,8 +602,8 @@ void op_pool_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     const bf16* x[3] = {R.n1, R.n2, R.a5};
     bf16* y[3] = {R.p1, R.p2, R.p5};
     uint8_t* a[3] = {R.arg1, R.arg2, R.arg5};
-    const long long total = (long long)h->B * g.Ho * g.Wo * (g.C / 8);
-    kn::pool_fwd_kernel<<<nblk(total, 256), 256, 0, st>>>(x[which], y[which], a[which], h->B, g.C, g.Hpi, g.Wpi, g.Ho, g.Wo, g.Hpo, g.Wpo);
+    const dim3 grid(nblk((long long)g.Wo * (g.C / 8), 256), g.Ho, h->B);
+    kn::pool_fwd_kernel<<<grid, 256, 0, st>>>(x[which], y[which], a[which], g.C / 8, g.Hpi, g.Wpi, g.Ho, g.Wo, g.Hpo, g.Wpo);
     h->launches++;
 }
 void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
@@ -598,9 +613,9 @@ void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     const uint8_t* a[3] = {R.arg1, R.arg2, R.arg5};
     const bf16* relu[3] = {nullptr, nullptr, R.a5};
     bf16* dx[3] = {R.dn1, R.dn2, R.da5};
-    const long long total = (long long)h->B * g.Hpi * g.Wpi * (g.C / 8);
-    kn::pool_bwd_kernel<<<nblk(total, 256), 256, 0, st>>>(dy[which], a[which], relu[which], dx[which], h->B, g.C, g.Hpi, g.Wpi,
-                                                          g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo, g.Wpo);
+    const dim3 grid(nblk((long long)g.Wpi * (g.C / 8), 256), g.Hpi, h->B);
+    kn::pool_bwd_kernel<<<grid, 256, 0, st>>>(dy[which], a[which], relu[which], dx[which], g.C / 8, g.Hpi, g.Wpi,
+                                              g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo, g.Wpo);
     h->launches++;
 }
 void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
@@ -793,6 +808,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     h->encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
     CKC(cudaFuncSetAttribute(tc::gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CKC(cudaFuncSetAttribute(tc::wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     {
         int dev = 0;
         CKC(cudaGetDevice(&dev));

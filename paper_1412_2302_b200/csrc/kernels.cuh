@@ -80,68 +80,78 @@ __global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* 
 }
 
 // ----------------------------------------------------------------------- LRN
-__device__ __forceinline__ float pow_neg(float s, float beta) {
-    if (beta == 0.75f) { float r = rsqrtf(s); return r * sqrtf(r); }
-    return exp2f(-beta * log2f(s));
+// All index arithmetic below is 32-bit: the largest activation tensor of a batch of 1024 has
+// 1024*57*57*12 < 2^31 sixteen-byte vectors.
+__device__ __forceinline__ float rsqrt_fast(float x) { float y; asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float sqrt_fast(float x) { float y; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+// s^-beta and 1/s; the exponent 0.75 of the paper's network costs two special-function instructions
+__device__ __forceinline__ void pow_neg(float s, float beta, float& sp, float& rs) {
+    if (beta == 0.75f) { const float r = rsqrt_fast(s); sp = r * sqrt_fast(r); rs = r * r; }
+    else { sp = exp2f(-beta * __log2f(s)); rs = __fdividef(1.f, s); }
 }
 // b_c = a_c * (k + alpha * sum_{c' in [c-2,c+2] clipped} a_c'^2)^(-beta); one thread = 8 channels of one pixel.
-__global__ void lrn_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ b,
-                               long long rows, int C, float alpha, float beta, float k) {
-    const int cpr = C >> 3;
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= rows * cpr) return;
-    const int ch = (int)(t % cpr);
+__global__ void __launch_bounds__(256) lrn_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ b,
+                                                      unsigned total, unsigned cpr, float alpha, float beta, float k) {
+    const unsigned t = blockIdx.x * 256u + threadIdx.x;
+    if (t >= total) return;
+    const unsigned ch = t % cpr;
     const uint4* ap = (const uint4*)a + t;
     const uint4 zero = make_uint4(0, 0, 0, 0);
     float f[24];
-    unpack8(ch > 0 ? ap[-1] : zero, f);
-    unpack8(ap[0], f + 8);
-    unpack8(ch < cpr - 1 ? ap[1] : zero, f + 16);
+    unpack8(ch > 0 ? __ldg(ap - 1) : zero, f);
+    unpack8(__ldg(ap), f + 8);
+    unpack8(ch < cpr - 1 ? __ldg(ap + 1) : zero, f + 16);
+    float sq[12];
+    #pragma unroll
+    for (int i = 0; i < 12; ++i) sq[i] = f[6 + i] * f[6 + i];
     float o[8];
     #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        float ss = 0.f;
-        #pragma unroll
-        for (int j = -2; j <= 2; ++j) ss += f[8 + i + j] * f[8 + i + j];
-        o[i] = f[8 + i] * pow_neg(k + alpha * ss, beta);
+        const float ss = (sq[i] + sq[i + 1]) + (sq[i + 2] + sq[i + 3]) + sq[i + 4];
+        float sp, rs;
+        pow_neg(fmaf(alpha, ss, k), beta, sp, rs);
+        o[i] = f[8 + i] * sp;
     }
     ((uint4*)b)[t] = pack8(o);
 }
 // da_m = [a_m > 0] * ( g_m s_m^-beta - 2 alpha beta a_m sum_{c in [m-2,m+2]} g_c a_c s_c^(-beta-1) )
-// (the ReLU mask of the convolution that produced a is applied here).
-__global__ void lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ g,
-                               __nv_bfloat16* __restrict__ da, long long rows, int C, float alpha, float beta, float k) {
-    const int cpr = C >> 3;
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= rows * cpr) return;
-    const int ch = (int)(t % cpr);
+// (the ReLU mask of the convolution that produced a is applied here).  One thread = 8 channels of one
+// pixel; it needs s for the 12 channels c0-2 .. c0+9 and a for c0-4 .. c0+11.
+__global__ void __launch_bounds__(256) lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ g,
+                                                      __nv_bfloat16* __restrict__ da, unsigned total, unsigned cpr,
+                                                      float alpha, float beta, float k) {
+    const unsigned t = blockIdx.x * 256u + threadIdx.x;
+    if (t >= total) return;
+    const unsigned ch = t % cpr;
     const uint4* ap = (const uint4*)a + t;
     const uint4* gp = (const uint4*)g + t;
     const uint4 zero = make_uint4(0, 0, 0, 0);
+    const bool has_l = ch > 0, has_r = ch < cpr - 1;
     float fa[24], fg[24];
-    unpack8(ch > 0 ? ap[-1] : zero, fa);
-    unpack8(ap[0], fa + 8);
-    unpack8(ch < cpr - 1 ? ap[1] : zero, fa + 16);
-    unpack8(ch > 0 ? gp[-1] : zero, fg);
-    unpack8(gp[0], fg + 8);
-    unpack8(ch < cpr - 1 ? gp[1] : zero, fg + 16);
+    unpack8(has_l ? __ldg(ap - 1) : zero, fa);
+    unpack8(__ldg(ap), fa + 8);
+    unpack8(has_r ? __ldg(ap + 1) : zero, fa + 16);
+    unpack8(has_l ? __ldg(gp - 1) : zero, fg);
+    unpack8(__ldg(gp), fg + 8);
+    unpack8(has_r ? __ldg(gp + 1) : zero, fg + 16);
+    float sq[16];
+    #pragma unroll
+    for (int i = 0; i < 16; ++i) sq[i] = fa[4 + i] * fa[4 + i];
     float sp[12], tt[12];   // channels c0-2 .. c0+9
     #pragma unroll
     for (int i = 0; i < 12; ++i) {
-        const int c = 6 + i;
-        float ss = 0.f;
-        #pragma unroll
-        for (int j = -2; j <= 2; ++j) ss += fa[c + j] * fa[c + j];
-        const float s = k + alpha * ss;
-        sp[i] = pow_neg(s, beta);
-        tt[i] = fg[c] * fa[c] * sp[i] / s;
+        const float ss = (sq[i] + sq[i + 1]) + (sq[i + 2] + sq[i + 3]) + sq[i + 4];
+        float rs;
+        pow_neg(fmaf(alpha, ss, k), beta, sp[i], rs);
+        tt[i] = fg[6 + i] * fa[6 + i] * sp[i] * rs;
     }
+    const float c2 = 2.f * alpha * beta;
     float o[8];
     #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const float acc = tt[i] + tt[i + 1] + tt[i + 2] + tt[i + 3] + tt[i + 4];
+        const float acc = (tt[i] + tt[i + 1]) + (tt[i + 2] + tt[i + 3]) + tt[i + 4];
         const float am = fa[8 + i];
-        const float v = fg[8 + i] * sp[i + 2] - 2.f * alpha * beta * am * acc;
+        const float v = fmaf(fg[8 + i], sp[i + 2], -c2 * am * acc);
         o[i] = am > 0.f ? v : 0.f;
     }
     ((uint4*)da)[t] = pack8(o);
@@ -149,68 +159,65 @@ __global__ void lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_b
 
 // ------------------------------------------------------------------ max pool
 // 3x3 stride 2, no padding; first maximum in (ky,kx) row-major order wins; argmax = ky*3+kx.
-__global__ void pool_fwd_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
-                                uint8_t* __restrict__ arg, int B, int C, int Hpi, int Wpi,
-                                int Ho, int Wo, int Hpo, int Wpo) {
-    const int cpr = C >> 3;
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= (long long)B * Ho * Wo * cpr) return;
-    const int ch = (int)(t % cpr);
-    long long r = t / cpr;
-    const int ox = (int)(r % Wo); r /= Wo;
-    const int oy = (int)(r % Ho);
-    const int n = (int)(r / Ho);
+// grid: (ceil(Wo*cpr / 256), Ho, B); one thread = 8 channels of one output pixel.
+__global__ void __launch_bounds__(256) pool_fwd_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
+                                                       uint8_t* __restrict__ arg, int cpr, int Hpi, int Wpi,
+                                                       int Ho, int Wo, int Hpo, int Wpo) {
+    const unsigned i = blockIdx.x * 256u + threadIdx.x;
+    if (i >= (unsigned)(Wo * cpr)) return;
+    const int ox = i / cpr, ch = i - ox * cpr;
+    const int oy = blockIdx.y, n = blockIdx.z;
     float best[8]; int bi[8];
+    const uint4* xp = (const uint4*)x + ((size_t)(n * Hpi + 2 * oy) * Wpi + 2 * ox) * cpr + ch;
     #pragma unroll
     for (int ky = 0; ky < 3; ++ky)
         #pragma unroll
         for (int kx = 0; kx < 3; ++kx) {
-            const uint4 u = ((const uint4*)x)[((size_t)(n * Hpi + 2 * oy + ky) * Wpi + 2 * ox + kx) * cpr + ch];
             float f[8];
-            unpack8(u, f);
+            unpack8(__ldg(xp + (ky * Wpi + kx) * cpr), f);
             #pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if ((ky == 0 && kx == 0) || f[i] > best[i]) { best[i] = f[i]; bi[i] = ky * 3 + kx; }
+            for (int q = 0; q < 8; ++q)
+                if ((ky == 0 && kx == 0) || f[q] > best[q]) { best[q] = f[q]; bi[q] = ky * 3 + kx; }
         }
     ((uint4*)y)[((size_t)(n * Hpo + oy) * Wpo + ox) * cpr + ch] = pack8(best);
     uint2 ab;
     ab.x = bi[0] | (bi[1] << 8) | (bi[2] << 16) | (bi[3] << 24);
     ab.y = bi[4] | (bi[5] << 8) | (bi[6] << 16) | (bi[7] << 24);
-    ((uint2*)arg)[t] = ab;
+    ((uint2*)arg)[((size_t)(n * Ho + oy) * Wo + ox) * cpr + ch] = ab;
 }
 // dx[y][x] = sum over the (up to 4) windows containing (y,x) whose argmax points at it; optional ReLU mask.
-__global__ void pool_bwd_kernel(const __nv_bfloat16* __restrict__ dy, const uint8_t* __restrict__ arg,
-                                const __nv_bfloat16* __restrict__ relu_src, __nv_bfloat16* __restrict__ dx,
-                                int B, int C, int Hpi, int Wpi, int Hi, int Wi, int Ho, int Wo, int Hpo, int Wpo) {
-    const int cpr = C >> 3;
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= (long long)B * Hpi * Wpi * cpr) return;
-    const int ch = (int)(t % cpr);
-    long long r = t / cpr;
-    const int x = (int)(r % Wpi); r /= Wpi;
-    const int y = (int)(r % Hpi);
-    const int n = (int)(r / Hpi);
+// grid: (ceil(Wpi*cpr / 256), Hpi, B); one thread = 8 channels of one input pixel (pad pixels get zero).
+__global__ void __launch_bounds__(256) pool_bwd_kernel(const __nv_bfloat16* __restrict__ dy, const uint8_t* __restrict__ arg,
+                                                       const __nv_bfloat16* __restrict__ relu_src, __nv_bfloat16* __restrict__ dx,
+                                                       int cpr, int Hpi, int Wpi, int Hi, int Wi, int Ho, int Wo, int Hpo, int Wpo) {
+    const unsigned i = blockIdx.x * 256u + threadIdx.x;
+    if (i >= (unsigned)(Wpi * cpr)) return;
+    const int x = i / cpr, ch = i - x * cpr;
+    const int y = blockIdx.y, n = blockIdx.z;
+    const size_t t = ((size_t)(n * Hpi + y) * Wpi + x) * cpr + ch;
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (y < Hi && x < Wi) {
         const int oy_lo = max(0, (y - 1) >> 1), oy_hi = min(Ho - 1, y >> 1);
         const int ox_lo = max(0, (x - 1) >> 1), ox_hi = min(Wo - 1, x >> 1);
         for (int oy = oy_lo; oy <= oy_hi; ++oy)
             for (int ox = ox_lo; ox <= ox_hi; ++ox) {
-                const int code = (y - 2 * oy) * 3 + (x - 2 * ox);
-                const uint2 ab = ((const uint2*)arg)[((size_t)(n * Ho + oy) * Wo + ox) * cpr + ch];
+                const unsigned code = (unsigned)((y - 2 * oy) * 3 + (x - 2 * ox)) * 0x01010101u;
+                const uint2 ab = __ldg((const uint2*)arg + ((size_t)(n * Ho + oy) * Wo + ox) * cpr + ch);
                 float f[8];
-                unpack8(((const uint4*)dy)[((size_t)(n * Hpo + oy) * Wpo + ox) * cpr + ch], f);
+                unpack8(__ldg((const uint4*)dy + ((size_t)(n * Hpo + oy) * Wpo + ox) * cpr + ch), f);
+                // byte-wise equality of the eight argmax codes with this pixel's code
+                const unsigned e0 = ab.x ^ code, e1 = ab.y ^ code;
                 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int a = (int)(((i < 4 ? ab.x : ab.y) >> (8 * (i & 3))) & 0xFF);
-                    if (a == code) acc[i] += f[i];
+                for (int q = 0; q < 4; ++q) {
+                    if (((e0 >> (8 * q)) & 0xFFu) == 0u) acc[q] += f[q];
+                    if (((e1 >> (8 * q)) & 0xFFu) == 0u) acc[q + 4] += f[q + 4];
                 }
             }
         if (relu_src) {
             float m[8];
-            unpack8(((const uint4*)relu_src)[t], m);
+            unpack8(__ldg((const uint4*)relu_src + t), m);
             #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = m[i] > 0.f ? acc[i] : 0.f;
+            for (int q = 0; q < 8; ++q) acc[q] = m[q] > 0.f ? acc[q] : 0.f;
         }
     }
     ((uint4*)dx)[t] = pack8(acc);

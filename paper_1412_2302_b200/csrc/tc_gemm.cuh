@@ -666,4 +666,158 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     }
 }
 
+// ===========================================================================
+// Convolution weight-gradient kernel.
+//
+//   dW[ky][kx][co][ci] = sum_m dy[m][co] * x[m + shift(ky,kx)][ci]
+//
+// Both operands are MN-major (the reduction runs over the rows m of the flat
+// grid).  One CTA owns one filter row ky, one block of 128 output channels, one
+// block of 64 input channels and one range of rows; per 64-row step it loads
+// the dy tile (two 64 x 64 boxes) and ONE halo of x rows (72 rows x 64
+// channels).  The kw taps of the filter row are the same halo shifted by whole
+// rows, so they are fed to the tensor core as consecutive 64-wide N blocks of a
+// single instruction: the B descriptor's leading-dimension offset is one row
+// (128 bytes), which makes N block j read the halo from row j on.  One
+// instruction therefore covers up to four taps (N = 64 * taps <= 256); a
+// five-tap row takes two accumulators with an issuer warp each.
+// Each CTA writes fp32 partial sums [split][tap][co][ci]; a reduction kernel
+// adds the splits in a fixed order.
+// Warps: 0 = TMA producer, 1..NI = MMA issuers, NI+1..NI+4 = epilogue.
+struct WgradParams {
+    CUtensorMap tmA, tmB;       // dy [M][cout] box {64, 64}; x [M][cin] box {64, 72}
+    int m_tiles, n_tiles, groups, kh, splits;   // tile decomposition (m fastest, then n, group, ky, split)
+    int tiles_total;
+    int kw;                     // taps per filter row
+    int NI;                     // accumulators = issuers (1 or 2)
+    int acc_kx0[2], acc_taps[2];  // first tap and tap count of each accumulator
+    int steps_total, steps_per_split, stages;
+    int a_gx, b_gx;             // per-group column strides of dy and x
+    int halo_shift[5];          // per ky: first halo row relative to the dy row
+    // output
+    int M_total;                // valid output channels per group
+    int n_valid;                // valid input channels per group
+    int ldo, out_gx;            // row pitch (= input channels per group), per-group row offset
+    long long split_stride, tap_stride;
+    int epi, relu; float mask_scale; const float* bias; const __nv_bfloat16* mask;   // fixed: EPI_F32, unused
+    void* out;
+    int* status;
+};
+constexpr int kWgABytes = 16384, kWgBBytes = 72 * 128;
+inline int wgrad_threads(const WgradParams& p) { return 32 * (5 + p.NI); }
+inline size_t wgrad_smem_bytes(const WgradParams& p) { return 1024 + (size_t)p.stages * (kWgABytes + kWgBBytes) + 256; }
+
+__global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant__ WgradParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const int stages = p.stages, NI = p.NI;
+    constexpr uint32_t stage_bytes = kWgABytes + kWgBBytes;
+    // barriers: full[8] @0, empty[8] @64, acc_full @128, tmem slot @136, abort flag @144
+    const uint32_t bar_base = base + stages * stage_bytes;
+    uint8_t* gen = smem_raw + (bar_base - raw);
+    volatile int* abort_flag = (volatile int*)(gen + 144);
+    volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 136);
+    const uint32_t full0 = bar_base, empty0 = bar_base + 64u, accf = bar_base + 128u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int acc_cols = 64 * p.kw;
+    uint32_t ncols = 32;
+    while ((int)ncols < acc_cols) ncols <<= 1;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < stages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, NI); }
+        mbar_init(accf, NI);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&p.tmA);
+        tma_prefetch_desc(&p.tmB);
+    }
+    if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), ncols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    // this CTA's tile (one per CTA: the grid equals the tile count)
+    int r = blockIdx.x;
+    const int m_tile = r % p.m_tiles; r /= p.m_tiles;
+    const int n_tile = r % p.n_tiles; r /= p.n_tiles;
+    const int g = r % p.groups; r /= p.groups;
+    const int ky = r % p.kh;
+    const int z = r / p.kh;
+    const int s_begin = z * p.steps_per_split;
+    const int nsteps = min(p.steps_total, s_begin + p.steps_per_split) - s_begin;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const int xa = g * p.a_gx + m_tile * 128, xb = g * p.b_gx + n_tile * 64, sh = p.halo_shift[ky];
+            int st = 0; uint32_t ph = 0;
+            for (int i = 0; i < nsteps; ++i) {
+                if (!mbar_wait(empty0 + 8u * st, ph ^ 1u, abort_flag)) break;
+                const uint32_t sa = base + st * stage_bytes, fb = full0 + 8u * st;
+                const int q = (s_begin + i) * 64;
+                mbar_expect_tx(fb, stage_bytes);
+                tma_load_2d(sa, &p.tmA, xa, q, fb);
+                tma_load_2d(sa + 8192, &p.tmA, xa + 64, q, fb);
+                tma_load_2d(sa + kWgABytes, &p.tmB, xb, q + sh, fb);
+                if (++st == stages) { st = 0; ph ^= 1u; }
+            }
+        }
+    } else if (warp <= NI) {
+        if (lane == 0) {
+            const int a = warp - 1;
+            const int taps = p.acc_taps[a], kx0 = p.acc_kx0[a];
+            const uint32_t idesc = instr_desc(64 * taps, 1, 1);
+            const uint64_t adesc0 = smem_desc(0, 8192, 1024), bdesc0 = smem_desc(0, 128, 1024);
+            const uint32_t d = tmem + (uint32_t)(kx0 * 64);
+            int st = 0; uint32_t ph = 0;
+            bool ok = true;
+            for (int i = 0; i < nsteps; ++i) {
+                if (!(ok = mbar_wait(full0 + 8u * st, ph, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t sa = base + st * stage_bytes;
+                const uint64_t ad = adesc0 + (uint64_t)(sa >> 4);
+                const uint64_t bd = bdesc0 + (uint64_t)((sa + kWgABytes + (uint32_t)kx0 * 128u) >> 4);
+                #pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    umma(d, ad + (uint64_t)(128 * j), bd + (uint64_t)(128 * j), idesc, (i > 0 || j > 0) ? 1u : 0u);
+                umma_commit(empty0 + 8u * st);
+                if (++st == stages) { st = 0; ph ^= 1u; }
+            }
+            if (ok) umma_commit(accf);
+        }
+    } else {
+        const int quad = warp & 3;
+        const int row = m_tile * 128 + quad * 32 + lane;     // output channel within the group
+        const bool row_ok = row < p.M_total;
+        if (mbar_wait(accf, 0, abort_flag)) {
+            tc_fence_after();
+            const uint32_t t0 = tmem + ((uint32_t)(quad * 32) << 16);
+            for (int kx = 0; kx < p.kw; ++kx) {
+                const long long row_off = (long long)z * p.split_stride + (long long)(ky * p.kw + kx) * p.tap_stride +
+                                          (long long)(g * p.out_gx + row) * p.ldo;
+                for (int c = 0; c < 64; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(t0 + (uint32_t)(kx * 64 + c), v);
+                    tmem_ld_wait();
+                    if (!row_ok) continue;
+                    epi_chunk(p, v, nsteps <= 0, false, row_off, n_tile * 64 + c, g);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && p.status) atomicExch(p.status, 1);
+        long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) { }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem, ncols);
+    }
+}
+
 }  // namespace tc
