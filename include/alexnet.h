@@ -159,12 +159,15 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters);
 /* Number of kernels launched by this handle since creation (for accounting). */
 uint64_t alexnet_launch_count(const alexnet_t* h);
 
-/* Optional timing of the tensor-core GEMM kernel: while enabled, every launch
- * of it is bracketed by a CUDA event pair on its stream.  profile_read waits for
- * both streams, returns the summed device time (ms) and the number of launches
- * recorded since the last read, and clears the record. */
+/* Optional timing of the tensor-core kernels: while enabled, every launch of
+ * one is bracketed by a CUDA event pair on its stream.  profile_read waits for
+ * both streams, returns per kernel the summed device time (ms) and the number
+ * of launches recorded since the last read, and clears the record.  Index 0 =
+ * conv_kernel (convolution forward and backward-data, FC forward), 1 =
+ * wgrad_kernel (convolution weight gradients), 2 = gemm_kernel (FC
+ * backward-data and weight gradients).  Both arrays have three entries. */
 int alexnet_profile(alexnet_t* h, int enable);
-int alexnet_profile_read(alexnet_t* h, double* gemm_ms, uint64_t* gemm_launches);
+int alexnet_profile_read(alexnet_t* h, double* ms3, uint64_t* launches3);
 
 /* Bias gradient db[c] = sum over rows of dy[row][c], for callers that cannot
  * allocate device memory when they need it.  (The paper has no counterpart of

@@ -195,10 +195,11 @@ class AlexNet:
         self._ck(self.lib.alexnet_profile(self.h, 1 if enable else 0))
 
     def profile_read(self):
-        """(summed GEMM-kernel device time in ms, launches) since the last read."""
-        ms, n = ctypes.c_double(), ctypes.c_uint64()
-        self._ck(self.lib.alexnet_profile_read(self.h, ctypes.byref(ms), ctypes.byref(n)))
-        return ms.value, int(n.value)
+        """Per tensor-core kernel (conv_kernel, wgrad_kernel, gemm_kernel): summed device time in ms and
+        launches since the last read, as two 3-tuples."""
+        ms, n = (ctypes.c_double * 3)(), (ctypes.c_uint64 * 3)()
+        self._ck(self.lib.alexnet_profile_read(self.h, ms, n))
+        return tuple(ms), tuple(int(v) for v in n)
 
     @property
     def launch_count(self):

@@ -142,6 +142,7 @@ struct alexnet {
     // optional per-launch timing of the GEMM kernel (event pairs on the launching stream)
     bool prof;
     std::vector<cudaEvent_t> prof_ev;
+    std::vector<int> prof_kind;     // kernel of each recorded pair: 0 conv_kernel, 1 wgrad_kernel, 2 gemm_kernel
     size_t prof_used;
 };
 
@@ -263,10 +264,24 @@ int make_tm(alexnet* h, CUtensorMap* tm, const void* ptr, uint64_t cols, uint64_
     return ALEXNET_OK;
 }
 
+// output tensor map of the staged epilogue: {columns, rows, splits}, box = {128 bytes of columns, 32 rows, 1}
+int make_tm_out(alexnet* h, CUtensorMap* tm, const void* ptr, bool f32, uint64_t cols, uint64_t rows, uint64_t nz,
+                uint64_t row_pitch_bytes, uint64_t z_pitch_bytes) {
+    cuuint64_t dims[3] = {cols, rows, nz};
+    cuuint64_t strides[2] = {row_pitch_bytes, z_pitch_bytes};
+    cuuint32_t box[3] = {f32 ? 32u : 64u, 32u, 1u};
+    cuuint32_t es[3] = {1, 1, 1};
+    CUresult r = h->encode(tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)ptr, dims, strides,
+                           box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(h, ALEXNET_ERR_CUDA, "cuTensorMapEncodeTiled (output) failed with code " + std::to_string((int)r));
+    return ALEXNET_OK;
+}
+
 void finish_plan(const alexnet* h, Plan& P) {
     tc::GemmParams& p = P.p;
     const int stage_bytes = tc::kABytes + tc::b_stage_bytes(p.mode, p.BN);
-    int stages = (227 * 1024 - 2048) / stage_bytes;
+    int stages = (227 * 1024 - 2048 - 4 * (int)tc::kEpiStageBytes) / stage_bytes;
     if (stages > tc::kMaxStages) stages = tc::kMaxStages;
     p.stages = stages;
     // every split gets at least one k-step
@@ -288,7 +303,7 @@ ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, in
     ConvShape best{1, N <= 256 ? N : 128, 1};
     double best_t = 1e30;
     const int a_rows = kw > 1 ? 136 : 128;
-    const size_t budget = 227 * 1024 - 2048;
+    const size_t budget = 227 * 1024 - 2048 - 4 * tc::kEpiStageBytes;
     for (int MH = 1; MH <= 4; MH *= 2) {
         for (int BN = 16; BN <= 256 && BN <= N; BN += 16) {
             if (N % BN) continue;
@@ -317,7 +332,7 @@ void finish_conv_plan(const alexnet* h, Plan& P) {
     c.asteps_per_split = per;
     c.tiles_total = c.m_tiles * c.n_tiles * c.groups * c.splits;
     const size_t a_bytes = (size_t)c.MH * c.a_box_rows * 128, b_bytes = (size_t)c.BN * 128;
-    const size_t budget = 227 * 1024 - 2048;
+    const size_t budget = 227 * 1024 - 2048 - 4 * tc::kEpiStageBytes;
     if (c.kw == 1) {
         int st = (int)(budget / (a_bytes + b_bytes));
         st = std::min(st, 8);
@@ -331,6 +346,20 @@ void finish_conv_plan(const alexnet* h, Plan& P) {
     P.smem = tc::conv_smem_bytes(c);
     P.grid = std::min(c.tiles_total, h->sm_count);
     P.valid = true;
+}
+
+// bf16 convolution output through the staged epilogue when whole 64-column slabs tile the channel range of a
+// group, or when the tile ends at the tensor's last column (TMA clips the rest) and the over-read stays inside the
+// TMEM allocation; otherwise the epilogue stores rows directly
+int conv_out_map(alexnet* h, tc::ConvParams& p, const void* out, int ldo, long long M) {
+    const int used = p.acc_stages * p.MH * p.BN;
+    int alloc = 32;
+    while (alloc < used) alloc <<= 1;
+    const bool whole = p.BN % 64 == 0;
+    const bool clipped = p.groups == 1 && p.n_tiles == 1 && used - p.BN + (p.BN + 63) / 64 * 64 <= alloc;
+    p.tma_store = (whole || clipped) ? 1 : 0;
+    if (!p.tma_store) return ALEXNET_OK;
+    return make_tm_out(h, &p.tmOut, out, false, (uint64_t)ldo, (uint64_t)M, 1, (uint64_t)ldo * 2, (uint64_t)ldo * 2 * (uint64_t)M);
 }
 
 int plan_conv_fwd(alexnet* h, Plan& P, const ConvL& c, const bf16* in, const bf16* wsh, const float* bias, bf16* out) {
@@ -354,6 +383,7 @@ int plan_conv_fwd(alexnet* h, Plan& P, const ConvL& c, const bf16* in, const bf1
     int rc;
     if ((rc = make_tm(h, &p.tmA, in, c.cin, M, (uint64_t)c.cin * 2, p.a_box_rows))) return rc;
     if ((rc = make_tm(h, &p.tmB, wsh, c.cig, (uint64_t)c.taps * c.cout, (uint64_t)c.cig * 2, p.BN))) return rc;
+    if ((rc = conv_out_map(h, p, out, c.cout, M))) return rc;
     finish_conv_plan(h, P);
     return ALEXNET_OK;
 }
@@ -379,6 +409,7 @@ int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf1
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, p.a_box_rows))) return rc;
     if ((rc = make_tm(h, &p.tmB, wt, c.cog, (uint64_t)c.taps * c.cin, (uint64_t)c.cog * 2, p.BN))) return rc;
+    if ((rc = conv_out_map(h, p, dx, c.cin, M))) return rc;
     finish_conv_plan(h, P);
     return ALEXNET_OK;
 }
@@ -426,6 +457,9 @@ int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* ws
     int rc;
     if ((rc = make_tm(h, &p.tmA, x, f.K, B, (uint64_t)f.K * 2, 128))) return rc;
     if ((rc = make_tm(h, &p.tmB, wsh, f.K, f.N, (uint64_t)f.K * 2, p.BN))) return rc;
+    p.tma_store = 1;
+    if ((rc = make_tm_out(h, &p.tmOut, h->ws, true, (uint64_t)f.N, (uint64_t)B, (uint64_t)p.splits, (uint64_t)f.N * 4,
+                          (uint64_t)B * f.N * 4))) return rc;
     finish_conv_plan(h, P);
     return ALEXNET_OK;
 }
@@ -442,6 +476,9 @@ int plan_fc_bwd(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* w
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, f.N, B, (uint64_t)f.N * 2, 128))) return rc;
     if ((rc = make_tm(h, &p.tmB, wsh, f.K, f.N, (uint64_t)f.K * 2, 64))) return rc;
+    p.tma_store = 1;
+    if ((rc = make_tm_out(h, &p.tmOut, h->ws, true, (uint64_t)f.K, (uint64_t)B, (uint64_t)p.splits, (uint64_t)f.K * 4,
+                          (uint64_t)B * f.K * 4))) return rc;
     finish_plan(h, P);
     return ALEXNET_OK;
 }
@@ -457,6 +494,8 @@ int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x,
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, f.N, B, (uint64_t)f.N * 2, 64))) return rc;
     if ((rc = make_tm(h, &p.tmB, x, f.K, B, (uint64_t)f.K * 2, 64))) return rc;
+    p.tma_store = 1;
+    if ((rc = make_tm_out(h, &p.tmOut, gout, true, (uint64_t)f.K, (uint64_t)f.N, 1, (uint64_t)f.K * 4, (uint64_t)f.K * 4 * f.N))) return rc;
     finish_plan(h, P);
     return ALEXNET_OK;
 }
@@ -505,7 +544,11 @@ void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
     if (P.wgrad) tc::wgrad_kernel<<<P.grid, tc::wgrad_threads(P.w), P.smem, st>>>(P.w);
     else if (P.conv) tc::conv_kernel<<<P.grid, tc::conv_threads(P.c), P.smem, st>>>(P.c);
     else tc::gemm_kernel<<<P.grid, tc::kThreads, P.smem, st>>>(P.p);
-    if (h->prof) { cudaEventRecord(h->prof_ev[h->prof_used + 1], st); h->prof_used += 2; }
+    if (h->prof) {
+        cudaEventRecord(h->prof_ev[h->prof_used + 1], st);
+        h->prof_kind.push_back(P.conv ? 0 : P.wgrad ? 1 : 2);
+        h->prof_used += 2;
+    }
     h->launches++;
 }
 void colsum(alexnet* h, const bf16* dy, long long rows, int C, float* db, cudaStream_t st) {
@@ -1036,19 +1079,20 @@ int alexnet_profile(alexnet_t* h, int enable) {
     return ALEXNET_OK;
 }
 
-int alexnet_profile_read(alexnet_t* h, double* gemm_ms, uint64_t* gemm_launches) {
-    if (!h || !gemm_ms || !gemm_launches) return ALEXNET_ERR_ARG;
+int alexnet_profile_read(alexnet_t* h, double* ms3, uint64_t* launches3) {
+    if (!h || !ms3 || !launches3) return ALEXNET_ERR_ARG;
     CK(cudaStreamSynchronize(h->ls));
     CK(cudaStreamSynchronize(h->cs));
-    double ms = 0.0;
+    for (int k = 0; k < 3; ++k) { ms3[k] = 0.0; launches3[k] = 0; }
     for (size_t i = 0; i + 1 < h->prof_used; i += 2) {
         float t = 0.f;
         CK(cudaEventElapsedTime(&t, h->prof_ev[i], h->prof_ev[i + 1]));
-        ms += t;
+        const int k = h->prof_kind[i / 2];
+        ms3[k] += t;
+        launches3[k]++;
     }
-    *gemm_ms = ms;
-    *gemm_launches = h->prof_used / 2;
     h->prof_used = 0;
+    h->prof_kind.clear();
     return ALEXNET_OK;
 }
 

@@ -32,7 +32,8 @@ constexpr int kMaxStages = 8;
 constexpr long long kWaitBudgetCycles = 400000000LL;  // ~0.2 s at 2 GHz
 
 struct GemmParams {
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmOut;   // tmOut: output as {columns, rows, splits}, box {128 bytes, 32, 1}, when tma_store
+    int tma_store;
     int mode, epi;
     int m_tiles, n_tiles, groups, taps_grid, splits;  // tile decomposition (m fastest)
     int tiles_total;
@@ -129,6 +130,28 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+// TMA store of one box from shared memory (bulk async-group completion)
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(tm), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1
@@ -216,13 +239,76 @@ __device__ __forceinline__ void epi_chunk(const P& p, uint32_t* v, bool zero, bo
     }
 }
 
+// Staged epilogue: one warp turns 32 accumulator rows x one 128-byte slab (64 bf16 or 32 fp32 columns) into a
+// 128-byte-swizzled 4 KB tile in shared memory and stores it with one TMA box; rows and columns outside the output
+// tensor are clipped by TMA.  kEpiStageBytes per warp holds two such tiles, used alternately: before a tile is
+// rewritten the store issued from it two slabs earlier must have finished reading (wait_group.read 1).
+constexpr uint32_t kEpiStageBytes = 8192;
+template <typename P>
+__device__ __forceinline__ void epi_slab(const P& p, uint32_t tmem_addr, bool pad_row, long long row_off, int col0, int g,
+                                         int x, int y, int z, uint32_t stage, int lane) {
+    uint32_t w[32];   // the packed 128-byte row
+    if (p.epi == EPI_F32) {
+        tmem_ld32(tmem_addr, w);
+        tmem_ld_wait();
+    } else {
+        const float* bp = p.bias ? p.bias + g * p.out_gx + col0 : nullptr;
+        const uint4* mp = p.mask ? (const uint4*)(p.mask + row_off + col0) : nullptr;
+        #pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint32_t v[32];
+            tmem_ld32(tmem_addr + 32u * half, v);
+            tmem_ld_wait();
+            #pragma unroll
+            for (int qq = 0; qq < 4; ++qq) {       // four 16-byte chunks of eight columns
+                const int q = 4 * half + qq;
+                float f[8];
+                #pragma unroll
+                for (int k = 0; k < 8; ++k) f[k] = __uint_as_float(v[8 * qq + k]);
+                if (bp) {
+                    const float4 b0 = __ldg((const float4*)(bp + 8 * q)), b1 = __ldg((const float4*)(bp + 8 * q + 4));
+                    f[0] += b0.x; f[1] += b0.y; f[2] += b0.z; f[3] += b0.w; f[4] += b1.x; f[5] += b1.y; f[6] += b1.z; f[7] += b1.w;
+                }
+                if (p.relu) {
+                    #pragma unroll
+                    for (int k = 0; k < 8; ++k) f[k] = fmaxf(f[k], 0.f);
+                }
+                if (mp) {
+                    const uint4 mv = __ldg(mp + q);
+                    const __nv_bfloat162* mh = (const __nv_bfloat162*)&mv;
+                    #pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const float2 m2 = __bfloat1622float2(mh[k]);
+                        f[2 * k] = m2.x > 0.f ? f[2 * k] * p.mask_scale : 0.f;
+                        f[2 * k + 1] = m2.y > 0.f ? f[2 * k + 1] * p.mask_scale : 0.f;
+                    }
+                }
+                #pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    __nv_bfloat162 hh = __floats2bfloat162_rn(pad_row ? 0.f : f[2 * k], pad_row ? 0.f : f[2 * k + 1]);
+                    w[4 * q + k] = *(uint32_t*)&hh;
+                }
+            }
+        }
+    }
+    if (lane == 0) bulk_wait_read_1();
+    __syncwarp();
+    const uint32_t rowp = stage + (uint32_t)lane * 128u;
+    #pragma unroll
+    for (int q = 0; q < 8; ++q)
+        st_shared_v4(rowp + (uint32_t)((q ^ (lane & 7)) << 4), w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) { tma_store_3d(&p.tmOut, stage, x, y, z); bulk_commit(); }
+}
+
 constexpr int kABytes = 128 * 128;  // 128 rows x 64 bf16, or 2 boxes of 64 x 64
 
 __host__ __device__ inline int b_stage_bytes(int mode, int BN) {
     return mode == MODE_KK ? BN * 128 : ((BN + 63) / 64) * 8192;
 }
 inline size_t smem_bytes(int mode, int BN, int stages) {
-    return 1024 + (size_t)stages * (kABytes + b_stage_bytes(mode, BN)) + 256;
+    return 1024 + (size_t)stages * (kABytes + b_stage_bytes(mode, BN)) + 4 * kEpiStageBytes + 256;
 }
 
 // position of a CTA in the tile list; tiles are numbered with m fastest, then
@@ -258,9 +344,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     const int bbytes = b_stage_bytes(p.mode, p.BN);
     const int stage_bytes = kABytes + bbytes;
     const int stages = p.stages;
-    // barriers: full[8] @0, empty[8] @64, acc_full[2] @128, acc_empty[2] @144, tmem slot @160, abort flag @168
-    const uint32_t bar_base = base + stages * stage_bytes;
-    uint8_t* gen = smem_raw + (base - raw) + stages * stage_bytes;
+    // epilogue staging (4 warps x kEpiStageBytes), then barriers: full[8] @0, empty[8] @64, acc_full[2] @128,
+    // acc_empty[2] @144, tmem slot @160, abort flag @168
+    const uint32_t epi_stage0 = base + stages * stage_bytes;
+    const uint32_t bar_base = epi_stage0 + 4u * kEpiStageBytes;
+    uint8_t* gen = smem_raw + (bar_base - raw);
     volatile int* abort_flag = (volatile int*)(gen + 168);
     volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 160);
     const uint32_t full0 = bar_base, empty0 = bar_base + 64u, accf0 = bar_base + 128u, acce0 = bar_base + 144u;
@@ -375,6 +463,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         const int r = quad * 32 + lane;          // row within the tile = TMEM lane
         TileCursor tc; tc.init(p);
         int ab = 0; uint32_t aph = 0;
+        int sbuf = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
             const int m0 = tc.m_tile * 128, n0 = tc.n_tile * p.BN, g = tc.g;
@@ -398,18 +487,29 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             if (!(ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag))) break;
             tc_fence_after();
             const uint32_t t0 = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * p.BN);
-            for (int c = 0; c < p.BN; c += 16) {
-                uint32_t v[16];
-                tmem_ld16(t0 + (uint32_t)c, v);
-                tmem_ld_wait();
-                if (!row_ok) continue;
-                epi_chunk(p, v, nsteps <= 0, pad_row, row_off, n0 + c, g);
+            if (p.tma_store) {
+                const int slab = p.epi == EPI_F32 ? 32 : 64;
+                for (int c = 0; c < p.BN; c += slab) {
+                    epi_slab(p, t0 + (uint32_t)c, pad_row, row_off, n0 + c, g, g * p.out_gx * (p.mode != MODE_MNMN) + n0 + c,
+                             m0 + quad * 32 + (p.mode == MODE_MNMN ? g * p.out_gx : 0), tc.z,
+                             epi_stage0 + (uint32_t)quad * kEpiStageBytes + (uint32_t)sbuf * 4096u, lane);
+                    sbuf ^= 1;
+                }
+            } else {
+                for (int c = 0; c < p.BN; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(t0 + (uint32_t)c, v);
+                    tmem_ld_wait();
+                    if (!row_ok) continue;
+                    epi_chunk(p, v, nsteps <= 0, pad_row, row_off, n0 + c, g);
+                }
             }
             // this accumulator buffer may be overwritten by the next tile but one
             tc_fence_before();
             mbar_arrive(acce0 + 8u * ab);
             if (++ab == 2) { ab = 0; aph ^= 1u; }
         }
+        if (p.tma_store && lane == 0) bulk_wait_all();
     }
     tc_fence_before();
     __syncthreads();
@@ -444,7 +544,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 // Accumulators: MH x BN columns per buffer, two buffers when they fit in the
 // 512 TMEM columns.
 struct ConvParams {
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmOut;   // tmOut: output as {columns, rows, splits}, box {128 bytes, 32, 1}, when tma_store
+    int tma_store;
     int m_tiles, n_tiles, groups, splits;   // tile decomposition (m fastest, then n, group, k split)
     int tiles_total;
     int MH;             // 128-row halves per tile (1, 2 or 4)
@@ -473,7 +574,7 @@ struct ConvParams {
 constexpr int kConvMaxThreads = 32 * 9;
 inline int conv_threads(const ConvParams& p) { return 32 * (5 + p.MH); }
 inline size_t conv_smem_bytes(const ConvParams& p) {
-    return 1024 + (size_t)p.a_stages * p.MH * p.a_box_rows * 128 + (size_t)p.b_stages * p.BN * 128 + 512;
+    return 1024 + (size_t)p.a_stages * p.MH * p.a_box_rows * 128 + (size_t)p.b_stages * p.BN * 128 + 4 * kEpiStageBytes + 512;
 }
 
 // tile cursor shared by the roles (m fastest, then n tile, group, split)
@@ -505,9 +606,10 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * 128u, a_bytes = a_box_bytes * MH, b_bytes = (uint32_t)BN * 128u;
     const int a_stages = p.a_stages, b_stages = p.b_stages;
     const uint32_t ring_a = base, ring_b = base + a_stages * a_bytes;
-    // barriers: fullA[8] @0, emptyA[8] @64, fullB[8] @128, emptyB[8] @192, acc_full[2] @256, acc_empty[2] @272,
-    // tmem slot @288, abort flag @296
-    const uint32_t bar_base = ring_b + b_stages * b_bytes;
+    // epilogue staging (4 warps x kEpiStageBytes), then barriers: fullA[8] @0, emptyA[8] @64, fullB[8] @128,
+    // emptyB[8] @192, acc_full[2] @256, acc_empty[2] @272, tmem slot @288, abort flag @296
+    const uint32_t epi_stage0 = ring_b + b_stages * b_bytes;
+    const uint32_t bar_base = epi_stage0 + 4u * kEpiStageBytes;
     uint8_t* gen = smem_raw + (bar_base - raw);
     volatile int* abort_flag = (volatile int*)(gen + 296);
     volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 288);
@@ -621,6 +723,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         const int r = quad * 32 + lane;          // row within a 128-row half = TMEM lane
         ConvCursor tc; tc.init(p);
         int ab = 0; uint32_t aph = 0;
+        int sbuf = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
             const int m0 = tc.m_tile * (128 * MH), n0 = tc.n_tile * BN, g = tc.g;
@@ -639,18 +742,28 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 }
                 const long long row_off = (long long)tc.z * p.split_stride + (long long)row * p.ldo + g * p.out_gx;
                 const uint32_t t0 = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * acc_cols + h * BN);
-                for (int c = 0; c < BN; c += 16) {
-                    uint32_t v[16];
-                    tmem_ld16(t0 + (uint32_t)c, v);
-                    tmem_ld_wait();
-                    if (!row_ok) continue;
-                    epi_chunk(p, v, nsteps <= 0, pad_row, row_off, n0 + c, g);
+                if (p.tma_store) {
+                    const int slab = p.epi == EPI_F32 ? 32 : 64;
+                    for (int c = 0; c < BN; c += slab) {
+                        epi_slab(p, t0 + (uint32_t)c, pad_row, row_off, n0 + c, g, g * p.out_gx + n0 + c, m0 + h * 128 + quad * 32,
+                                 tc.z, epi_stage0 + (uint32_t)quad * kEpiStageBytes + (uint32_t)sbuf * 4096u, lane);
+                        sbuf ^= 1;
+                    }
+                } else {
+                    for (int c = 0; c < BN; c += 16) {
+                        uint32_t v[16];
+                        tmem_ld16(t0 + (uint32_t)c, v);
+                        tmem_ld_wait();
+                        if (!row_ok) continue;
+                        epi_chunk(p, v, nsteps <= 0, pad_row, row_off, n0 + c, g);
+                    }
                 }
             }
             tc_fence_before();
             mbar_arrive(acce0 + 8u * ab);
             if (++ab == acc_stages) { ab = 0; aph ^= 1u; }
         }
+        if (p.tma_store && lane == 0) bulk_wait_all();
     }
     tc_fence_before();
     __syncthreads();
