@@ -432,6 +432,7 @@ int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16
     p.tap_stride = (long long)c.cout * c.cig; p.split_stride = (long long)c.taps * c.cout * c.cig;
     p.epi = tc::EPI_F32; p.mask_scale = 1.f;
     p.out = h->ws; p.status = h->status;
+    p.bias_partial = h->cs_partial; p.bias_ld = c.cout;
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, 64))) return rc;
     if ((rc = make_tm(h, &p.tmB, xin, c.cin, M, (uint64_t)c.cin * 2, 72))) return rc;
@@ -579,12 +580,11 @@ void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
     Replica& R = h->rep[r];
     const ConvL& c = h->L.conv[l];
     const Plan& P = R.conv_wg[l][slot];
-    launch_gemm(h, P, st);
+    launch_gemm(h, P, st);     // weight-gradient partials per row split, and the bias-gradient partials
     const long long total = (long long)c.taps * c.cout * c.cig;
-    kn::wgrad_reduce_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.w.splits, P.w.split_stride, total, R.g + c.w_off, l == 0);
+    kn::wgrad_reduce_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.w.splits, P.w.split_stride, total, R.g + c.w_off, l == 0,
+                                                              h->cs_partial, c.cout, R.g + c.b_off);
     h->launches++;
-    bf16* dyv[5] = {R.da1, R.da2, R.da3, R.da4, R.da5};
-    colsum(h, dyv[l], (long long)h->B * c.gout.Hp * c.gout.Wp, c.cout, R.g + c.b_off, st);
 }
 void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st) {
     Replica& R = h->rep[r];
@@ -606,18 +606,22 @@ void op_fc_bwd(alexnet* h, int r, int l, cudaStream_t st) {
     const FcL& f = h->L.fc[l];
     const Plan& P = R.fc_bwd[l];
     launch_gemm(h, P, st);
-    const long long total = (long long)h->B * f.K;
     const bf16* masks[3] = {nullptr, R.f6, R.f7};
     bf16* outs[3] = {R.dp5, R.df6, R.df7};
-    kn::fc_reduce_bwd_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, masks[l], h->drop_scale, total, outs[l]);
+    // the data gradient of layer l is the output gradient of layer l-1: its column sums are that layer's bias gradient
+    float* db = l > 0 ? R.g + h->L.fc[l - 1].b_off : nullptr;
+    kn::fc_reduce_bwd_kernel<<<nblk(f.K, 32), 256, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, masks[l], h->drop_scale, h->B, f.K,
+                                                           outs[l], db);
     h->launches++;
 }
-void op_fc_wg(alexnet* h, int r, int l, cudaStream_t st) {
+void op_fc_wg(alexnet* h, int r, int l, bool with_bias, cudaStream_t st) {
     Replica& R = h->rep[r];
     const FcL& f = h->L.fc[l];
     launch_gemm(h, R.fc_wg[l], st);
-    const bf16* dyv[3] = {R.df6, R.df7, R.dz};
-    colsum(h, dyv[l], h->B, f.N, R.g + f.b_off, st);
+    if (with_bias) {    // in the step only fc8 needs this: fc6 / fc7 get theirs from the data-gradient reduction above them
+        const bf16* dyv[3] = {R.df6, R.df7, R.dz};
+        colsum(h, dyv[l], h->B, f.N, R.g + f.b_off, st);
+    }
 }
 void op_lrn_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
@@ -699,9 +703,9 @@ void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
     op_pool_fwd(h, r, 2, st);
     op_fc_fwd(h, r, 0, step, st); op_fc_fwd(h, r, 1, step, st); op_fc_fwd(h, r, 2, step, st);
     op_softmax(h, r, slot, st);
-    op_fc_wg(h, r, 2, st); op_fc_bwd(h, r, 2, st);
-    op_fc_wg(h, r, 1, st); op_fc_bwd(h, r, 1, st);
-    op_fc_wg(h, r, 0, st); op_fc_bwd(h, r, 0, st);
+    op_fc_wg(h, r, 2, true, st); op_fc_bwd(h, r, 2, st);
+    op_fc_wg(h, r, 1, false, st); op_fc_bwd(h, r, 1, st);
+    op_fc_wg(h, r, 0, false, st); op_fc_bwd(h, r, 0, st);
     op_pool_bwd(h, r, 2, st);
     op_conv_wg(h, r, 4, slot, st); op_conv_bwd(h, r, 4, st);
     op_conv_wg(h, r, 3, slot, st); op_conv_bwd(h, r, 3, st);
@@ -1057,7 +1061,7 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
         else if (op <= ALEXNET_OP_CONV5_BWD_WEIGHT) op_conv_wg(h, replica, op - ALEXNET_OP_CONV1_BWD_WEIGHT, slot, st);
         else if (op <= ALEXNET_OP_FC8_FWD) op_fc_fwd(h, replica, op - ALEXNET_OP_FC6_FWD, R.slot_step[slot], st);
         else if (op <= ALEXNET_OP_FC8_BWD_DATA) op_fc_bwd(h, replica, op - ALEXNET_OP_FC6_BWD_DATA, st);
-        else if (op <= ALEXNET_OP_FC8_BWD_WEIGHT) op_fc_wg(h, replica, op - ALEXNET_OP_FC6_BWD_WEIGHT, st);
+        else if (op <= ALEXNET_OP_FC8_BWD_WEIGHT) op_fc_wg(h, replica, op - ALEXNET_OP_FC6_BWD_WEIGHT, true, st);
         else if (op <= ALEXNET_OP_LRN2_FWD) op_lrn_fwd(h, replica, op - ALEXNET_OP_LRN1_FWD, st);
         else if (op <= ALEXNET_OP_LRN2_BWD) op_lrn_bwd(h, replica, op - ALEXNET_OP_LRN1_BWD, st);
         else if (op <= ALEXNET_OP_POOL5_FWD) op_pool_fwd(h, replica, op - ALEXNET_OP_POOL1_FWD, st);

@@ -246,20 +246,41 @@ __global__ void fc_reduce_fwd_kernel(const float* __restrict__ ws, int splits, l
     }
     if (out_f32) out_f32[t] = v; else out_bf16[t] = __float2bfloat16_rn(v);
 }
-// dx[b][k] = [mask[b][k] > 0] * scale * sum_z ws[z][b][k] -> bf16 (mask = the layer input, post ReLU and dropout)
-__global__ void fc_reduce_bwd_kernel(const float* __restrict__ ws, int splits, long long split_stride,
-                                     const __nv_bfloat16* __restrict__ mask, float scale, long long total,
-                                     __nv_bfloat16* __restrict__ out) {
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= total) return;
-    float v = 0.f;
-    for (int z = 0; z < splits; ++z) v += ws[z * split_stride + t];
-    if (mask) v = __bfloat162float(mask[t]) > 0.f ? v * scale : 0.f;
-    out[t] = __float2bfloat16_rn(v);
+// dx[b][k] = [mask[b][k] > 0] * scale * sum_z ws[z][b][k] -> bf16 (mask = the layer input, post ReLU and dropout);
+// db[k] = sum_b dx[b][k] (of the bf16-rounded values: the bias gradient of the layer below), when db != nullptr.
+// grid: K/32 blocks of 256 threads = 32 columns x 8 row lanes.
+__global__ void __launch_bounds__(256) fc_reduce_bwd_kernel(const float* __restrict__ ws, int splits, long long split_stride,
+                                                            const __nv_bfloat16* __restrict__ mask, float scale, int B, int K,
+                                                            __nv_bfloat16* __restrict__ out, float* __restrict__ db) {
+    __shared__ float red[8][33];
+    const int c = blockIdx.x * 32 + (threadIdx.x & 31), rl = threadIdx.x >> 5;
+    float acc = 0.f;
+    if (c < K) {
+        for (int b = rl; b < B; b += 8) {
+            const size_t t = (size_t)b * K + c;
+            float v = 0.f;
+            for (int z = 0; z < splits; ++z) v += ws[z * split_stride + t];
+            if (mask) v = __bfloat162float(mask[t]) > 0.f ? v * scale : 0.f;
+            const __nv_bfloat16 o = __float2bfloat16_rn(v);
+            out[t] = o;
+            acc += __bfloat162float(o);
+        }
+    }
+    if (!db) return;
+    red[rl][threadIdx.x & 31] = acc;
+    __syncthreads();
+    if (threadIdx.x < 32 && c < K) {
+        float s = 0.f;
+        #pragma unroll
+        for (int q = 0; q < 8; ++q) s += red[q][threadIdx.x];
+        db[c] = s;
+    }
 }
 // g[i] = sum_z ws[z][i]; conv1: entries of the 12x12 zero-padded filter outside 11x11 stay zero.
+// The first `cout` threads also add the per-split bias-gradient partials: db[c] = sum_z bias_partial[z][c].
 __global__ void wgrad_reduce_kernel(const float* __restrict__ ws, int splits, long long split_stride,
-                                    long long total, float* __restrict__ g, int conv1_pad_mask) {
+                                    long long total, float* __restrict__ g, int conv1_pad_mask,
+                                    const float* __restrict__ bias_partial, int cout, float* __restrict__ db) {
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= total) return;
     float v = 0.f;
@@ -270,6 +291,11 @@ __global__ void wgrad_reduce_kernel(const float* __restrict__ ws, int splits, lo
         if (ky > 10 || kx > 10) v = 0.f;
     }
     g[t] = v;
+    if (bias_partial && t < cout) {
+        float b = 0.f;
+        for (int z = 0; z < splits; ++z) b += bias_partial[(size_t)z * cout + t];
+        db[t] = b;
+    }
 }
 
 // db[c] = sum over rows of dy[row][c] (bf16 in, fp32 out), two stages: grid (ceil(C/64), row_splits)

@@ -814,11 +814,13 @@ struct WgradParams {
     long long split_stride, tap_stride;
     int epi, relu; float mask_scale; const float* bias; const __nv_bfloat16* mask;   // fixed: EPI_F32, unused
     void* out;
+    float* bias_partial;        // [split][all output channels] column sums of dy, or nullptr
+    int bias_ld;                // output channels over all groups
     int* status;
 };
 constexpr int kWgABytes = 16384, kWgBBytes = 72 * 128;
 inline int wgrad_threads(const WgradParams& p) { return 32 * (5 + p.NI); }
-inline size_t wgrad_smem_bytes(const WgradParams& p) { return 1024 + (size_t)p.stages * (kWgABytes + kWgBBytes) + 256; }
+inline size_t wgrad_smem_bytes(const WgradParams& p) { return 1024 + (size_t)p.stages * (kWgABytes + kWgBBytes) + 4096 + 256; }
 
 __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant__ WgradParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -826,8 +828,10 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
     const uint32_t base = (raw + 1023u) & ~1023u;
     const int stages = p.stages, NI = p.NI;
     constexpr uint32_t stage_bytes = kWgABytes + kWgBBytes;
-    // barriers: full[8] @0, empty[8] @64, acc_full @128, tmem slot @136, abort flag @144
-    const uint32_t bar_base = base + stages * stage_bytes;
+    // 4 KB for the bias-gradient reduction, then barriers: full[8] @0, empty[8] @64, acc_full @128, tmem slot @136,
+    // abort flag @144
+    const uint32_t red_base = base + stages * stage_bytes;
+    const uint32_t bar_base = red_base + 4096u;
     uint8_t* gen = smem_raw + (bar_base - raw);
     volatile int* abort_flag = (volatile int*)(gen + 144);
     volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 136);
@@ -836,20 +840,6 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
     const int acc_cols = 64 * p.kw;
     uint32_t ncols = 32;
     while ((int)ncols < acc_cols) ncols <<= 1;
-
-    if (threadIdx.x == 0) {
-        *abort_flag = 0;
-        for (int s = 0; s < stages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, NI); }
-        mbar_init(accf, NI);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        tma_prefetch_desc(&p.tmA);
-        tma_prefetch_desc(&p.tmB);
-    }
-    if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), ncols);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
 
     // this CTA's tile (one per CTA: the grid equals the tile count)
     int r = blockIdx.x;
@@ -860,6 +850,24 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
     const int z = r / p.kh;
     const int s_begin = z * p.steps_per_split;
     const int nsteps = min(p.steps_total, s_begin + p.steps_per_split) - s_begin;
+
+    // the CTAs of filter row 0 and input block 0 also sum the dy tile over the rows (the bias gradient): their four
+    // epilogue warps read every A stage and release it together with the issuers
+    const bool do_bias = p.bias_partial != nullptr && ky == 0 && n_tile == 0;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < stages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, NI + (do_bias ? 4 : 0)); }
+        mbar_init(accf, NI);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&p.tmA);
+        tma_prefetch_desc(&p.tmB);
+    }
+    if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), ncols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -903,6 +911,39 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
         const int quad = warp & 3;
         const int row = m_tile * 128 + quad * 32 + lane;     // output channel within the group
         const bool row_ok = row < p.M_total;
+        if (do_bias) {
+            // thread te: eight output channels (16-byte chunk cc of the 128-channel tile) of rows rg*8 .. rg*8+7 of a stage
+            const int te = (warp - NI - 1) * 32 + lane, cc = te & 15, rg = te >> 4;
+            float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            int st = 0; uint32_t ph = 0;
+            bool ok = true;
+            for (int i = 0; i < nsteps; ++i) {
+                if (!(ok = mbar_wait(full0 + 8u * st, ph, abort_flag))) break;
+                const uint32_t a0 = base + st * stage_bytes + (uint32_t)(cc >> 3) * 8192u + (uint32_t)rg * 1024u;
+                #pragma unroll
+                for (int rr = 0; rr < 8; ++rr) {
+                    uint4 u;
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w)
+                                 : "r"(a0 + (uint32_t)rr * 128u + (uint32_t)(((cc & 7) ^ rr) << 4)));
+                    const __nv_bfloat162* hh = (const __nv_bfloat162*)&u;
+                    #pragma unroll
+                    for (int k = 0; k < 4; ++k) { const float2 f = __bfloat1622float2(hh[k]); acc[2 * k] += f.x; acc[2 * k + 1] += f.y; }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty0 + 8u * st);
+                if (++st == stages) { st = 0; ph ^= 1u; }
+            }
+            float* red = (float*)(smem_raw + (red_base - raw));     // [8 row groups][128 channels]
+            #pragma unroll
+            for (int k = 0; k < 8; ++k) red[rg * 128 + cc * 8 + k] = acc[k];
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (ok && te + m_tile * 128 < p.M_total) {
+                float sum = 0.f;
+                #pragma unroll
+                for (int q = 0; q < 8; ++q) sum += red[q * 128 + te];
+                p.bias_partial[(size_t)z * p.bias_ld + g * p.out_gx + m_tile * 128 + te] = sum;
+            }
+        }
         if (mbar_wait(accf, 0, abort_flag)) {
             tc_fence_after();
             const uint32_t t0 = tmem + ((uint32_t)(quad * 32) << 16);
