@@ -118,6 +118,8 @@ struct Replica {
     bool consumed_valid[2];
     uint64_t slot_step[2];
     int next_load, next_train, loaded, last_slot;
+    // the step fuses LRN with pooling and never writes n1/n2 or dn1/dn2; get_tensor fills them in on demand
+    bool n_stale[2], dn_stale[2];
     // plans
     Plan conv_fwd[5][2], conv_bwd[5], conv_wg[5][2], fc_fwd[3], fc_bwd[3], fc_wg[3];
 };
@@ -610,7 +612,7 @@ void op_fc_bwd(alexnet* h, int r, int l, cudaStream_t st) {
     bf16* outs[3] = {R.dp5, R.df6, R.df7};
     // the data gradient of layer l is the output gradient of layer l-1: its column sums are that layer's bias gradient
     float* db = l > 0 ? R.g + h->L.fc[l - 1].b_off : nullptr;
-    kn::fc_reduce_bwd_kernel<<<nblk(f.K, 32), 256, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, masks[l], h->drop_scale, h->B, f.K,
+    kn::fc_reduce_bwd_kernel<<<nblk(f.K, 32), 1024, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, masks[l], h->drop_scale, h->B, f.K,
                                                            outs[l], db);
     h->launches++;
 }
@@ -625,6 +627,7 @@ void op_fc_wg(alexnet* h, int r, int l, bool with_bias, cudaStream_t st) {
 }
 void op_lrn_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
+    R.n_stale[which] = false;
     const Grid& g = h->L.conv[which].gout;
     const long long rows = (long long)h->B * g.Hp * g.Wp;
     kn::lrn_fwd_kernel<<<nblk(rows * (g.C / 8), 256), 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.n2 : R.n1,
@@ -655,6 +658,7 @@ void op_pool_fwd(alexnet* h, int r, int which, cudaStream_t st) {
 }
 void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
+    if (which < 2) R.dn_stale[which] = false;
     const PoolGeo& g = kPool[which];
     const bf16* dy[3] = {R.dp1, R.dp2, R.dp5};
     const uint8_t* a[3] = {R.arg1, R.arg2, R.arg5};
@@ -664,6 +668,29 @@ void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     kn::pool_bwd_kernel<<<grid, 256, 0, st>>>(dy[which], a[which], relu[which], dx[which], g.C / 8, g.Hpi, g.Wpi,
                                               g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo, g.Wpo);
     h->launches++;
+}
+void op_lrn_pool_fwd(alexnet* h, int r, int which, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const PoolGeo& g = kPool[which];
+    const int cpr = g.C / 8;
+    const dim3 grid((g.Ho + 1) / 2, h->B);
+    const size_t smem = (size_t)5 * g.Wi * cpr * 16;
+    kn::lrn_pool_fwd_kernel<<<grid, 256, smem, st>>>(which ? R.a2 : R.a1, which ? R.p2 : R.p1, which ? R.arg2 : R.arg1, cpr, g.Hpi,
+                                                     g.Wpi, g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta,
+                                                     h->cfg.lrn_k);
+    h->launches++;
+    R.n_stale[which] = true;
+}
+void op_pool_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const PoolGeo& g = kPool[which];
+    const int cpr = g.C / 8, ppb = 256 / cpr;
+    const dim3 grid((g.Wpi + ppb - 1) / ppb, g.Hpi, h->B);
+    kn::pool_lrn_bwd_kernel<<<grid, 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.dp2 : R.dp1, which ? R.arg2 : R.arg1,
+                                                  which ? R.da2 : R.da1, cpr, ppb, g.Hpi, g.Wpi, g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo,
+                                                  g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
+    h->launches++;
+    R.dn_stale[which] = true;
 }
 void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
     Replica& R = h->rep[r];
@@ -697,8 +724,8 @@ void op_preprocess(alexnet* h, int r, int slot, uint64_t step, cudaStream_t st) 
 void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
     Replica& R = h->rep[r];
     const uint64_t step = R.slot_step[slot];
-    op_conv_fwd(h, r, 0, slot, st); op_lrn_fwd(h, r, 0, st); op_pool_fwd(h, r, 0, st);
-    op_conv_fwd(h, r, 1, slot, st); op_lrn_fwd(h, r, 1, st); op_pool_fwd(h, r, 1, st);
+    op_conv_fwd(h, r, 0, slot, st); op_lrn_pool_fwd(h, r, 0, st);
+    op_conv_fwd(h, r, 1, slot, st); op_lrn_pool_fwd(h, r, 1, st);
     op_conv_fwd(h, r, 2, slot, st); op_conv_fwd(h, r, 3, slot, st); op_conv_fwd(h, r, 4, slot, st);
     op_pool_fwd(h, r, 2, st);
     op_fc_fwd(h, r, 0, step, st); op_fc_fwd(h, r, 1, step, st); op_fc_fwd(h, r, 2, step, st);
@@ -710,9 +737,9 @@ void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
     op_conv_wg(h, r, 4, slot, st); op_conv_bwd(h, r, 4, st);
     op_conv_wg(h, r, 3, slot, st); op_conv_bwd(h, r, 3, st);
     op_conv_wg(h, r, 2, slot, st); op_conv_bwd(h, r, 2, st);
-    op_pool_bwd(h, r, 1, st); op_lrn_bwd(h, r, 1, st);
+    op_pool_lrn_bwd(h, r, 1, st);
     op_conv_wg(h, r, 1, slot, st); op_conv_bwd(h, r, 1, st);
-    op_pool_bwd(h, r, 0, st); op_lrn_bwd(h, r, 0, st);
+    op_pool_lrn_bwd(h, r, 0, st);
     op_conv_wg(h, r, 0, slot, st);
 }
 
@@ -856,6 +883,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     CKC(cudaFuncSetAttribute(tc::gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CKC(cudaFuncSetAttribute(kn::lrn_pool_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
     {
         int dev = 0;
         CKC(cudaGetDevice(&dev));
@@ -867,6 +895,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     for (int r = 0; r < cfg->replicas; ++r) {
         Replica& R = h->rep[r];
         R.next_load = R.next_train = R.loaded = R.last_slot = 0;
+        R.n_stale[0] = R.n_stale[1] = R.dn_stale[0] = R.dn_stale[1] = false;
         for (int s = 0; s < 2; ++s) {
             CKC(cudaEventCreateWithFlags(&R.ready[s], cudaEventDisableTiming));
             CKC(cudaEventCreateWithFlags(&R.consumed[s], cudaEventDisableTiming));
@@ -986,6 +1015,13 @@ int alexnet_get_tensor(alexnet_t* h, int replica, int tensor_id, float* out, siz
     if (replica < 0 || replica >= h->cfg.replicas || !out || !tensor_desc(h, replica, tensor_id, &T) || n != tensor_elems(T, h->B))
         return fail(h, ALEXNET_ERR_ARG, "get_tensor: bad argument");
     const int B = h->B;
+    {
+        Replica& R = h->rep[replica];
+        if (tensor_id == ALEXNET_T_N1 && R.n_stale[0]) op_lrn_fwd(h, replica, 0, h->cs);
+        if (tensor_id == ALEXNET_T_N2 && R.n_stale[1]) op_lrn_fwd(h, replica, 1, h->cs);
+        if (tensor_id == ALEXNET_T_DN1 && R.dn_stale[0]) op_pool_bwd(h, replica, 0, h->cs);
+        if (tensor_id == ALEXNET_T_DN2 && R.dn_stale[1]) op_pool_bwd(h, replica, 1, h->cs);
+    }
     std::vector<uint8_t> raw(tensor_dev_bytes(T, B));
     CK(cudaStreamSynchronize(h->cs));
     CK(cudaStreamSynchronize(h->ls));
@@ -1043,6 +1079,13 @@ int alexnet_set_tensor(alexnet_t* h, int replica, int tensor_id, const float* in
     CK(cudaStreamSynchronize(h->cs));
     CK(cudaStreamSynchronize(h->ls));
     CK(cudaMemcpy(T.ptr, raw.data(), raw.size(), cudaMemcpyHostToDevice));
+    {
+        Replica& R = h->rep[replica];
+        if (tensor_id == ALEXNET_T_N1) R.n_stale[0] = false;
+        if (tensor_id == ALEXNET_T_N2) R.n_stale[1] = false;
+        if (tensor_id == ALEXNET_T_DN1) R.dn_stale[0] = false;
+        if (tensor_id == ALEXNET_T_DN2) R.dn_stale[1] = false;
+    }
     return ALEXNET_OK;
 }
 

@@ -90,17 +90,12 @@ __device__ __forceinline__ void pow_neg(float s, float beta, float& sp, float& r
     else { sp = exp2f(-beta * __log2f(s)); rs = __fdividef(1.f, s); }
 }
 // b_c = a_c * (k + alpha * sum_{c' in [c-2,c+2] clipped} a_c'^2)^(-beta); one thread = 8 channels of one pixel.
-__global__ void __launch_bounds__(256) lrn_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ b,
-                                                      unsigned total, unsigned cpr, float alpha, float beta, float k) {
-    const unsigned t = blockIdx.x * 256u + threadIdx.x;
-    if (t >= total) return;
-    const unsigned ch = t % cpr;
-    const uint4* ap = (const uint4*)a + t;
+__device__ __forceinline__ uint4 lrn_fwd8(const uint4* ap, bool has_l, bool has_r, float alpha, float beta, float k) {
     const uint4 zero = make_uint4(0, 0, 0, 0);
     float f[24];
-    unpack8(ch > 0 ? __ldg(ap - 1) : zero, f);
+    unpack8(has_l ? __ldg(ap - 1) : zero, f);
     unpack8(__ldg(ap), f + 8);
-    unpack8(ch < cpr - 1 ? __ldg(ap + 1) : zero, f + 16);
+    unpack8(has_r ? __ldg(ap + 1) : zero, f + 16);
     float sq[12];
     #pragma unroll
     for (int i = 0; i < 12; ++i) sq[i] = f[6 + i] * f[6 + i];
@@ -112,28 +107,19 @@ __global__ void __launch_bounds__(256) lrn_fwd_kernel(const __nv_bfloat16* __res
         pow_neg(fmaf(alpha, ss, k), beta, sp, rs);
         o[i] = f[8 + i] * sp;
     }
-    ((uint4*)b)[t] = pack8(o);
+    return pack8(o);
+}
+__global__ void __launch_bounds__(256) lrn_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ b,
+                                                      unsigned total, unsigned cpr, float alpha, float beta, float k) {
+    const unsigned t = blockIdx.x * 256u + threadIdx.x;
+    if (t >= total) return;
+    const unsigned ch = t % cpr;
+    ((uint4*)b)[t] = lrn_fwd8((const uint4*)a + t, ch > 0, ch < cpr - 1, alpha, beta, k);
 }
 // da_m = [a_m > 0] * ( g_m s_m^-beta - 2 alpha beta a_m sum_{c in [m-2,m+2]} g_c a_c s_c^(-beta-1) )
 // (the ReLU mask of the convolution that produced a is applied here).  One thread = 8 channels of one
 // pixel; it needs s for the 12 channels c0-2 .. c0+9 and a for c0-4 .. c0+11.
-__global__ void __launch_bounds__(256) lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ g,
-                                                      __nv_bfloat16* __restrict__ da, unsigned total, unsigned cpr,
-                                                      float alpha, float beta, float k) {
-    const unsigned t = blockIdx.x * 256u + threadIdx.x;
-    if (t >= total) return;
-    const unsigned ch = t % cpr;
-    const uint4* ap = (const uint4*)a + t;
-    const uint4* gp = (const uint4*)g + t;
-    const uint4 zero = make_uint4(0, 0, 0, 0);
-    const bool has_l = ch > 0, has_r = ch < cpr - 1;
-    float fa[24], fg[24];
-    unpack8(has_l ? __ldg(ap - 1) : zero, fa);
-    unpack8(__ldg(ap), fa + 8);
-    unpack8(has_r ? __ldg(ap + 1) : zero, fa + 16);
-    unpack8(has_l ? __ldg(gp - 1) : zero, fg);
-    unpack8(__ldg(gp), fg + 8);
-    unpack8(has_r ? __ldg(gp + 1) : zero, fg + 16);
+__device__ __forceinline__ uint4 lrn_bwd8(const float* fa, const float* fg, float alpha, float beta, float k) {
     float sq[16];
     #pragma unroll
     for (int i = 0; i < 16; ++i) sq[i] = fa[4 + i] * fa[4 + i];
@@ -154,7 +140,26 @@ __global__ void __launch_bounds__(256) lrn_bwd_kernel(const __nv_bfloat16* __res
         const float v = fmaf(fg[8 + i], sp[i + 2], -c2 * am * acc);
         o[i] = am > 0.f ? v : 0.f;
     }
-    ((uint4*)da)[t] = pack8(o);
+    return pack8(o);
+}
+__global__ void __launch_bounds__(256) lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ g,
+                                                      __nv_bfloat16* __restrict__ da, unsigned total, unsigned cpr,
+                                                      float alpha, float beta, float k) {
+    const unsigned t = blockIdx.x * 256u + threadIdx.x;
+    if (t >= total) return;
+    const unsigned ch = t % cpr;
+    const uint4* ap = (const uint4*)a + t;
+    const uint4* gp = (const uint4*)g + t;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    const bool has_l = ch > 0, has_r = ch < cpr - 1;
+    float fa[24], fg[24];
+    unpack8(has_l ? __ldg(ap - 1) : zero, fa);
+    unpack8(__ldg(ap), fa + 8);
+    unpack8(has_r ? __ldg(ap + 1) : zero, fa + 16);
+    unpack8(has_l ? __ldg(gp - 1) : zero, fg);
+    unpack8(__ldg(gp), fg + 8);
+    unpack8(has_r ? __ldg(gp + 1) : zero, fg + 16);
+    ((uint4*)da)[t] = lrn_bwd8(fa, fg, alpha, beta, k);
 }
 
 // ------------------------------------------------------------------ max pool
@@ -187,6 +192,25 @@ __global__ void __launch_bounds__(256) pool_fwd_kernel(const __nv_bfloat16* __re
 }
 // dx[y][x] = sum over the (up to 4) windows containing (y,x) whose argmax points at it; optional ReLU mask.
 // grid: (ceil(Wpi*cpr / 256), Hpi, B); one thread = 8 channels of one input pixel (pad pixels get zero).
+__device__ __forceinline__ void pool_bwd8(const __nv_bfloat16* __restrict__ dy, const uint8_t* __restrict__ arg, float* acc,
+                                          int n, int y, int x, int ch, int cpr, int Ho, int Wo, int Hpo, int Wpo) {
+    const int oy_lo = max(0, (y - 1) >> 1), oy_hi = min(Ho - 1, y >> 1);
+    const int ox_lo = max(0, (x - 1) >> 1), ox_hi = min(Wo - 1, x >> 1);
+    for (int oy = oy_lo; oy <= oy_hi; ++oy)
+        for (int ox = ox_lo; ox <= ox_hi; ++ox) {
+            const unsigned code = (unsigned)((y - 2 * oy) * 3 + (x - 2 * ox)) * 0x01010101u;
+            const uint2 ab = __ldg((const uint2*)arg + ((size_t)(n * Ho + oy) * Wo + ox) * cpr + ch);
+            float f[8];
+            unpack8(__ldg((const uint4*)dy + ((size_t)(n * Hpo + oy) * Wpo + ox) * cpr + ch), f);
+            // byte-wise equality of the eight argmax codes with this pixel's code
+            const unsigned e0 = ab.x ^ code, e1 = ab.y ^ code;
+            #pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (((e0 >> (8 * q)) & 0xFFu) == 0u) acc[q] += f[q];
+                if (((e1 >> (8 * q)) & 0xFFu) == 0u) acc[q + 4] += f[q + 4];
+            }
+        }
+}
 __global__ void __launch_bounds__(256) pool_bwd_kernel(const __nv_bfloat16* __restrict__ dy, const uint8_t* __restrict__ arg,
                                                        const __nv_bfloat16* __restrict__ relu_src, __nv_bfloat16* __restrict__ dx,
                                                        int cpr, int Hpi, int Wpi, int Hi, int Wi, int Ho, int Wo, int Hpo, int Wpo) {
@@ -197,22 +221,7 @@ __global__ void __launch_bounds__(256) pool_bwd_kernel(const __nv_bfloat16* __re
     const size_t t = ((size_t)(n * Hpi + y) * Wpi + x) * cpr + ch;
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (y < Hi && x < Wi) {
-        const int oy_lo = max(0, (y - 1) >> 1), oy_hi = min(Ho - 1, y >> 1);
-        const int ox_lo = max(0, (x - 1) >> 1), ox_hi = min(Wo - 1, x >> 1);
-        for (int oy = oy_lo; oy <= oy_hi; ++oy)
-            for (int ox = ox_lo; ox <= ox_hi; ++ox) {
-                const unsigned code = (unsigned)((y - 2 * oy) * 3 + (x - 2 * ox)) * 0x01010101u;
-                const uint2 ab = __ldg((const uint2*)arg + ((size_t)(n * Ho + oy) * Wo + ox) * cpr + ch);
-                float f[8];
-                unpack8(__ldg((const uint4*)dy + ((size_t)(n * Hpo + oy) * Wpo + ox) * cpr + ch), f);
-                // byte-wise equality of the eight argmax codes with this pixel's code
-                const unsigned e0 = ab.x ^ code, e1 = ab.y ^ code;
-                #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    if (((e0 >> (8 * q)) & 0xFFu) == 0u) acc[q] += f[q];
-                    if (((e1 >> (8 * q)) & 0xFFu) == 0u) acc[q + 4] += f[q + 4];
-                }
-            }
+        pool_bwd8(dy, arg, acc, n, y, x, ch, cpr, Ho, Wo, Hpo, Wpo);
         if (relu_src) {
             float m[8];
             unpack8(__ldg((const uint4*)relu_src + t), m);
@@ -221,6 +230,79 @@ __global__ void __launch_bounds__(256) pool_bwd_kernel(const __nv_bfloat16* __re
         }
     }
     ((uint4*)dx)[t] = pack8(acc);
+}
+
+// ------------------------------------------------- LRN + pool fused (the training step)
+// Forward: p = maxpool(LRN(a)) without writing the normalised tensor.  One block = one image and two output
+// rows: the (up to five) input rows they cover are normalised once into shared memory as bf16 (the same rounding
+// as lrn_fwd_kernel's output), then pooled from there with pool_fwd_kernel's tie rule.
+// grid: (ceil(Ho/2), B); dynamic shared memory 5 * Wi * cpr * 16 bytes.
+__global__ void __launch_bounds__(256) lrn_pool_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ y,
+                                                           uint8_t* __restrict__ arg, int cpr, int Hpi, int Wpi, int Hi, int Wi,
+                                                           int Ho, int Wo, int Hpo, int Wpo, float alpha, float beta, float k) {
+    extern __shared__ uint4 nrm[];            // [row][x][chunk]
+    const int n = blockIdx.y, oy0 = 2 * blockIdx.x;
+    const int iy0 = 2 * oy0, nrows = min(5, Hi - iy0);
+    const int row_vecs = Wi * cpr;
+    for (int t = threadIdx.x; t < nrows * row_vecs; t += 256) {
+        const int r = t / row_vecs, q = t - r * row_vecs;
+        const int x = q / cpr, ch = q - x * cpr;
+        nrm[t] = lrn_fwd8((const uint4*)a + ((size_t)(n * Hpi + iy0 + r) * Wpi + x) * cpr + ch, ch > 0, ch < cpr - 1, alpha, beta, k);
+    }
+    __syncthreads();
+    const int out_vecs = Wo * cpr;
+    for (int t = threadIdx.x; t < 2 * out_vecs; t += 256) {
+        const int oyl = t / out_vecs, q = t - oyl * out_vecs;
+        const int oy = oy0 + oyl;
+        if (oy >= Ho) break;
+        const int ox = q / cpr, ch = q - ox * cpr;
+        float best[8]; int bi[8];
+        #pragma unroll
+        for (int ky = 0; ky < 3; ++ky)
+            #pragma unroll
+            for (int kx = 0; kx < 3; ++kx) {
+                float f[8];
+                unpack8(nrm[((2 * oyl + ky) * Wi + 2 * ox + kx) * cpr + ch], f);
+                #pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if ((ky == 0 && kx == 0) || f[j] > best[j]) { best[j] = f[j]; bi[j] = ky * 3 + kx; }
+            }
+        ((uint4*)y)[((size_t)(n * Hpo + oy) * Wpo + ox) * cpr + ch] = pack8(best);
+        uint2 ab;
+        ab.x = bi[0] | (bi[1] << 8) | (bi[2] << 16) | (bi[3] << 24);
+        ab.y = bi[4] | (bi[5] << 8) | (bi[6] << 16) | (bi[7] << 24);
+        ((uint2*)arg)[((size_t)(n * Ho + oy) * Wo + ox) * cpr + ch] = ab;
+    }
+}
+// Backward: da = LRN'(a, dn) with dn = maxpool'(dp, arg) formed on the fly (rounded to bf16 as pool_bwd_kernel
+// stores it) and passed to the channel neighbours of the same pixel through shared memory.
+// One thread = 8 channels of one pixel of the padded grid; ppb = floor(256 / cpr) pixels per block.
+// grid: (ceil(Wpi / ppb), Hpi, B).
+__global__ void __launch_bounds__(256) pool_lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ dp,
+                                                           const uint8_t* __restrict__ arg, __nv_bfloat16* __restrict__ da,
+                                                           int cpr, int ppb, int Hpi, int Wpi, int Hi, int Wi, int Ho, int Wo,
+                                                           int Hpo, int Wpo, float alpha, float beta, float k) {
+    __shared__ uint4 dn[256];
+    const int px = threadIdx.x / cpr, ch = threadIdx.x - px * cpr;
+    const int x = blockIdx.x * ppb + px, y = blockIdx.y, n = blockIdx.z;
+    const bool active = px < ppb && x < Wpi;
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (active && y < Hi && x < Wi) pool_bwd8(dp, arg, acc, n, y, x, ch, cpr, Ho, Wo, Hpo, Wpo);
+    dn[threadIdx.x] = pack8(acc);
+    __syncthreads();
+    if (!active) return;
+    const size_t t = ((size_t)(n * Hpi + y) * Wpi + x) * cpr + ch;
+    const uint4* ap = (const uint4*)a + t;
+    const uint4 zero = make_uint4(0, 0, 0, 0);
+    const bool has_l = ch > 0, has_r = ch < cpr - 1;
+    float fa[24], fg[24];
+    unpack8(has_l ? __ldg(ap - 1) : zero, fa);
+    unpack8(__ldg(ap), fa + 8);
+    unpack8(has_r ? __ldg(ap + 1) : zero, fa + 16);
+    unpack8(has_l ? dn[threadIdx.x - 1] : zero, fg);
+    unpack8(dn[threadIdx.x], fg + 8);
+    unpack8(has_r ? dn[threadIdx.x + 1] : zero, fg + 16);
+    ((uint4*)da)[t] = lrn_bwd8(fa, fg, alpha, beta, k);
 }
 
 // ------------------------------------------------- split-K reductions (FC, wgrad)
@@ -248,15 +330,15 @@ __global__ void fc_reduce_fwd_kernel(const float* __restrict__ ws, int splits, l
 }
 // dx[b][k] = [mask[b][k] > 0] * scale * sum_z ws[z][b][k] -> bf16 (mask = the layer input, post ReLU and dropout);
 // db[k] = sum_b dx[b][k] (of the bf16-rounded values: the bias gradient of the layer below), when db != nullptr.
-// grid: K/32 blocks of 256 threads = 32 columns x 8 row lanes.
-__global__ void __launch_bounds__(256) fc_reduce_bwd_kernel(const float* __restrict__ ws, int splits, long long split_stride,
-                                                            const __nv_bfloat16* __restrict__ mask, float scale, int B, int K,
-                                                            __nv_bfloat16* __restrict__ out, float* __restrict__ db) {
-    __shared__ float red[8][33];
+// grid: K/32 blocks of 1024 threads = 32 columns x 32 row lanes.
+__global__ void __launch_bounds__(1024) fc_reduce_bwd_kernel(const float* __restrict__ ws, int splits, long long split_stride,
+                                                             const __nv_bfloat16* __restrict__ mask, float scale, int B, int K,
+                                                             __nv_bfloat16* __restrict__ out, float* __restrict__ db) {
+    __shared__ float red[32][33];
     const int c = blockIdx.x * 32 + (threadIdx.x & 31), rl = threadIdx.x >> 5;
     float acc = 0.f;
     if (c < K) {
-        for (int b = rl; b < B; b += 8) {
+        for (int b = rl; b < B; b += 32) {
             const size_t t = (size_t)b * K + c;
             float v = 0.f;
             for (int z = 0; z < splits; ++z) v += ws[z * split_stride + t];
@@ -272,7 +354,7 @@ __global__ void __launch_bounds__(256) fc_reduce_bwd_kernel(const float* __restr
     if (threadIdx.x < 32 && c < K) {
         float s = 0.f;
         #pragma unroll
-        for (int q = 0; q < 8; ++q) s += red[q][threadIdx.x];
+        for (int q = 0; q < 32; ++q) s += red[q][threadIdx.x];
         db[c] = s;
     }
 }

@@ -646,8 +646,12 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 const int m0 = tc.m_tile * (128 * MH), n0 = tc.n_tile * BN;
                 const int a_begin = tc.z * per;
                 const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
-                int ky = 0, ch = a_begin;
-                if (p.chunks < p.asteps_total && a_begin > 0) { ky = a_begin / p.chunks; ch = a_begin - ky * p.chunks; }
+                // the reduction order is free: every CTA starts at a different (filter row, chunk) so that the SMs do not
+                // all ask L2 for the same weight tile at the same moment
+                const int a_end = a_begin + nsteps;
+                int a = a_begin + (int)(blockIdx.x % (unsigned)nsteps);
+                int ky = a / p.chunks, ch = a - ky * p.chunks;
+                const int ky0 = a_begin / p.chunks, ch0 = a_begin - ky0 * p.chunks;
                 const int xa = p.a_x0 + tc.g * p.a_gx, yb = tc.g * p.b_g_rows + n0;
                 for (int i = 0; i < nsteps && ok; ++i) {
                     if (!(ok = mbar_wait(emptyA + 8u * sa, pha ^ 1u, abort_flag))) break;
@@ -667,7 +671,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                         tma_load_2d(ring_b + sb * b_bytes, &p.tmB, ch * 64, brow, fb);
                         if (++sb == b_stages) { sb = 0; phb ^= 1u; }
                     }
-                    if (++ch == p.chunks) { ch = 0; ++ky; }
+                    if (++a == a_end) { a = a_begin; ky = ky0; ch = ch0; } else if (++ch == p.chunks) { ch = 0; ++ky; }
                 }
             }
         }
