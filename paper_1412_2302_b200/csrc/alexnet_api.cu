@@ -310,12 +310,14 @@ ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, in
         for (int BN = 16; BN <= 256 && BN <= N; BN += 16) {
             if (N % BN) continue;
             if (MH * BN > 512) continue;
-            if (2 * (size_t)MH * a_rows * 128 + 4 * (size_t)BN * 128 > budget) continue;
+            if (2 * (size_t)MH * a_rows * 128 + 2 * (size_t)std::min(kw, 3) * BN * 128 > budget) continue;
             const int acc = 2 * MH * BN <= 512 ? 2 : 1;
             const long long tiles = ((M + 128 * MH - 1) / (128 * MH)) * (N / BN) * groups;
             const long long rounds = (tiles + h->sm_count - 1) / h->sm_count;
-            // per weight stage: the pipe needs MH*kk*BN/2 cycles, each issuer about 105 cycles per instruction
-            const double mma = kw * kk * std::max(MH * BN / 2.0, 105.0);
+            // per filter row and chunk: the pipe needs kw*kk*MH*BN/2 cycles; each issuer warp pays about 330 cycles per
+            // loop trip plus 50 per instruction (measured); TMA brings about 72 bytes per cycle
+            const int ngroups = kw <= 3 ? 1 : (kw + 2) / 3;
+            const double mma = std::max(kw * kk * MH * BN / 2.0, ngroups * 330.0 + kw * kk * 50.0);
             const double tma = ((double)MH * a_rows * 128 + (double)kw * BN * 128) / 72.0;
             double tile_t = (double)kh * chunks * std::max(mma, tma) + 800.0;
             const double epi = MH * (BN / 16) * 170.0;
@@ -335,14 +337,15 @@ void finish_conv_plan(const alexnet* h, Plan& P) {
     c.tiles_total = c.m_tiles * c.n_tiles * c.groups * c.splits;
     const size_t a_bytes = (size_t)c.MH * c.a_box_rows * 128, b_bytes = (size_t)c.BN * 128;
     const size_t budget = 227 * 1024 - 2048 - 4 * tc::kEpiStageBytes;
+    c.tpg = c.kw <= 3 ? c.kw : 3;               // weight tiles travel in groups: a filter row, or 3 + 2 taps of a five-tap row
+    const size_t g_bytes = b_bytes * c.tpg;
     if (c.kw == 1) {
-        int st = (int)(budget / (a_bytes + b_bytes));
+        int st = (int)(budget / (a_bytes + g_bytes));
         st = std::min(st, 8);
         c.a_stages = c.b_stages = st;
     } else {
-        c.a_stages = 3;
-        if (budget < 3 * a_bytes + 4 * b_bytes) c.a_stages = 2;
-        c.b_stages = (int)std::min<size_t>(8, (budget - c.a_stages * a_bytes) / b_bytes);
+        c.a_stages = (budget >= 3 * a_bytes + 2 * g_bytes) ? 3 : 2;
+        c.b_stages = (int)std::min<size_t>(8, (budget - c.a_stages * a_bytes) / g_bytes);
     }
     P.conv = true;
     P.smem = tc::conv_smem_bytes(c);

@@ -153,7 +153,7 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src
                  ::"l"(tm), "r"(src), "r"(x), "r"(y), "r"(z) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
@@ -248,9 +248,10 @@ __device__ __forceinline__ void epi_chunk(const P& p, uint32_t* v, bool zero, bo
 
 // Staged epilogue: one warp turns 32 accumulator rows x one 128-byte slab (64 bf16 or 32 fp32 columns) into a
 // 128-byte-swizzled 4 KB tile in shared memory and stores it with one TMA box; rows and columns outside the output
-// tensor are clipped by TMA.  kEpiStageBytes per warp holds two such tiles, used alternately: before a tile is
-// rewritten the store issued from it two slabs earlier must have finished reading (wait_group.read 1).
-constexpr uint32_t kEpiStageBytes = 8192;
+// tensor are clipped by TMA.  Each epilogue warp owns one kEpiStageBytes tile: before rewriting it the warp waits
+// until the previous store has finished reading it (wait_group.read 0), which the TMEM loads and the arithmetic of
+// the next slab overlap.
+constexpr uint32_t kEpiStageBytes = 4096;
 template <typename P>
 __device__ __forceinline__ void epi_slab(const P& p, uint32_t tmem_addr, bool pad_row, long long row_off, int col0, int g,
                                          int x, int y, int z, uint32_t stage, int lane) {
@@ -298,7 +299,7 @@ __device__ __forceinline__ void epi_slab(const P& p, uint32_t tmem_addr, bool pa
             }
         }
     }
-    if (lane == 0) bulk_wait_read_1();
+    if (lane == 0) bulk_wait_read_0();
     __syncwarp();
     const uint32_t rowp = stage + (uint32_t)lane * 128u;
     #pragma unroll
@@ -470,7 +471,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         const int r = quad * 32 + lane;          // row within the tile = TMEM lane
         TileCursor tc; tc.init(p);
         int ab = 0; uint32_t aph = 0;
-        int sbuf = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
             const int m0 = tc.m_tile * 128, n0 = tc.n_tile * p.BN, g = tc.g;
@@ -499,8 +499,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 for (int c = 0; c < p.BN; c += slab) {
                     epi_slab(p, t0 + (uint32_t)c, pad_row, row_off, n0 + c, g, g * p.out_gx * (p.mode != MODE_MNMN) + n0 + c,
                              m0 + quad * 32 + (p.mode == MODE_MNMN ? g * p.out_gx : 0), tc.z,
-                             epi_stage0 + (uint32_t)quad * kEpiStageBytes + (uint32_t)sbuf * 4096u, lane);
-                    sbuf ^= 1;
+                             epi_stage0 + (uint32_t)quad * kEpiStageBytes, lane);
                 }
             } else {
                 for (int c = 0; c < p.BN; c += 16) {
@@ -558,10 +557,11 @@ struct ConvParams {
     int MH;             // 128-row halves per tile (1, 2 or 4)
     int BN, kk;         // MMA N (multiple of 16, <= 256); K=16 MMAs per weight stage (<= 4)
     int kh, kw;         // filter rows; taps per filter row
+    int tpg;            // taps per weight group (one barrier pair per group): kw, or 3 for a five-tap row (groups 3 + 2)
     int chunks;         // 64-channel chunks
     int asteps_total;   // kh * chunks, split evenly over `splits`
     int asteps_per_split;
-    int a_stages, b_stages, acc_stages;
+    int a_stages, b_stages, acc_stages;   // b_stages counts groups of kw weight tiles (one barrier pair per group)
     int a_box_rows;     // rows per activation box (128, or 136 when kw > 1)
     int a_x0, a_gx;     // A column origin and per-group column stride
     int b_tap_rows, b_g_rows;   // B row = (ky*kw+kx)*b_tap_rows + g*b_g_rows + n0
@@ -581,7 +581,7 @@ struct ConvParams {
 constexpr int kConvMaxThreads = 32 * 9;
 inline int conv_threads(const ConvParams& p) { return 32 * (5 + p.MH); }
 inline size_t conv_smem_bytes(const ConvParams& p) {
-    return 1024 + (size_t)p.a_stages * p.MH * p.a_box_rows * 128 + (size_t)p.b_stages * p.BN * 128 + 4 * kEpiStageBytes + 512;
+    return 1024 + (size_t)p.a_stages * p.MH * p.a_box_rows * 128 + (size_t)p.b_stages * p.tpg * p.BN * 128 + 4 * kEpiStageBytes + 512;
 }
 
 // tile cursor shared by the roles (m fastest, then n tile, group, split)
@@ -605,6 +605,19 @@ struct ConvCursor {
     }
 };
 
+// MMAs of one filter row (KW taps x KK K=16 steps) on one accumulator, fully unrolled; descriptors in 16-byte units
+template <int KW, int KK>
+__device__ __forceinline__ void issue_row(uint32_t d, uint64_t ad, uint64_t bd, uint32_t b_tile16, const int* tap_off,
+                                          uint32_t idesc, uint32_t accum) {
+    #pragma unroll
+    for (int kx = 0; kx < KW; ++kx) {
+        const uint64_t a_tap = ad + (uint64_t)(tap_off[kx] * 8);      // one row = 128 bytes = 8 units
+        #pragma unroll
+        for (int j = 0; j < KK; ++j)
+            umma(d, a_tap + (uint64_t)(2 * j), bd + (uint64_t)(kx * b_tile16 + 2 * j), idesc, (kx == 0 && j == 0) ? accum : 1u);
+    }
+}
+
 __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_constant__ ConvParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -615,7 +628,8 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     const uint32_t ring_a = base, ring_b = base + a_stages * a_bytes;
     // epilogue staging (4 warps x kEpiStageBytes), then barriers: fullA[8] @0, emptyA[8] @64, fullB[8] @128,
     // emptyB[8] @192, acc_full[2] @256, acc_empty[2] @272, tmem slot @288, abort flag @296
-    const uint32_t epi_stage0 = ring_b + b_stages * b_bytes;
+    const uint32_t g_bytes = b_bytes * (uint32_t)p.tpg;         // one group slot holds up to tpg weight tiles of a filter row
+    const uint32_t epi_stage0 = ring_b + b_stages * g_bytes;
     const uint32_t bar_base = epi_stage0 + 4u * kEpiStageBytes;
     uint8_t* gen = smem_raw + (bar_base - raw);
     volatile int* abort_flag = (volatile int*)(gen + 296);
@@ -671,11 +685,13 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                     }
                     if (++sa == a_stages) { sa = 0; pha ^= 1u; }
                     int brow = ky * kw * p.b_tap_rows + yb;
-                    for (int kx = 0; kx < kw; ++kx, brow += p.b_tap_rows) {
+                    for (int kx0 = 0; kx0 < kw; kx0 += p.tpg) {
                         if (!(ok = mbar_wait(emptyB + 8u * sb, phb ^ 1u, abort_flag))) break;
-                        const uint32_t fb = fullB + 8u * sb;
-                        mbar_expect_tx(fb, b_bytes);
-                        tma_load_2d(ring_b + sb * b_bytes, &p.tmB, ch * 64, brow, fb);
+                        const uint32_t fb = fullB + 8u * sb, dst = ring_b + sb * g_bytes;
+                        const int taps = min(p.tpg, kw - kx0);
+                        mbar_expect_tx(fb, (uint32_t)taps * b_bytes);
+                        for (int t = 0; t < taps; ++t, brow += p.b_tap_rows)
+                            tma_load_2d(dst + t * b_bytes, &p.tmB, ch * 64, brow, fb);
                         if (++sb == b_stages) { sb = 0; phb ^= 1u; }
                     }
                     if (++a == a_end) { a = a_begin; ky = ky0; ch = ch0; } else if (++ch == p.chunks) { ch = 0; ++ky; }
@@ -704,15 +720,23 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 uint32_t accum = 0;
                 for (int i = 0; i < nsteps && ok; ++i) {
                     if (!(ok = mbar_wait_warp(fullA + 8u * sa, pha, abort_flag))) break;
-                    const uint32_t a_half = ring_a + sa * a_bytes + (uint32_t)h * 16384u;
-                    for (int kx = 0; kx < kw; ++kx) {
+                    const uint64_t ad = dbase + (uint64_t)((ring_a + sa * a_bytes + (uint32_t)h * 16384u) >> 4);
+                    // the MMAs of a weight group in straight-line code: the fixed cost of a loop trip with a barrier wait
+                    // (a few hundred cycles) is paid once per taps*kk instructions
+                    for (int kx0 = 0; kx0 < kw; kx0 += p.tpg) {
                         if (!(ok = mbar_wait_warp(fullB + 8u * sb, phb, abort_flag))) break;
-                        tc_fence_after();
-                        const uint64_t bd = dbase + (uint64_t)((ring_b + sb * b_bytes) >> 4);
-                        const uint64_t ad = dbase + (uint64_t)((a_half + (uint32_t)p.tap_off[kx] * 128u) >> 4);
-                        #pragma unroll 4
-                        for (int j = 0; j < kk; ++j)
-                            umma(d, ad + (uint64_t)(2 * j), bd + (uint64_t)(2 * j), idesc, accum | (uint32_t)j);
+                        const uint64_t bd = dbase + (uint64_t)((ring_b + sb * g_bytes) >> 4);
+                        const int taps = min(p.tpg, kw - kx0);
+                        const int* toff = p.tap_off + kx0;
+                        if (kk == 4) {
+                            if (taps == 3) issue_row<3, 4>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            else if (taps == 2) issue_row<2, 4>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            else issue_row<1, 4>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                        } else {
+                            if (taps == 3) issue_row<3, 3>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            else if (taps == 2) issue_row<2, 3>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            else issue_row<1, 3>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                        }
                         accum = 1;
                         umma_commit(emptyB + 8u * sb);
                         if (++sb == b_stages) { sb = 0; phb ^= 1u; }
@@ -734,7 +758,6 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         const int r = quad * 32 + lane;          // row within a 128-row half = TMEM lane
         ConvCursor tc; tc.init(p);
         int ab = 0; uint32_t aph = 0;
-        int sbuf = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
             const int m0 = tc.m_tile * (128 * MH), n0 = tc.n_tile * BN, g = tc.g;
@@ -757,8 +780,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                     const int slab = p.epi == EPI_F32 ? 32 : 64;
                     for (int c = 0; c < BN; c += slab) {
                         epi_slab(p, t0 + (uint32_t)c, pad_row, row_off, n0 + c, g, g * p.out_gx + n0 + c, m0 + h * 128 + quad * 32,
-                                 tc.z, epi_stage0 + (uint32_t)quad * kEpiStageBytes + (uint32_t)sbuf * 4096u, lane);
-                        sbuf ^= 1;
+                                 tc.z, epi_stage0 + (uint32_t)quad * kEpiStageBytes, lane);
                     }
                 } else {
                     for (int c = 0; c < BN; c += 16) {
