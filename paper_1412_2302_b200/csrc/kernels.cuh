@@ -282,27 +282,59 @@ __global__ void __launch_bounds__(256) pool_lrn_bwd_kernel(const __nv_bfloat16* 
                                                            const uint8_t* __restrict__ arg, __nv_bfloat16* __restrict__ da,
                                                            int cpr, int ppb, int Hpi, int Wpi, int Hi, int Wi, int Ho, int Wo,
                                                            int Hpo, int Wpo, float alpha, float beta, float k) {
-    __shared__ uint4 dn[256];
+    __shared__ float4 edge[256];      // tt of the two lowest and two highest channels of every thread, for its neighbours
     const int px = threadIdx.x / cpr, ch = threadIdx.x - px * cpr;
     const int x = blockIdx.x * ppb + px, y = blockIdx.y, n = blockIdx.z;
     const bool active = px < ppb && x < Wpi;
-    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    if (active && y < Hi && x < Wi) pool_bwd8(dp, arg, acc, n, y, x, ch, cpr, Ho, Wo, Hpo, Wpo);
-    dn[threadIdx.x] = pack8(acc);
+    const bool valid = active && y < Hi && x < Wi;         // pad pixels of the grid: da = 0
+    const size_t t = ((size_t)(n * Hpi + y) * Wpi + x) * cpr + ch;
+    // this thread's 8 channels: dn (bf16-rounded, as pool_bwd_kernel stores it), s^-beta and tt = dn a s^(-beta-1);
+    // s needs a of channels c0-2 .. c0+9, read from the neighbouring 16-byte vectors
+    float fa[24], g8[8], sp[8], tt[8];
+    if (valid) {
+        float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        pool_bwd8(dp, arg, acc, n, y, x, ch, cpr, Ho, Wo, Hpo, Wpo);
+        unpack8(pack8(acc), g8);
+        const uint4* ap = (const uint4*)a + t;
+        const uint4 zero = make_uint4(0, 0, 0, 0);
+        unpack8(ch > 0 ? __ldg(ap - 1) : zero, fa);
+        unpack8(__ldg(ap), fa + 8);
+        unpack8(ch < cpr - 1 ? __ldg(ap + 1) : zero, fa + 16);
+        float sq[12];
+        #pragma unroll
+        for (int i = 0; i < 12; ++i) sq[i] = fa[6 + i] * fa[6 + i];
+        #pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float ss = (sq[i] + sq[i + 1]) + (sq[i + 2] + sq[i + 3]) + sq[i + 4];
+            float rs;
+            pow_neg(fmaf(alpha, ss, k), beta, sp[i], rs);
+            tt[i] = g8[i] * fa[8 + i] * sp[i] * rs;
+        }
+    } else {
+        #pragma unroll
+        for (int i = 0; i < 8; ++i) tt[i] = 0.f;
+    }
+    edge[threadIdx.x] = make_float4(tt[0], tt[1], tt[6], tt[7]);
     __syncthreads();
     if (!active) return;
-    const size_t t = ((size_t)(n * Hpi + y) * Wpi + x) * cpr + ch;
-    const uint4* ap = (const uint4*)a + t;
-    const uint4 zero = make_uint4(0, 0, 0, 0);
-    const bool has_l = ch > 0, has_r = ch < cpr - 1;
-    float fa[24], fg[24];
-    unpack8(has_l ? __ldg(ap - 1) : zero, fa);
-    unpack8(__ldg(ap), fa + 8);
-    unpack8(has_r ? __ldg(ap + 1) : zero, fa + 16);
-    unpack8(has_l ? dn[threadIdx.x - 1] : zero, fg);
-    unpack8(dn[threadIdx.x], fg + 8);
-    unpack8(has_r ? dn[threadIdx.x + 1] : zero, fg + 16);
-    ((uint4*)da)[t] = lrn_bwd8(fa, fg, alpha, beta, k);
+    if (!valid) { ((uint4*)da)[t] = make_uint4(0, 0, 0, 0); return; }
+    // tt of channels c0-2, c0-1 (left neighbour's two highest) and c0+8, c0+9 (right neighbour's two lowest)
+    float te[12];
+    const float4 l = ch > 0 ? edge[threadIdx.x - 1] : make_float4(0, 0, 0, 0);
+    const float4 r = ch < cpr - 1 ? edge[threadIdx.x + 1] : make_float4(0, 0, 0, 0);
+    te[0] = l.z; te[1] = l.w; te[10] = r.x; te[11] = r.y;
+    #pragma unroll
+    for (int i = 0; i < 8; ++i) te[2 + i] = tt[i];
+    const float c2 = 2.f * alpha * beta;
+    float o[8];
+    #pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float acc = (te[i] + te[i + 1]) + (te[i + 2] + te[i + 3]) + te[i + 4];
+        const float am = fa[8 + i];
+        const float v = fmaf(g8[i], sp[i], -c2 * am * acc);
+        o[i] = am > 0.f ? v : 0.f;
+    }
+    ((uint4*)da)[t] = pack8(o);
 }
 
 // ------------------------------------------------- split-K reductions (FC, wgrad)
