@@ -335,9 +335,10 @@ void finish_conv_plan(const alexnet* h, Plan& P) {
     c.splits = (c.asteps_total + per - 1) / per;
     c.asteps_per_split = per;
     c.tiles_total = c.m_tiles * c.n_tiles * c.groups * c.splits;
-    const size_t a_bytes = (size_t)c.MH * c.a_box_rows * 128, b_bytes = (size_t)c.BN * 128;
+    if (c.cpg < 1) c.cpg = 1;
+    const size_t a_bytes = (size_t)c.MH * c.cpg * c.a_box_rows * 128, b_bytes = (size_t)c.BN * 128;
     const size_t budget = 227 * 1024 - 2048 - 4 * tc::kEpiStageBytes;
-    c.tpg = c.kw <= 3 ? c.kw : 3;               // weight tiles travel in groups: a filter row, or 3 + 2 taps of a five-tap row
+    c.tpg = c.cpg > 1 ? c.cpg : (c.kw <= 3 ? c.kw : 3);   // weight tiles travel in groups: a filter row (3 + 2 taps of a five-tap row), or the chunks of an FC stage
     const size_t g_bytes = b_bytes * c.tpg;
     if (c.kw == 1) {
         int st = (int)(budget / (a_bytes + g_bytes));
@@ -451,13 +452,13 @@ int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* ws
     memset(&P, 0, sizeof(P));
     tc::ConvParams& p = P.c;
     const int B = h->B;
-    p.kh = p.kw = 1; p.chunks = f.K / 64; p.kk = 4;
+    p.kh = p.kw = 1; p.cpg = 2; p.chunks = f.K / 64 / p.cpg; p.kk = 4;   // K is a multiple of 128 in all three layers
     p.MH = 1; p.BN = fc_fwd_bn(f); p.acc_stages = 2;
     p.M_total = B; p.m_tiles = (B + 127) / 128; p.n_tiles = (f.N + p.BN - 1) / p.BN;
     p.groups = 1; p.splits = fc_fwd_splits(f, B);
     p.asteps_total = p.chunks;
     p.a_box_rows = 128;
-    p.halo_shift[0] = 0; p.tap_off[0] = 0;
+    p.halo_shift[0] = 0; p.tap_off[0] = 0; p.tap_off[1] = 128;   // the second chunk's box follows the first in the stage
     p.epi = tc::EPI_F32; p.n_valid = f.N; p.ldo = f.N; p.split_stride = (long long)B * f.N;
     p.mask_scale = 1.f; p.out = h->ws; p.status = h->status;
     int rc;

@@ -568,6 +568,8 @@ struct ConvParams {
     int MH;             // 128-row halves per tile (1, 2 or 4)
     int BN, kk;         // MMA N (multiple of 16, <= 256); K=16 MMAs per weight stage (<= 4)
     int kh, kw;         // filter rows; taps per filter row
+    int cpg;            // 64-channel chunks per A stage: 1 for convolutions; 2 for FC layers (kw = 1), whose A stage then holds
+                        // cpg activation boxes side by side and whose weight group holds the cpg matching weight tiles
     int tpg;            // taps per weight group (one barrier pair per group): kw, or 3 for a five-tap row (groups 3 + 2)
     int chunks;         // 64-channel chunks
     int asteps_total;   // kh * chunks, split evenly over `splits`
@@ -592,7 +594,7 @@ struct ConvParams {
 constexpr int kConvMaxThreads = 32 * 9;
 inline int conv_threads(const ConvParams& p) { return 32 * (5 + p.MH); }
 inline size_t conv_smem_bytes(const ConvParams& p) {
-    return 1024 + (size_t)p.a_stages * p.MH * p.a_box_rows * 128 + (size_t)p.b_stages * p.tpg * p.BN * 128 + 4 * kEpiStageBytes + 512;
+    return 1024 + (size_t)p.a_stages * p.MH * p.cpg * p.a_box_rows * 128 + (size_t)p.b_stages * p.tpg * p.BN * 128 + 4 * kEpiStageBytes + 512;
 }
 
 // tile cursor shared by the roles (m fastest, then n tile, group, split)
@@ -634,7 +636,8 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     const int MH = p.MH, BN = p.BN;
-    const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * 128u, a_bytes = a_box_bytes * MH, b_bytes = (uint32_t)BN * 128u;
+    const int cpg = p.cpg, gw = cpg > 1 ? cpg : p.kw;            // weight tiles per A stage
+    const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * 128u, a_bytes = a_box_bytes * MH * cpg, b_bytes = (uint32_t)BN * 128u;
     const int a_stages = p.a_stages, b_stages = p.b_stages;
     const uint32_t ring_a = base, ring_b = base + a_stages * a_bytes;
     // epilogue staging (4 warps x kEpiStageBytes), then barriers: fullA[8] @0, emptyA[8] @64, fullB[8] @128,
@@ -691,18 +694,20 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                         const uint32_t dst = ring_a + sa * a_bytes, fb = fullA + 8u * sa;
                         const int y = m0 + p.halo_shift[ky];
                         mbar_expect_tx(fb, a_bytes);
-                        for (int h = 0; h < MH; ++h)
-                            tma_load_2d(dst + h * a_box_bytes, &p.tmA, xa + ch * 64, y + h * p.a_box_rows, fb);
+                        for (int c = 0; c < cpg; ++c)
+                            for (int h = 0; h < MH; ++h)
+                                tma_load_2d(dst + (c * MH + h) * a_box_bytes, &p.tmA, xa + (ch * cpg + c) * 64, y + h * p.a_box_rows, fb);
                     }
                     if (++sa == a_stages) { sa = 0; pha ^= 1u; }
-                    int brow = ky * kw * p.b_tap_rows + yb;
-                    for (int kx0 = 0; kx0 < kw; kx0 += p.tpg) {
+                    int brow = ky * kw * p.b_tap_rows + yb, bcol = ch * cpg * 64;
+                    const int brow_step = cpg > 1 ? 0 : p.b_tap_rows, bcol_step = cpg > 1 ? 64 : 0;
+                    for (int kx0 = 0; kx0 < gw; kx0 += p.tpg) {
                         if (!(ok = mbar_wait(emptyB + 8u * sb, phb ^ 1u, abort_flag))) break;
                         const uint32_t fb = fullB + 8u * sb, dst = ring_b + sb * g_bytes;
-                        const int taps = min(p.tpg, kw - kx0);
+                        const int taps = min(p.tpg, gw - kx0);
                         mbar_expect_tx(fb, (uint32_t)taps * b_bytes);
-                        for (int t = 0; t < taps; ++t, brow += p.b_tap_rows)
-                            tma_load_2d(dst + t * b_bytes, &p.tmB, ch * 64, brow, fb);
+                        for (int t = 0; t < taps; ++t, brow += brow_step, bcol += bcol_step)
+                            tma_load_2d(dst + t * b_bytes, &p.tmB, bcol, brow, fb);
                         if (++sb == b_stages) { sb = 0; phb ^= 1u; }
                     }
                     if (++a == a_end) { a = a_begin; ky = ky0; ch = ch0; } else if (++ch == p.chunks) { ch = 0; ++ky; }
@@ -734,10 +739,10 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                     const uint64_t ad = dbase + (uint64_t)((ring_a + sa * a_bytes + (uint32_t)h * 16384u) >> 4);
                     // the MMAs of a weight group in straight-line code: the fixed cost of a loop trip with a barrier wait
                     // (a few hundred cycles) is paid once per taps*kk instructions
-                    for (int kx0 = 0; kx0 < kw; kx0 += p.tpg) {
+                    for (int kx0 = 0; kx0 < gw; kx0 += p.tpg) {
                         if (!(ok = mbar_wait_warp(fullB + 8u * sb, phb, abort_flag))) break;
                         const uint64_t bd = dbase + (uint64_t)((ring_b + sb * g_bytes) >> 4);
-                        const int taps = min(p.tpg, kw - kx0);
+                        const int taps = min(p.tpg, gw - kx0);
                         const int* toff = p.tap_off + kx0;
                         if (kk == 4) {
                             if (taps == 3) issue_row<3, 4>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
