@@ -119,7 +119,10 @@ int alexnet_set_params(alexnet_t* h, int replica, int which, const float* host_i
 /* Debug / parity access to intermediate tensors of the last step of a replica,
  * converted to fp32 in canonical NCHW (or [B][N]) order.  alexnet_tensor_size
  * gives the element count.  set_tensor writes a tensor (rounded to its device
- * type) so that one operation can be run in isolation by alexnet_run_op. */
+ * type) so that one operation can be run in isolation by alexnet_run_op.  The
+ * training step fuses LRN with pooling and does not store the normalised
+ * tensors N1/N2 nor their gradients DN1/DN2; get_tensor recomputes them on
+ * demand with the single-operation kernels (same arithmetic). */
 enum {
     ALEXNET_T_CROPFLIP = 0, /* [B][3]: ox, oy, flip */
     ALEXNET_T_X0, ALEXNET_T_A1, ALEXNET_T_N1, ALEXNET_T_P1, ALEXNET_T_ARG1,

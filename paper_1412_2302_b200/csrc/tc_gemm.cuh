@@ -5,9 +5,13 @@
 // swizzle) through a ring of `stages` buffers; fp32 accumulators live in tensor
 // memory, double buffered, so the epilogue of tile i overlaps the main loop of
 // tile i+1.  Warp roles: warp 0 = TMA producer (one lane), warp 1 = MMA issuer
-// (one lane) and TMEM owner, warps 2..5 = epilogue (each reads the 32 TMEM
-// lanes of its quadrant).  The single-lane loops carry no division or modulo:
-// stage, phase, tap and chunk counters advance incrementally.
+// (the whole warp runs the loop, an elected lane issues) and TMEM owner, warps
+// 2..5 = epilogue (each reads the 32 TMEM lanes of its quadrant and stores its
+// rows through a swizzled shared-memory tile and TMA).  The producer and issuer
+// loops carry no division or modulo: stage, phase, tap and chunk counters
+// advance incrementally.  This file holds three kernels: gemm_kernel (FC
+// backward), conv_kernel (convolution forward / backward-data, FC forward) and
+// wgrad_kernel (convolution weight gradients).
 // Three operand arrangements:
 //   MODE_KK   A K-major, B K-major   conv fwd, conv bwd-data, FC fwd
 //   MODE_KMN  A K-major, B MN-major  FC bwd-data (weights read untransposed)
