@@ -163,10 +163,11 @@ struct Carver {
     }
 };
 
-int pick_splits(int tiles, int steps, int cap) {
-    int s = (296 + tiles - 1) / tiles;
-    if (s > cap) s = cap;
-    if (s > steps) s = steps;
+// k splits of a GEMM with `tiles` output tiles and `steps` k-steps: fill one wave of 148 CTAs, never more (a second,
+// nearly empty round costs a whole tile time), and keep at least two k-steps per split
+int pick_splits(int tiles, int steps) {
+    int s = 148 / tiles;
+    if (s > steps / 2) s = steps / 2;
     if (s < 1) s = 1;
     return s;
 }
@@ -183,11 +184,11 @@ int conv_wg_splits(const ConvL& c, int B, int sm_count = 148) {
 int fc_fwd_bn(const FcL&) { return 128; }
 int fc_fwd_splits(const FcL& f, int B) {
     const int tiles = ((B + 127) / 128) * ((f.N + 127) / 128);
-    return pick_splits(tiles, f.K / 64, 16);
+    return pick_splits(tiles, f.K / 128);    // k-steps of two 64-channel chunks
 }
 int fc_bwd_splits(const FcL& f, int B) {
     const int tiles = ((B + 127) / 128) * (f.K / 256);
-    return pick_splits(tiles, (f.N + 63) / 64, 16);
+    return pick_splits(tiles, (f.N + 63) / 64);
 }
 size_t ws_need(const Layout& L, int B) {
     size_t need = 0;
@@ -705,10 +706,10 @@ void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
 void op_update(alexnet* h, int r, cudaStream_t st) {
     Replica& R = h->rep[r];
     const long long nd = (h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES) ? h->L.n_total : h->L.n_weights;
+    // all conv filters precede the FC weights in the internal order
     kn::sgd_update_kernel<<<1184, 256, 0, st>>>(R.w, R.v, R.g, R.shadow, h->L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum,
-                                                h->cfg.weight_decay);
+                                                h->cfg.weight_decay, R.wt, h->L.tjobs, h->L.fc[0].w_off / 4);
     h->launches++;
-    refresh_shadows(h, r, false, st);
 }
 void op_average(alexnet* h, cudaStream_t st) {
     Replica &A = h->rep[0], &Bq = h->rep[1];

@@ -501,10 +501,17 @@ __global__ void mean_kernel(const float* __restrict__ v, int n, float* __restric
 }
 
 // ------------------------------------------------ momentum update and average
+// transposed bf16 copies of the grouped conv filters for the backward-data pass:
+// wt[tap][g*cig + ci][co'] = wf[tap][g*cog + co'][ci]
+struct TransposeJob { long long src_off, dst_off; int taps, cout, cig, groups; long long count; };
+struct TransposeJobs { TransposeJob j[4]; int n; };
 // v <- mu v - lr wd w [i < n_decay] - lr g ; w <- w + v ; bf16 shadow of w.  22 bytes per parameter.
+// The conv filters of layers 2-5 (the first conv_end4 vectors hold all conv filters) are also written to their
+// transposed bf16 copies for the backward-data pass, so no separate transposition pass is needed after a step.
 __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g,
                                   __nv_bfloat16* __restrict__ shadow, long long n4, long long n_decay4,
-                                  float lr, float mu, float wd) {
+                                  float lr, float mu, float wd, __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs,
+                                  long long conv_end4) {
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
         float4 wv = ((float4*)w)[i], vv = ((float4*)v)[i];
@@ -518,6 +525,21 @@ __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, 
         ((float4*)v)[i] = vv;
         __nv_bfloat162 lo = __floats2bfloat162_rn(wv.x, wv.y), hi = __floats2bfloat162_rn(wv.z, wv.w);
         ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
+        if (i < conv_end4) {
+            const long long e = 4 * i;
+            for (int q = 0; q < jobs.n; ++q) {
+                const TransposeJob J = jobs.j[q];
+                const long long sidx = e - J.src_off;          // [tap][cout][cig], four consecutive ci
+                if (sidx < 0 || sidx >= J.count) continue;
+                const int cog = J.cout / J.groups;
+                const int ci = (int)(sidx % J.cig);
+                const long long r = sidx / J.cig;
+                const int co = (int)(r % J.cout), tap = (int)(r / J.cout);
+                const int grp = co / cog, co_ = co - grp * cog;
+                __nv_bfloat16* dst = wt + J.dst_off + ((long long)tap * J.cig * J.groups + grp * J.cig + ci) * cog + co_;
+                dst[0] = lo.x; dst[cog] = lo.y; dst[2 * cog] = hi.x; dst[3 * cog] = hi.y;   // cig is a multiple of 4
+            }
+        }
     }
 }
 // exchange-and-average with both replicas in one HBM: w_a = w_b = (w_a+w_b)/2, same for momentum; refresh both shadows.
@@ -546,10 +568,6 @@ __global__ void shadow_kernel(const float* __restrict__ w, __nv_bfloat16* __rest
     }
 }
 
-// transposed bf16 copies of the grouped conv filters for the backward-data pass:
-// wt[tap][g*cig + ci][co'] = wf[tap][g*cog + co'][ci]
-struct TransposeJob { long long src_off, dst_off; int taps, cout, cig, groups; long long count; };
-struct TransposeJobs { TransposeJob j[4]; int n; };
 __global__ void conv_transpose_shadow_kernel(const __nv_bfloat16* __restrict__ shadow, __nv_bfloat16* __restrict__ wt,
                                              const TransposeJobs jobs) {
     const long long stride = (long long)gridDim.x * blockDim.x;
