@@ -561,7 +561,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 // One thread issues a tcgen05.mma roughly every 100 cycles, which is slower
 // than the tensor pipe for N < 192; so each 128-row half has its own issuer
 // warp (they write disjoint accumulators) and the pipe stays fed.
-// Warps: 0 = TMA producer, 1..MH = MMA issuers, MH+1..MH+4 = epilogue.
+// Warps: 0 and 1 = TMA producers (halos, weight groups), 2..MH+1 = MMA issuers, then four epilogue warps.
 // Accumulators: MH x BN columns per buffer, two buffers when they fit in the
 // 512 TMEM columns.
 struct ConvParams {
@@ -595,8 +595,8 @@ struct ConvParams {
     int* status;
 };
 
-constexpr int kConvMaxThreads = 32 * 9;
-inline int conv_threads(const ConvParams& p) { return 32 * (5 + p.MH); }
+constexpr int kConvMaxThreads = 32 * 10;
+inline int conv_threads(const ConvParams& p) { return 32 * (6 + p.MH); }
 inline size_t conv_smem_bytes(const ConvParams& p) {
     return 1024 + (size_t)p.a_stages * p.MH * p.cpg * p.a_box_rows * 128 + (size_t)p.b_stages * p.tpg * p.BN * 128 + 4 * kEpiStageBytes + 512;
 }
@@ -668,7 +668,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         tma_prefetch_desc(&p.tmA);
         tma_prefetch_desc(&p.tmB);
     }
-    if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), ncols);
+    if (warp == 2) tmem_alloc(smem_u32((const void*)tmem_slot), ncols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -676,13 +676,14 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     const int per = p.asteps_per_split, kw = p.kw;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ TMA producers: lane 0 of warp 0 feeds the ring of
+        // activation halos, lane 0 of warp 1 the ring of weight groups, so that neither ring waits for the other
         if (lane == 0) {
             ConvCursor tc; tc.init(p);
-            int sa = 0, sb = 0; uint32_t pha = 0, phb = 0;
+            int sa = 0; uint32_t pha = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
-                const int m0 = tc.m_tile * (128 * MH), n0 = tc.n_tile * BN;
+                const int m0 = tc.m_tile * (128 * MH);
                 const int a_begin = tc.z * per;
                 const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
                 // the reduction order is free: every CTA starts at a different (filter row, chunk) so that the SMs do not
@@ -691,7 +692,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 int a = a_begin + (int)(blockIdx.x % (unsigned)nsteps);
                 int ky = a / p.chunks, ch = a - ky * p.chunks;
                 const int ky0 = a_begin / p.chunks, ch0 = a_begin - ky0 * p.chunks;
-                const int xa = p.a_x0 + tc.g * p.a_gx, yb = tc.g * p.b_g_rows + n0;
+                const int xa = p.a_x0 + tc.g * p.a_gx;
                 for (int i = 0; i < nsteps && ok; ++i) {
                     if (!(ok = mbar_wait(emptyA + 8u * sa, pha ^ 1u, abort_flag))) break;
                     {
@@ -703,6 +704,27 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                                 tma_load_2d(dst + (c * MH + h) * a_box_bytes, &p.tmA, xa + (ch * cpg + c) * 64, y + h * p.a_box_rows, fb);
                     }
                     if (++sa == a_stages) { sa = 0; pha ^= 1u; }
+                    if (++a == a_end) { a = a_begin; ky = ky0; ch = ch0; } else if (++ch == p.chunks) { ch = 0; ++ky; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            ConvCursor tc; tc.init(p);
+            int sb = 0; uint32_t phb = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
+                const int n0 = tc.n_tile * BN;
+                const int a_begin = tc.z * per;
+                const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
+                // the reduction order is free: every CTA starts at a different (filter row, chunk) so that the SMs do not
+                // all ask L2 for the same weight tile at the same moment
+                const int a_end = a_begin + nsteps;
+                int a = a_begin + (int)(blockIdx.x % (unsigned)nsteps);
+                int ky = a / p.chunks, ch = a - ky * p.chunks;
+                const int ky0 = a_begin / p.chunks, ch0 = a_begin - ky0 * p.chunks;
+                const int yb = tc.g * p.b_g_rows + n0;
+                for (int i = 0; i < nsteps && ok; ++i) {
                     int brow = ky * kw * p.b_tap_rows + yb, bcol = ch * cpg * 64;
                     const int brow_step = cpg > 1 ? 0 : p.b_tap_rows, bcol_step = cpg > 1 ? 64 : 0;
                     for (int kx0 = 0; kx0 < gw; kx0 += p.tpg) {
@@ -718,10 +740,10 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 }
             }
         }
-    } else if (warp <= MH) {
+    } else if (warp <= MH + 1) {
         // ------------------------------------------------------------ MMA issuer of row half h (whole warp)
         {
-            const int h = warp - 1;
+            const int h = warp - 2;
             const uint32_t idesc = instr_desc(BN, 0, 0);
             const uint64_t dbase = smem_desc(0, 16, 1024);
             const int kk = p.kk;
@@ -826,7 +848,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         while (clock64() - t0 < 2000000LL) { }
         __syncthreads();
     }
-    if (warp == 1) {
+    if (warp == 2) {
         tc_fence_after();
         tmem_dealloc(tmem, ncols);
     }
