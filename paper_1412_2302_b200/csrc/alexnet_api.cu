@@ -174,7 +174,7 @@ int pick_splits(int tiles, int steps) {
 int conv_wg_splits(const ConvL& c, int B, int sm_count = 148) {
     // one wave: (filter rows x 64-channel input blocks x 128-channel output blocks x groups) units times the row splits
     const long long M = (long long)B * c.gin.Hp * c.gin.Wp;
-    const int steps = (int)((M + 63) / 64);
+    const int steps = (int)((M + tc::kWgRows - 1) / tc::kWgRows);
     const int units = ((c.cog + 127) / 128) * ((c.cig + 63) / 64) * c.groups * c.k;
     int s = sm_count / units;
     if (s > steps) s = steps;
@@ -425,7 +425,7 @@ int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16
     tc::WgradParams& p = P.w;
     const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
     p.m_tiles = (c.cog + 127) / 128; p.n_tiles = (c.cig + 63) / 64; p.groups = c.groups; p.kh = c.k; p.kw = c.k;
-    p.steps_total = (int)((M + 63) / 64);
+    p.steps_total = (int)((M + tc::kWgRows - 1) / tc::kWgRows);
     p.splits = conv_wg_splits(c, h->B, std::min(h->sm_count, 148));   // never more than the workspace was sized for
     p.steps_per_split = (p.steps_total + p.splits - 1) / p.splits;
     p.splits = (p.steps_total + p.steps_per_split - 1) / p.steps_per_split;
@@ -441,8 +441,8 @@ int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16
     p.out = h->ws; p.status = h->status;
     p.bias_partial = h->cs_partial; p.bias_ld = c.cout;
     int rc;
-    if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, 64))) return rc;
-    if ((rc = make_tm(h, &p.tmB, xin, c.cin, M, (uint64_t)c.cin * 2, 72))) return rc;
+    if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, tc::kWgRows))) return rc;
+    if ((rc = make_tm(h, &p.tmB, xin, c.cin, M, (uint64_t)c.cin * 2, tc::kWgRows + 8))) return rc;
     P.wgrad = true;
     P.smem = tc::wgrad_smem_bytes(p);
     P.grid = p.tiles_total;

@@ -873,7 +873,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
 // adds the splits in a fixed order.
 // Warps: 0 = TMA producer, 1..NI = MMA issuers, NI+1..NI+4 = epilogue.
 struct WgradParams {
-    CUtensorMap tmA, tmB;       // dy [M][cout] box {64, 64}; x [M][cin] box {64, 72}
+    CUtensorMap tmA, tmB;       // dy [M][cout] box {64, kWgRows}; x [M][cin] box {64, kWgRows + 8}
     int m_tiles, n_tiles, groups, kh, splits;   // tile decomposition (m fastest, then n, group, ky, split)
     int tiles_total;
     int kw;                     // taps per filter row
@@ -893,7 +893,8 @@ struct WgradParams {
     int bias_ld;                // output channels over all groups
     int* status;
 };
-constexpr int kWgABytes = 16384, kWgBBytes = 72 * 128;
+constexpr int kWgRows = 128;                           // rows of the flat grid per step: 8 MMAs (K = 16 each) per barrier wait
+constexpr int kWgABytes = 2 * kWgRows * 128, kWgBBytes = (kWgRows + 8) * 128;
 inline int wgrad_threads(const WgradParams& p) { return 32 * (5 + p.NI); }
 inline size_t wgrad_smem_bytes(const WgradParams& p) { return 1024 + (size_t)p.stages * (kWgABytes + kWgBBytes) + 4096 + 256; }
 
@@ -951,10 +952,10 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
             for (int i = 0; i < nsteps; ++i) {
                 if (!mbar_wait(empty0 + 8u * st, ph ^ 1u, abort_flag)) break;
                 const uint32_t sa = base + st * stage_bytes, fb = full0 + 8u * st;
-                const int q = (s_begin + i) * 64;
+                const int q = (s_begin + i) * kWgRows;
                 mbar_expect_tx(fb, stage_bytes);
                 tma_load_2d(sa, &p.tmA, xa, q, fb);
-                tma_load_2d(sa + 8192, &p.tmA, xa + 64, q, fb);
+                tma_load_2d(sa + kWgRows * 128, &p.tmA, xa + 64, q, fb);
                 tma_load_2d(sa + kWgABytes, &p.tmB, xb, q + sh, fb);
                 if (++st == stages) { st = 0; ph ^= 1u; }
             }
@@ -964,7 +965,7 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
             const int a = warp - 1;
             const int taps = p.acc_taps[a], kx0 = p.acc_kx0[a];
             const uint32_t idesc = instr_desc(64 * taps, 1, 1);
-            const uint64_t adesc0 = smem_desc(0, 8192, 1024), bdesc0 = smem_desc(0, 128, 1024);
+            const uint64_t adesc0 = smem_desc(0, kWgRows * 128, 1024), bdesc0 = smem_desc(0, 128, 1024);
             const uint32_t d = tmem + (uint32_t)(kx0 * 64);
             int st = 0; uint32_t ph = 0;
             bool ok = true;
@@ -975,7 +976,7 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
                 const uint64_t ad = adesc0 + (uint64_t)(sa >> 4);
                 const uint64_t bd = bdesc0 + (uint64_t)((sa + kWgABytes + (uint32_t)kx0 * 128u) >> 4);
                 #pragma unroll
-                for (int j = 0; j < 4; ++j)
+                for (int j = 0; j < kWgRows / 16; ++j)
                     umma(d, ad + (uint64_t)(128 * j), bd + (uint64_t)(128 * j), idesc, (i > 0 || j > 0) ? 1u : 0u);
                 umma_commit(empty0 + 8u * st);
                 if (++st == stages) { st = 0; ph ^= 1u; }
@@ -987,19 +988,19 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
         const int row = m_tile * 128 + quad * 32 + lane;     // output channel within the group
         const bool row_ok = row < p.M_total;
         if (do_bias) {
-            // thread te: eight output channels (16-byte chunk cc of the 128-channel tile) of rows rg*8 .. rg*8+7 of a stage
+            // thread te: eight output channels (16-byte chunk cc of the 128-channel tile) of rows rg*16 .. rg*16+15 of a stage
             const int te = (warp - NI - 1) * 32 + lane, cc = te & 15, rg = te >> 4;
             float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
             int st = 0; uint32_t ph = 0;
             bool ok = true;
             for (int i = 0; i < nsteps; ++i) {
                 if (!(ok = mbar_wait(full0 + 8u * st, ph, abort_flag))) break;
-                const uint32_t a0 = base + st * stage_bytes + (uint32_t)(cc >> 3) * 8192u + (uint32_t)rg * 1024u;
+                const uint32_t a0 = base + st * stage_bytes + (uint32_t)(cc >> 3) * (kWgRows * 128u) + (uint32_t)rg * (kWgRows / 8 * 128u);
                 #pragma unroll
-                for (int rr = 0; rr < 8; ++rr) {
+                for (int rr = 0; rr < kWgRows / 8; ++rr) {
                     uint4 u;
                     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(u.x), "=r"(u.y), "=r"(u.z), "=r"(u.w)
-                                 : "r"(a0 + (uint32_t)rr * 128u + (uint32_t)(((cc & 7) ^ rr) << 4)));
+                                 : "r"(a0 + (uint32_t)rr * 128u + (uint32_t)(((cc & 7) ^ (rr & 7)) << 4)));
                     const __nv_bfloat162* hh = (const __nv_bfloat162*)&u;
                     #pragma unroll
                     for (int k = 0; k < 4; ++k) { const float2 f = __bfloat1622float2(hh[k]); acc[2 * k] += f.x; acc[2 * k + 1] += f.y; }
