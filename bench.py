@@ -134,7 +134,7 @@ def cpu_baseline():
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
-    from paper_1412_2302_b200 import synth
+    from paper_1412_2302_b200 import multi, synth
     from paper_1412_2302_b200.alexnet import AlexNet
 
     torch.cuda.set_device(local_rank)
@@ -144,14 +144,14 @@ def run_ours(args, rank, world, local_rank):
     seed = synth.BASE_SEED + 3
     net = AlexNet(batch=BATCH, replicas=1, seed=seed, mean_image=synth.mean_image(seed), device=str(dev))
     net.set_params(synth.init_params(seed))
-    host = [(torch.from_numpy(synth.images(seed, rank, i, BATCH)).pin_memory(),
-             torch.from_numpy(synth.labels(seed, rank, i, BATCH)).pin_memory()) for i in range(N_POOL)]
+    stream = multi.rank_stream(rank)
+    host = [(torch.from_numpy(synth.images(seed, stream, i, BATCH)).pin_memory(),
+             torch.from_numpy(synth.labels(seed, stream, i, BATCH)).pin_memory()) for i in range(N_POOL)]
     devb = [(a.to(dev), b.to(dev)) for a, b in host]
     cs = net.compute_stream
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        multi.barrier(world)
         torch.cuda.synchronize()
 
     def loop(pool, n, first, want_loss):
@@ -170,11 +170,7 @@ def run_ours(args, rank, world, local_rank):
         loop(pool, args.steps, first, want_loss)
         e1.record(cs)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = t.item()
+        ms = multi.max_over_ranks(e0.elapsed_time(e1), world, dev)
         return ms, net.launch_count - l0
 
     loop(devb, args.warmup, 0, False)
