@@ -311,17 +311,25 @@ ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, in
         for (int BN = 16; BN <= 256 && BN <= N; BN += 16) {
             if (N % BN) continue;
             if (MH * BN > 512) continue;
-            if (2 * (size_t)MH * a_rows * 128 + 2 * (size_t)std::min(kw, 3) * BN * 128 > budget) continue;
+            const size_t g_tiles = kw <= 3 ? kw : 2;     // weight tiles per group (see finish_conv_plan)
+            if (2 * (size_t)MH * a_rows * 128 + 2 * g_tiles * BN * 128 > budget) continue;
             const int acc = 2 * MH * BN <= 512 ? 2 : 1;
             const long long tiles = ((M + 128 * MH - 1) / (128 * MH)) * (N / BN) * groups;
             const long long rounds = (tiles + h->sm_count - 1) / h->sm_count;
             // per filter row and chunk: the pipe needs kw*kk*MH*BN/2 cycles; each issuer warp pays about 330 cycles per
-            // loop trip plus 50 per instruction (measured); TMA brings about 72 bytes per cycle
-            const int ngroups = kw <= 3 ? 1 : (kw + 2) / 3;
-            const double mma = std::max(kw * kk * MH * BN / 2.0, ngroups * 330.0 + kw * kk * 50.0);
+            // weight group plus 50 per instruction; all issuers together get about one instruction per 40 cycles
+            // dispatched (measured: 4 issuers of N = 64 are slower than one of N = 192); TMA brings about 72 B/cycle,
+            // and a ring of only two halos (large MH) cannot hide its latency
+            const int ngroups = kw <= 3 ? 1 : (kw + 1) / 2;
+            const double n_mma = (double)kw * kk;
+            const double mma = std::max(std::max(n_mma * MH * BN / 2.0, ngroups * 330.0 + n_mma * 50.0), n_mma * MH * 40.0);
+            const bool shallow = 3 * (size_t)MH * a_rows * 128 + 2 * g_tiles * BN * 128 > budget;
             const double tma = ((double)MH * a_rows * 128 + (double)kw * BN * 128) / 72.0;
-            double tile_t = (double)kh * chunks * std::max(mma, tma) + 800.0;
-            const double epi = MH * (BN / 16) * 170.0;
+            double tile_t = (double)kh * chunks * (std::max(mma, tma) + (shallow ? 600.0 : 0.0)) + 800.0;
+            // epilogue per 16 columns and row half: about 170 cycles through the staged TMA store, about 1000 with direct
+            // stores (tiles whose 64-column slabs would not fit the group's channel range)
+            const bool staged = BN % 64 == 0 || (groups == 1 && N == BN);
+            const double epi = MH * (BN / 16) * (staged ? 170.0 : 1000.0);
             if (acc == 1) tile_t += epi; else tile_t = std::max(tile_t, epi + 300.0);
             const double t = rounds * tile_t;
             if (t < best_t) { best_t = t; best = ConvShape{MH, BN, acc}; }
@@ -339,7 +347,8 @@ void finish_conv_plan(const alexnet* h, Plan& P) {
     if (c.cpg < 1) c.cpg = 1;
     const size_t a_bytes = (size_t)c.MH * c.cpg * c.a_box_rows * 128, b_bytes = (size_t)c.BN * 128;
     const size_t budget = 227 * 1024 - 2048 - 4 * tc::kEpiStageBytes;
-    c.tpg = c.cpg > 1 ? c.cpg : (c.kw <= 3 ? c.kw : 3);   // weight tiles travel in groups: a filter row (3 + 2 taps of a five-tap row), or the chunks of an FC stage
+    c.tpg = c.cpg > 1 ? c.cpg : (c.kw <= 3 ? c.kw : 2);   // weight tiles travel in groups: a filter row (2 + 2 + 1 taps of a five-tap row, which keeps
+                                                          // four groups in flight), or the chunks of an FC stage
     const size_t g_bytes = b_bytes * c.tpg;
     if (c.kw == 1) {
         int st = (int)(budget / (a_bytes + g_bytes));
