@@ -301,9 +301,9 @@ void finish_plan(const alexnet* h, Plan& P) {
 // groups, a kh x kw filter over `chunks` 64-channel chunks: the (row halves, BN) pair with the lowest
 // modelled time.  Per weight stage the tensor pipe needs MH*kk*BN/2 cycles; TMA brings about 64 bytes
 // per cycle per SM from L2; tiles are dealt to the SMs in rounds.
-struct ConvShape { int MH, BN, acc_stages; };
+struct ConvShape { int MH, BN, acc_stages, epi_sets; };
 ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, int kh, int kw, int chunks, int kk) {
-    ConvShape best{1, N <= 256 ? N : 128, 1};
+    ConvShape best{1, N <= 256 ? N : 128, 1, 1};
     double best_t = 1e30;
     const int a_rows = kw > 1 ? 136 : 128;
     const size_t budget = 227 * 1024 - 2048 - 4 * tc::kEpiStageBytes;
@@ -326,13 +326,18 @@ ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, in
             const bool shallow = 3 * (size_t)MH * a_rows * 128 + 2 * g_tiles * BN * 128 > budget;
             const double tma = ((double)MH * a_rows * 128 + (double)kw * BN * 128) / 72.0;
             double tile_t = (double)kh * chunks * (std::max(mma, tma) + (shallow ? 600.0 : 0.0)) + 800.0;
-            // epilogue per 16 columns and row half: about 170 cycles through the staged TMA store, about 1000 with direct
+            // epilogue per 16 columns and row half: about 450 cycles through the staged TMA store (single staging tile per warp), about 1000 with direct
             // stores (tiles whose 64-column slabs would not fit the group's channel range)
             const bool staged = BN % 64 == 0 || (groups == 1 && N == BN);
-            const double epi = MH * (BN / 16) * (staged ? 170.0 : 1000.0);
-            if (acc == 1) tile_t += epi; else tile_t = std::max(tile_t, epi + 300.0);
-            const double t = rounds * tile_t;
-            if (t < best_t) { best_t = t; best = ConvShape{MH, BN, acc}; }
+            const double epi = MH * (BN / 16) * (staged ? 450.0 : 1000.0);
+            // a second set of epilogue warps (each takes every other row half) when the epilogue is the longer side
+            for (int E = 1; E <= (MH >= 2 && staged ? 2 : 1); ++E) {
+                if (E == 2 && 2 * (size_t)MH * a_rows * 128 + 2 * g_tiles * BN * 128 + 4 * tc::kEpiStageBytes > budget) continue;
+                double tt = tile_t;
+                if (acc == 1) tt += epi / E; else tt = std::max(tt, epi / E + 300.0);
+                const double t = rounds * tt + (E == 2 ? 1.0 : 0.0);     // ties go to the smaller block
+                if (t < best_t) { best_t = t; best = ConvShape{MH, BN, acc, E}; }
+            }
         }
     }
     return best;
@@ -346,7 +351,8 @@ void finish_conv_plan(const alexnet* h, Plan& P) {
     c.tiles_total = c.m_tiles * c.n_tiles * c.groups * c.splits;
     if (c.cpg < 1) c.cpg = 1;
     const size_t a_bytes = (size_t)c.MH * c.cpg * c.a_box_rows * 128, b_bytes = (size_t)c.BN * 128;
-    const size_t budget = 227 * 1024 - 2048 - 4 * tc::kEpiStageBytes;
+    if (c.epi_sets < 1) c.epi_sets = 1;
+    const size_t budget = 227 * 1024 - 2048 - 4 * c.epi_sets * tc::kEpiStageBytes;
     c.tpg = c.cpg > 1 ? c.cpg : (c.kw <= 3 ? c.kw : 2);   // weight tiles travel in groups: a filter row (2 + 2 + 1 taps of a five-tap row, which keeps
                                                           // four groups in flight), or the chunks of an FC stage
     const size_t g_bytes = b_bytes * c.tpg;
@@ -385,7 +391,7 @@ int plan_conv_fwd(alexnet* h, Plan& P, const ConvL& c, const bf16* in, const bf1
     const int gp = c.gin.Wp;
     p.kh = p.kw = c.k; p.chunks = (c.cig + 63) / 64; p.kk = c.cig == 48 ? 3 : 4;
     const ConvShape sh = choose_conv_shape(h, M, c.cog, c.groups, p.kh, p.kw, p.chunks, p.kk);
-    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages;
+    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages; p.epi_sets = sh.epi_sets;
     p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH - 1) / (128 * p.MH));
     p.n_tiles = c.cog / p.BN; p.groups = c.groups; p.splits = 1;
     p.asteps_total = p.kh * p.chunks;
@@ -410,7 +416,7 @@ int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf1
     const int gp = c.gin.Wp;
     p.kh = p.kw = c.k; p.chunks = c.cog / 64; p.kk = 4;
     const ConvShape sh = choose_conv_shape(h, M, c.cig, c.groups, p.kh, p.kw, p.chunks, p.kk);
-    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages;
+    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages; p.epi_sets = sh.epi_sets;
     p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH - 1) / (128 * p.MH));
     p.n_tiles = c.cig / p.BN; p.groups = c.groups; p.splits = 1;
     p.asteps_total = p.kh * p.chunks;

@@ -578,6 +578,7 @@ struct ConvParams {
     int chunks;         // 64-channel chunks
     int asteps_total;   // kh * chunks, split evenly over `splits`
     int asteps_per_split;
+    int epi_sets;       // 1 or 2 sets of four epilogue warps; with two, set e handles the row halves h with h % 2 == e
     int a_stages, b_stages, acc_stages;   // b_stages counts groups of kw weight tiles (one barrier pair per group)
     int a_box_rows;     // rows per activation box (128, or 136 when kw > 1)
     int a_x0, a_gx;     // A column origin and per-group column stride
@@ -595,10 +596,10 @@ struct ConvParams {
     int* status;
 };
 
-constexpr int kConvMaxThreads = 32 * 10;
-inline int conv_threads(const ConvParams& p) { return 32 * (6 + p.MH); }
+constexpr int kConvMaxThreads = 32 * 12;
+inline int conv_threads(const ConvParams& p) { return 32 * (2 + p.MH + 4 * p.epi_sets); }
 inline size_t conv_smem_bytes(const ConvParams& p) {
-    return 1024 + (size_t)p.a_stages * p.MH * p.cpg * p.a_box_rows * 128 + (size_t)p.b_stages * p.tpg * p.BN * 128 + 4 * kEpiStageBytes + 512;
+    return 1024 + (size_t)p.a_stages * p.MH * p.cpg * p.a_box_rows * 128 + (size_t)p.b_stages * p.tpg * p.BN * 128 + 4 * p.epi_sets * kEpiStageBytes + 512;
 }
 
 // tile cursor shared by the roles (m fastest, then n tile, group, split)
@@ -644,11 +645,11 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * 128u, a_bytes = a_box_bytes * MH * cpg, b_bytes = (uint32_t)BN * 128u;
     const int a_stages = p.a_stages, b_stages = p.b_stages;
     const uint32_t ring_a = base, ring_b = base + a_stages * a_bytes;
-    // epilogue staging (4 warps x kEpiStageBytes), then barriers: fullA[8] @0, emptyA[8] @64, fullB[8] @128,
+    // epilogue staging (4 * epi_sets warps x kEpiStageBytes), then barriers: fullA[8] @0, emptyA[8] @64, fullB[8] @128,
     // emptyB[8] @192, acc_full[2] @256, acc_empty[2] @272, tmem slot @288, abort flag @296
     const uint32_t g_bytes = b_bytes * (uint32_t)p.tpg;         // one group slot holds up to tpg weight tiles of a filter row
     const uint32_t epi_stage0 = ring_b + b_stages * g_bytes;
-    const uint32_t bar_base = epi_stage0 + 4u * kEpiStageBytes;
+    const uint32_t bar_base = epi_stage0 + 4u * (uint32_t)p.epi_sets * kEpiStageBytes;
     uint8_t* gen = smem_raw + (bar_base - raw);
     volatile int* abort_flag = (volatile int*)(gen + 296);
     volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 288);
@@ -663,7 +664,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         *abort_flag = 0;
         for (int s = 0; s < a_stages; ++s) { mbar_init(fullA + 8u * s, 1); mbar_init(emptyA + 8u * s, MH); }
         for (int s = 0; s < b_stages; ++s) { mbar_init(fullB + 8u * s, 1); mbar_init(emptyB + 8u * s, MH); }
-        for (int s = 0; s < 2; ++s) { mbar_init(accf0 + 8u * s, MH); mbar_init(acce0 + 8u * s, 128); }
+        for (int s = 0; s < 2; ++s) { mbar_init(accf0 + 8u * s, MH); mbar_init(acce0 + 8u * s, 128 * p.epi_sets); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&p.tmA);
         tma_prefetch_desc(&p.tmB);
@@ -797,6 +798,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     } else {
         // ------------------------------------------------------------ epilogue
         const int quad = warp & 3;
+        const int ew = warp - (MH + 2), eset = ew >> 2, E = p.epi_sets;     // epilogue warp index and its set
         const int r = quad * 32 + lane;          // row within a 128-row half = TMEM lane
         ConvCursor tc; tc.init(p);
         int ab = 0; uint32_t aph = 0;
@@ -808,7 +810,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
             if (!(ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag))) break;
             tc_fence_after();
             #pragma unroll 1
-            for (int h = 0; h < MH; ++h) {
+            for (int h = eset; h < MH; h += E) {
                 const int row = m0 + h * 128 + r;
                 const bool row_ok = row < p.M_total;
                 bool pad_row = false;
@@ -822,7 +824,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                     const int slab = p.epi == EPI_F32 ? 32 : 64;
                     for (int c = 0; c < BN; c += slab) {
                         epi_slab(p, t0 + (uint32_t)c, pad_row, row_off, n0 + c, g, g * p.out_gx + n0 + c, m0 + h * 128 + quad * 32,
-                                 tc.z, epi_stage0 + (uint32_t)quad * kEpiStageBytes, lane);
+                                 tc.z, epi_stage0 + (uint32_t)ew * kEpiStageBytes, lane);
                     }
                 } else {
                     for (int c = 0; c < BN; c += 16) {
