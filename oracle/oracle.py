@@ -440,6 +440,51 @@ class OracleNet:
         return T
 
 
+EVAL_CROP = 14      # (256 - 227) // 2: the centre 227 x 227 window starts at row/column 14
+
+
+def topk_correct(z, labels, k):
+    """Per sample 1 if the label is among the k largest logits, else 0.  Rank of the label = number of logits
+    strictly greater than it plus the number of equal logits with a smaller class index (so ties are broken
+    towards the smaller index and every sample has exactly k classes in its top k)."""
+    z = _f64(z)
+    labels = np.asarray(labels, np.int64)
+    zl = z[np.arange(z.shape[0]), labels][:, None]
+    idx = np.arange(z.shape[1])[None, :]
+    rank = (z > zl).sum(axis=1) + ((z == zl) & (idx < labels[:, None])).sum(axis=1)
+    return (rank < k).astype(np.int32)
+
+
+def evaluate(net: OracleNet, img_u8, labels, mean):
+    """Evaluation forward pass (the accuracy measurements of the paper's Experiments section are top-1 / top-5
+    errors): centre crop, no flip, no dropout mask; with the non-inverted dropout of training the outputs of
+    fc6 and fc7 are multiplied by (1 - p) instead (Krizhevsky et al. 2012, Sec. 4.2).  Returns logits, mean
+    loss, and the per-sample top-1 / top-5 indicator vectors."""
+    c = net.cfg
+    P = unpack(net.w)
+    B = img_u8.shape[0]
+    cf = np.tile(np.array([EVAL_CROP, EVAL_CROP, 0], np.int32), (B, 1))
+    x = preprocess(img_u8, mean, cf)
+    la = net._lrn_args()
+
+    def conv_block(name, x):
+        cc = CONV[name]
+        return np.maximum(conv_fwd(x, P[name + ".W"], P[name + ".b"], cc["s"], cc["p"], cc["g"]), 0.0)
+
+    a = conv_block("conv1", x)
+    a, _ = pool_fwd(lrn_fwd(a, **la))
+    a = conv_block("conv2", a)
+    a, _ = pool_fwd(lrn_fwd(a, **la))
+    a = conv_block("conv5", conv_block("conv4", conv_block("conv3", a)))
+    a, _ = pool_fwd(a)
+    scale = 1.0 if (c.inverted_dropout or c.dropout_p == 0) else 1.0 - c.dropout_p
+    f6 = np.maximum(fc_fwd(a.reshape(B, 9216), P["fc6.W"], P["fc6.b"]), 0.0) * scale
+    f7 = np.maximum(fc_fwd(f6, P["fc7.W"], P["fc7.b"]), 0.0) * scale
+    z = fc_fwd(f7, P["fc8.W"], P["fc8.b"])
+    _, loss, _ = softmax_xent(z, labels)
+    return dict(x0=x, f6=f6, f7=f7, z=z, loss=loss, top1=topk_correct(z, labels, 1), top5=topk_correct(z, labels, 5))
+
+
 def average_replicas(a: OracleNet, b: OracleNet):
     """Exchange and average weights, biases and momentum of two replicas."""
     a.w, b.w = replica_average(a.w, b.w)

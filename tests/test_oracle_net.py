@@ -93,3 +93,39 @@ def test_conv1_block_against_autograd():
     assert np.allclose(T["p1"], y.detach().numpy(), rtol=1e-12, atol=1e-12)
     assert np.linalg.norm(T["dW1"] - wt.grad.numpy()) < 1e-10 * np.linalg.norm(T["dW1"])
     assert np.linalg.norm(T["db1"] - bt.grad.numpy()) < 1e-10 * np.linalg.norm(T["db1"])
+
+
+def test_topk_correct_against_sorting_and_ties():
+    rng = np.random.default_rng(5)
+    z = rng.standard_normal((64, 1000))
+    lab = rng.integers(0, 1000, 64)
+    order = np.argsort(-z, axis=1, kind="stable")
+    for k in (1, 5):
+        want = np.array([int(lab[i] in order[i, :k]) for i in range(64)])
+        assert np.array_equal(O.topk_correct(z, lab, k), want)
+    # all-equal logits: exactly the classes 0..k-1 are "in the top k"
+    z0 = np.zeros((6, 10))
+    assert O.topk_correct(z0, np.array([0, 1, 4, 5, 9, 2]), 5).tolist() == [1, 1, 1, 0, 0, 1]
+    assert O.topk_correct(z0, np.array([0, 1, 4, 5, 9, 2]), 1).tolist() == [1, 0, 0, 0, 0, 0]
+
+
+def test_evaluation_pass_centre_crop_scaling_and_training_limit():
+    """Evaluation = the training forward pass with the centre crop, no flip and the dropout masks replaced by their
+    expectation: with p = 0 (no dropout) and the same crop the two passes must agree exactly."""
+    seed, B = synth.BASE_SEED + 21, 2
+    w = synth.init_params(seed, variance_preserving=True).astype(np.float64)
+    img, lab, mean = synth.images(seed, 0, 0, B), synth.labels(seed, 0, 0, B), synth.mean_image(seed)
+    net0 = O.OracleNet(O.OracleConfig(seed=seed, dropout_p=0.0), w)
+    E0 = O.evaluate(net0, img, lab, mean)
+    cf = np.tile(np.array([14, 14, 0], np.int32), (B, 1))
+    T = net0.forward_backward(img, lab, mean, 0, cf=cf)
+    assert np.allclose(E0["z"], T["z"], rtol=0, atol=1e-12) and abs(E0["loss"] - T["loss"]) < 1e-12
+    # the crop is the centre window of the mean-subtracted image
+    assert np.array_equal(E0["x0"][0, 1], img[0, 14:241, 14:241, 1].astype(np.float64) - mean[14:241, 14:241, 1])
+    # p = 0.5 without rescaling at training time: evaluation halves the fc6 / fc7 outputs; inverted dropout does not
+    Eh = O.evaluate(O.OracleNet(O.OracleConfig(seed=seed, dropout_p=0.5), w), img, lab, mean)
+    Ei = O.evaluate(O.OracleNet(O.OracleConfig(seed=seed, dropout_p=0.5, inverted_dropout=True), w), img, lab, mean)
+    assert np.allclose(Eh["f6"], 0.5 * E0["f6"]) and np.allclose(Ei["f6"], E0["f6"]) and np.allclose(Ei["z"], E0["z"])
+    assert not np.allclose(Eh["z"], E0["z"])
+    # mean over dropout masks of the training-time fc6 output (given identical inputs) approaches the halved output
+    assert Eh["top1"].shape == (B,) and set(np.unique(Eh["top5"])) <= {0, 1}
