@@ -105,6 +105,21 @@ int alexnet_load_batch_async(alexnet_t* h, int replica, const uint8_t* images, c
  * Errors: STATE (no loaded batch), DEVICE_TIMEOUT (latched), CUDA. */
 int alexnet_train_step(alexnet_t* h, int replica, float* host_loss);
 
+/* Evaluation of one minibatch, the measurement behind the paper's reported
+ * validation errors ("Experiments": top-1 and top-5 error): forward pass only,
+ * on the centre 227 x 227 crop without flip, with the dropout masks replaced by
+ * their expectation (outputs of fc6 / fc7 times 1 - p, unless training uses
+ * inverted dropout).  Copies images [B][256][256][3] uint8 and labels [B] int32
+ * (pinned host or device memory) like load_batch_async, runs on both streams
+ * and waits for the result.  A sample counts for top-k when fewer than k classes
+ * rank before its label (greater logit, or equal logit and smaller index).
+ *   host_top1, host_top5  number of samples of the batch in the top 1 / top 5 (may be NULL)
+ *   host_loss             mean cross-entropy of the batch (may be NULL)
+ * Parameters are not changed.  Errors: ARG, STATE (a loaded training batch is
+ * still waiting for its train_step), DEVICE_TIMEOUT, CUDA. */
+int alexnet_eval_batch(alexnet_t* h, int replica, const uint8_t* images, const int32_t* labels, int32_t* host_top1,
+                       int32_t* host_top5, float* host_loss);
+
 /* Steps 2 and 3 of the paper's data-parallel figure for two replicas held in
  * one GPU memory: w_a = w_b = (w_a+w_b)/2 and the same for momentum, over all
  * weights and biases.  No-op returning OK when replicas == 1. */

@@ -31,7 +31,7 @@ OP = {n: i for i, n in enumerate(OPS)}
 
 EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "alexnet_destroy",
            "alexnet_load_batch_async", "alexnet_train_step", "alexnet_replica_average", "alexnet_get_params",
-           "alexnet_set_params", "alexnet_tensor_size", "alexnet_get_tensor", "alexnet_set_tensor", "alexnet_run_op",
+           "alexnet_set_params", "alexnet_eval_batch", "alexnet_tensor_size", "alexnet_get_tensor", "alexnet_set_tensor", "alexnet_run_op",
            "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error", "alexnet_bias_grad_noalloc"]
 
 
@@ -70,6 +70,8 @@ def load_library():
     L.alexnet_load_batch_async.argtypes = [vp, i32, vp, vp, u64]
     L.alexnet_train_step.argtypes = [vp, i32, vp]
     L.alexnet_replica_average.argtypes = [vp]
+    L.alexnet_eval_batch.argtypes = [vp, i32, vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
+                                     ctypes.POINTER(ctypes.c_float)]
     L.alexnet_get_params.argtypes = [vp, i32, i32, vp, sz]
     L.alexnet_set_params.argtypes = [vp, i32, i32, vp, sz]
     L.alexnet_tensor_size.restype = sz
@@ -159,6 +161,14 @@ class AlexNet:
             return loss.value
         self._ck(self.lib.alexnet_train_step(self.h, replica, None))
         return None
+
+    def eval_batch(self, replica, images, labels):
+        """(top-1 count, top-5 count, mean loss) of one minibatch: forward pass on the centre crop, no dropout mask."""
+        t1, t5, loss = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_float()
+        self._keep = self._keep[-8:] + [(images, labels)]
+        self._ck(self.lib.alexnet_eval_batch(self.h, replica, _ptr(images), _ptr(labels), ctypes.byref(t1), ctypes.byref(t5),
+                                             ctypes.byref(loss)))
+        return t1.value, t5.value, loss.value
 
     def replica_average(self):
         self._ck(self.lib.alexnet_replica_average(self.h))

@@ -608,7 +608,7 @@ void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
                                                               h->cs_partial, c.cout, R.g + c.b_off);
     h->launches++;
 }
-void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st) {
+void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool eval = false) {
     Replica& R = h->rep[r];
     const FcL& f = h->L.fc[l];
     const Plan& P = R.fc_fwd[l];
@@ -616,10 +616,15 @@ void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st) {
     const long long total = (long long)h->B * f.N;
     bf16* outs[3] = {R.f6, R.f7, nullptr};
     uint8_t* keeps[3] = {R.m6, R.m7, nullptr};
-    const int drop = l < 2 && h->cfg.dropout_p > 0.f;
+    int drop = l < 2 && h->cfg.dropout_p > 0.f;
+    float scale = h->drop_scale;
+    if (eval && drop) {    // no mask at evaluation: its expectation, unless training already rescales (inverted dropout)
+        drop = 2;
+        scale = (h->cfg.flags & ALEXNET_FLAG_INVERTED_DROPOUT) ? 1.f : 1.f - h->cfg.dropout_p;
+    }
     const uint64_t key = kn::stream_key(h->cfg.seed, 2 + l, r, step);
     kn::fc_reduce_fwd_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.c.splits, P.c.split_stride, R.w + f.b_off, h->B, f.N,
-                                                                l < 2, drop, key, h->thr24, h->drop_scale, outs[l],
+                                                                l < 2, drop, key, h->thr24, scale, outs[l],
                                                                 l == 2 ? R.z : nullptr, keeps[l]);
     h->launches++;
 }
@@ -733,23 +738,27 @@ void op_average(alexnet* h, cudaStream_t st) {
     refresh_shadows(h, 0, false, st);
     refresh_shadows(h, 1, false, st);
 }
-void op_preprocess(alexnet* h, int r, int slot, uint64_t step, cudaStream_t st) {
+void op_preprocess(alexnet* h, int r, int slot, uint64_t step, cudaStream_t st, bool eval = false) {
     Replica& R = h->rep[r];
     const long long total = (long long)h->B * 57 * 57 * 4;
     kn::preprocess_kernel<<<nblk(total, 256), 256, 0, st>>>(R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
-                                                            kn::stream_key(h->cfg.seed, 1, r, step));
+                                                            kn::stream_key(h->cfg.seed, 1, r, step), eval ? 1 : 0);
     h->launches++;
 }
 
-void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
+void forward(alexnet* h, int r, int slot, cudaStream_t st, bool eval) {
     Replica& R = h->rep[r];
     const uint64_t step = R.slot_step[slot];
     op_conv_fwd(h, r, 0, slot, st); op_lrn_pool_fwd(h, r, 0, st);
     op_conv_fwd(h, r, 1, slot, st); op_lrn_pool_fwd(h, r, 1, st);
     op_conv_fwd(h, r, 2, slot, st); op_conv_fwd(h, r, 3, slot, st); op_conv_fwd(h, r, 4, slot, st);
     op_pool_fwd(h, r, 2, st);
-    op_fc_fwd(h, r, 0, step, st); op_fc_fwd(h, r, 1, step, st); op_fc_fwd(h, r, 2, step, st);
+    op_fc_fwd(h, r, 0, step, st, eval); op_fc_fwd(h, r, 1, step, st, eval); op_fc_fwd(h, r, 2, step, st, eval);
     op_softmax(h, r, slot, st);
+}
+void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    forward(h, r, slot, st, false);
     op_fc_wg(h, r, 2, true, st); op_fc_bwd(h, r, 2, st);
     op_fc_wg(h, r, 1, false, st); op_fc_bwd(h, r, 1, st);
     op_fc_wg(h, r, 0, false, st); op_fc_bwd(h, r, 0, st);
@@ -983,6 +992,40 @@ int alexnet_train_step(alexnet_t* h, int replica, float* host_loss) {
         return poll_status(h);
     }
     return ALEXNET_OK;
+}
+
+int alexnet_eval_batch(alexnet_t* h, int replica, const uint8_t* images, const int32_t* labels, int32_t* host_top1,
+                       int32_t* host_top5, float* host_loss) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas || !images || !labels) return fail(h, ALEXNET_ERR_ARG, "eval_batch: bad argument");
+    if (int rc = check_status(h)) return rc;
+    Replica& R = h->rep[replica];
+    if (R.loaded != 0) return fail(h, ALEXNET_ERR_STATE, "eval_batch: a loaded training batch is waiting for its train_step");
+    const int s = R.next_load;      // the free slot the next training load would use; it stays free afterwards
+    if (R.consumed_valid[s]) CK(cudaStreamWaitEvent(h->ls, R.consumed[s], 0));
+    CK(cudaMemcpyAsync(R.stage[s], images, (size_t)h->B * 196608, cudaMemcpyDefault, h->ls));
+    CK(cudaMemcpyAsync(R.labels[s], labels, (size_t)h->B * sizeof(int32_t), cudaMemcpyDefault, h->ls));
+    op_preprocess(h, replica, s, 0, h->ls, true);
+    CK(cudaEventRecord(R.ready[s], h->ls));
+    R.slot_step[s] = 0; R.last_slot = s;
+    CK(cudaStreamWaitEvent(h->cs, R.ready[s], 0));
+    forward(h, replica, s, h->cs, true);
+    int32_t* counts = (int32_t*)(h->status + 4);    // two counters in the status block
+    CK(cudaMemsetAsync(counts, 0, 2 * sizeof(int32_t), h->cs));
+    kn::topk_count_kernel<<<h->B, 256, 0, h->cs>>>(R.z, R.labels[s], 1000, counts);
+    h->launches++;
+    CK(cudaEventRecord(R.consumed[s], h->cs));
+    R.consumed_valid[s] = true;
+    int32_t hc[2] = {0, 0};
+    float loss = 0.f;
+    CK(cudaMemcpyAsync(hc, counts, sizeof(hc), cudaMemcpyDeviceToHost, h->cs));
+    CK(cudaMemcpyAsync(&loss, R.loss, sizeof(float), cudaMemcpyDeviceToHost, h->cs));
+    CK(cudaStreamSynchronize(h->cs));
+    CK(cudaGetLastError());
+    if (host_top1) *host_top1 = hc[0];
+    if (host_top5) *host_top5 = hc[1];
+    if (host_loss) *host_loss = loss;
+    return poll_status(h);
 }
 
 int alexnet_replica_average(alexnet_t* h) {

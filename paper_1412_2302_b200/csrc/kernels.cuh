@@ -46,7 +46,7 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 // with row/column 227 of the 228-padded image set to zero.
 __global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* __restrict__ mean,
                                   __nv_bfloat16* __restrict__ out, int32_t* __restrict__ cf_out,
-                                  int B, uint64_t key) {
+                                  int B, uint64_t key, int eval_mode) {
     // one thread per (n, by, bx, dy): 12 output values (4 dx * 3 colours) = 24 bytes
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long total = (long long)B * 57 * 57 * 4;
@@ -57,7 +57,9 @@ __global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* 
     const int by = (int)(cell % 57);
     const int n = (int)(cell / 57);
     const uint64_t r = draw(key, (uint64_t)n);
-    const int ox = (int)((r & 0xFFFF) % 30), oy = (int)(((r >> 16) & 0xFFFF) % 30), flip = (int)((r >> 32) & 1);
+    // evaluation: the centre 227 x 227 window, never flipped
+    const int ox = eval_mode ? 14 : (int)((r & 0xFFFF) % 30), oy = eval_mode ? 14 : (int)(((r >> 16) & 0xFFFF) % 30);
+    const int flip = eval_mode ? 0 : (int)((r >> 32) & 1);
     if (cf_out && by == 0 && bx == 0 && dy == 0) { cf_out[3 * n] = ox; cf_out[3 * n + 1] = oy; cf_out[3 * n + 2] = flip; }
     const int Y = by * 4 + dy;
     float v[12];
@@ -351,7 +353,10 @@ __global__ void fc_reduce_fwd_kernel(const float* __restrict__ ws, int splits, l
     for (int z = 0; z < splits; ++z) v += ws[z * split_stride + t];
     v += bias[n];
     if (relu) v = fmaxf(v, 0.f);
-    if (use_dropout) {
+    if (use_dropout == 2) {            // evaluation: the expectation of the mask instead of a mask
+        v *= scale;
+        if (keep_out) keep_out[t] = 1;
+    } else if (use_dropout) {
         const bool keep = (uint32_t)(draw(key, (uint64_t)t) >> 40) >= thr24;
         if (keep_out) keep_out[t] = keep ? 1 : 0;
         v = keep ? v * scale : 0.f;
@@ -497,6 +502,30 @@ __global__ void mean_kernel(const float* __restrict__ v, int n, float* __restric
         float t = 0.f;
         for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += red[w];
         *out = t / (float)n;
+    }
+}
+
+// top-1 / top-5 counting: one block per sample.  rank of the label = logits strictly greater than it plus equal
+// logits with a smaller class index; the sample counts for top-k when rank < k.  counts[0] += top-1, counts[1] += top-5
+// (integer atomics: the result does not depend on the order).
+__global__ void topk_count_kernel(const float* __restrict__ z, const int32_t* __restrict__ labels, int N, int32_t* __restrict__ counts) {
+    __shared__ int red[32];
+    const int n = blockIdx.x, lab = labels[n];
+    const float* zr = z + (size_t)n * N;
+    const float zl = zr[lab];
+    int c = 0;
+    for (int j = threadIdx.x; j < N; j += blockDim.x) {
+        const float v = zr[j];
+        c += (v > zl) || (v == zl && j < lab);
+    }
+    for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(~0u, c, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int rank = 0;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) rank += red[w];
+        if (rank < 1) atomicAdd(counts, 1);
+        if (rank < 5) atomicAdd(counts + 1, 1);
     }
 }
 

@@ -104,6 +104,18 @@ def main(argv=None):
             else:
                 gbs = hb[name] / (ms * 1e-3) / 1e9
                 rows.append({"op": name, "ms": ms, "gbs": gbs, "frac": gbs / hbm_peak, "bound": "hbm"})
+    # the evaluation pass (forward only, centre crop, top-1 / top-5 counts), batch resident on the device; the call
+    # waits for its result, so this is wall-clock time per call
+    import time
+    dimg, dlab = img.to(net.device), lab.to(net.device)
+    eval_ms = None
+    if not args.ops:
+        for _ in range(3):
+            net.eval_batch(0, dimg, dlab)
+        t0 = time.perf_counter()
+        for _ in range(args.iters):
+            net.eval_batch(0, dimg, dlab)
+        eval_ms = (time.perf_counter() - t0) * 1e3 / args.iters
     net.close()
     print(f"# batch {B}, median of {args.iters} runs, L2 flushed before each; peaks ({kind}): "
           f"{tf_peak:.0f} TFLOP/s bf16 burst, {hbm_peak:.0f} GB/s HBM")
@@ -112,6 +124,8 @@ def main(argv=None):
         print(f"{r['op']:<20}{r['ms']:>9.4f}{r.get('tflops', float('nan')):>10.1f}{r.get('gbs', float('nan')):>9.0f}{r['frac']:>9.3f}")
     tot = sum(r["ms"] for r in rows)
     print(f"# sum of all operations: {tot:.3f} ms")
+    if eval_ms is not None:
+        print(f"# alexnet_eval_batch (forward + top-k, synchronous call): {eval_ms:.3f} ms per batch, {B / eval_ms * 1e3:.0f} images/s")
     if args.json:
         json.dump({"batch": B, "iters": args.iters, "peaks": {"bf16_tflops": tf_peak, "hbm_gbs": hbm_peak, "kind": kind},
                    "rows": rows}, open(args.json, "w"), indent=1)
