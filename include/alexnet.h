@@ -211,6 +211,33 @@ int alexnet_profile_read(alexnet_t* h, double* ms3, uint64_t* launches3);
 int alexnet_bias_grad_noalloc(const void* dev_dy, int64_t rows, int32_t channels, float* dev_db, void* stream,
                               char* err, size_t err_len);
 
+/* Host half of the paper's loading process ("Parallel Data Loading": a second
+ * process loads the next minibatch while the current one trains): a worker
+ * pool of `threads` threads (each fills whole batches, in turn) gathers
+ * minibatches from a dataset in host memory (for instance a
+ * memory-mapped file of uint8 [n][256][256][3] images and int32 labels) into a
+ * ring of `depth` staging slots.  Sample j of the stream is dataset entry
+ * perm_e[j mod n_epoch] with e = j / n_epoch and n_epoch = floor(n / batch) *
+ * batch (an epoch drops the incomplete last batch); perm_e is the identity, or
+ * with `shuffle` a Fisher-Yates shuffle (i from n_epoch-1 down to 1, swap with
+ * hash(key_e, i) mod (i+1), key_e = mix(seed ^ 9<<56 ^ e), same counter hash as
+ * crop / flip).  No CUDA calls are made: `ring` is caller memory of
+ * alexnet_loader_ring_bytes(batch, depth) bytes, pinned if
+ * alexnet_load_batch_async is to copy from it asynchronously.
+ *   next     waits up to timeout_ms for the next batch in order and returns pointers to its images [batch][256][256][3]
+ *            and labels [batch] inside the ring (STATE on time-out or when all `depth` slots are held)
+ *   release  returns the oldest held slot to the worker; call it once the copy out of that slot has finished
+ *            (for example after the train_step consuming it returned its loss, or after alexnet_sync)
+ * Errors: ARG, NOMEM (ring too small), STATE. */
+typedef struct alexnet_loader alexnet_loader_t;
+size_t alexnet_loader_ring_bytes(int32_t batch, int32_t depth);
+int alexnet_loader_create(const uint8_t* host_images, const int32_t* host_labels, uint64_t n_images, int32_t batch,
+                          uint8_t* ring, size_t ring_bytes, int32_t depth, int32_t threads, uint64_t seed, int32_t shuffle,
+                          alexnet_loader_t** out);
+int alexnet_loader_next(alexnet_loader_t* l, int32_t timeout_ms, const uint8_t** images, const int32_t** labels, uint64_t* batch_index);
+int alexnet_loader_release(alexnet_loader_t* l);
+int alexnet_loader_destroy(alexnet_loader_t* l);
+
 /* Wait for both streams; returns a latched DEVICE_TIMEOUT or CUDA error if any. */
 int alexnet_sync(alexnet_t* h);
 const char* alexnet_last_error(const alexnet_t* h);

@@ -440,6 +440,31 @@ class OracleNet:
         return T
 
 
+def loader_order(n_images, batch, seed, shuffle, n_batches):
+    """Dataset indices of the first n_batches minibatches of the loading process: sample j of the stream is entry
+    perm_e[j mod n_epoch] of the dataset, e = j // n_epoch, n_epoch = (n_images // batch) * batch; perm_e is the
+    identity or, with shuffle, the Fisher-Yates shuffle driven by the counter hash (stream 9, keyed by the epoch):
+    for i = n_epoch-1 .. 1: swap entries i and draw(key_e, i) mod (i+1)."""
+    n_epoch = (n_images // batch) * batch
+    out, perms = [], {}
+    for b in range(n_batches):
+        idx = []
+        for i in range(batch):
+            j = b * batch + i
+            e, pos = divmod(j, n_epoch)
+            if e not in perms:
+                perm = list(range(n_epoch))
+                if shuffle:
+                    key = mix64((seed ^ (9 << 56) ^ e) & (2**64 - 1))
+                    for t in range(n_epoch - 1, 0, -1):
+                        r = draw(key, t) % (t + 1)
+                        perm[t], perm[r] = perm[r], perm[t]
+                perms[e] = perm
+            idx.append(perms[e][pos])
+        out.append(np.array(idx, np.int64))
+    return out
+
+
 EVAL_CROP = 14      # (256 - 227) // 2: the centre 227 x 227 window starts at row/column 14
 
 

@@ -32,7 +32,8 @@ OP = {n: i for i, n in enumerate(OPS)}
 EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "alexnet_destroy",
            "alexnet_load_batch_async", "alexnet_train_step", "alexnet_replica_average", "alexnet_get_params",
            "alexnet_set_params", "alexnet_eval_batch", "alexnet_tensor_size", "alexnet_get_tensor", "alexnet_set_tensor", "alexnet_run_op",
-           "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error", "alexnet_bias_grad_noalloc"]
+           "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error", "alexnet_bias_grad_noalloc", "alexnet_loader_ring_bytes",
+           "alexnet_loader_create", "alexnet_loader_next", "alexnet_loader_release", "alexnet_loader_destroy"]
 
 
 class Config(ctypes.Structure):
@@ -86,6 +87,13 @@ def load_library():
     L.alexnet_sync.argtypes = [vp]
     L.alexnet_last_error.restype = ctypes.c_char_p
     L.alexnet_last_error.argtypes = [vp]
+    L.alexnet_loader_ring_bytes.restype = sz
+    L.alexnet_loader_ring_bytes.argtypes = [ctypes.c_int32, ctypes.c_int32]
+    L.alexnet_loader_create.argtypes = [vp, vp, u64, ctypes.c_int32, vp, sz, ctypes.c_int32, ctypes.c_int32, u64, ctypes.c_int32,
+                                        ctypes.POINTER(vp)]
+    L.alexnet_loader_next.argtypes = [vp, ctypes.c_int32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(u64)]
+    L.alexnet_loader_release.argtypes = [vp]
+    L.alexnet_loader_destroy.argtypes = [vp]
     L.alexnet_bias_grad_noalloc.argtypes = [vp, ctypes.c_int64, ctypes.c_int32, vp, vp, ctypes.c_char_p, sz]
     _lib = L
     return L
@@ -214,6 +222,58 @@ class AlexNet:
     @property
     def launch_count(self):
         return int(self.lib.alexnet_launch_count(self.h))
+
+
+class Loader:
+    """Worker thread that gathers minibatches from a dataset in host memory into a ring of staging slots
+    (include/alexnet.h, alexnet_loader_*).  images: uint8 array [n,256,256,3]; labels: int32 [n] (numpy arrays or
+    memory maps; they must outlive the loader).  The ring is allocated here: pinned through torch when pin=True."""
+
+    def __init__(self, images, labels, batch, depth=3, seed=0, shuffle=True, pin=False, threads=2):
+        self.lib = load_library()
+        self.images, self.labels, self.batch = images, labels, batch
+        nbytes = int(self.lib.alexnet_loader_ring_bytes(batch, depth))
+        if nbytes == 0:
+            raise AlexNetError(ERR_ARG, "invalid loader configuration")
+        if pin:
+            import torch
+            self.ring = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+            ring_ptr = self.ring.data_ptr()
+        else:
+            self.ring = np.empty(nbytes, np.uint8)
+            ring_ptr = self.ring.ctypes.data
+        h = ctypes.c_void_p()
+        rc = self.lib.alexnet_loader_create(_ptr(images), _ptr(labels), int(images.shape[0]), batch, ctypes.c_void_p(ring_ptr),
+                                            nbytes, depth, threads, int(seed), 1 if shuffle else 0, ctypes.byref(h))
+        if rc != OK:
+            raise AlexNetError(rc, "alexnet_loader_create failed")
+        self.h = h
+
+    def next(self, timeout_ms=10000):
+        """(images, labels, batch index): numpy views into the ring slot, valid until release()."""
+        pi, pl, idx = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_uint64()
+        rc = self.lib.alexnet_loader_next(self.h, int(timeout_ms), ctypes.byref(pi), ctypes.byref(pl), ctypes.byref(idx))
+        if rc != OK:
+            raise AlexNetError(rc, "loader: no batch (time-out, or every slot is held)")
+        img = np.ctypeslib.as_array(ctypes.cast(pi, ctypes.POINTER(ctypes.c_uint8)), shape=(self.batch, 256, 256, 3))
+        lab = np.ctypeslib.as_array(ctypes.cast(pl, ctypes.POINTER(ctypes.c_int32)), shape=(self.batch,))
+        return img, lab, int(idx.value)
+
+    def release(self):
+        rc = self.lib.alexnet_loader_release(self.h)
+        if rc != OK:
+            raise AlexNetError(rc, "loader: nothing to release")
+
+    def close(self):
+        if getattr(self, "h", None):
+            self.lib.alexnet_loader_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def bias_grad_noalloc(dy, db, stream=None):

@@ -284,3 +284,40 @@ def test_full_size_batch128_two_replicas_sampled_against_oracle():
         assert np.array_equal(net.get_params(0, 0), net.get_params(1, 0))
         assert np.array_equal(net.get_params(0, 1), net.get_params(1, 1))
     net.close()
+
+
+def test_training_from_the_loader_thread_equals_direct_feeding():
+    """Batches gathered by the host loader thread (shuffled, pinned ring) give bit-identical parameters to feeding the
+    same dataset entries, in the oracle's order, by hand."""
+    from paper_1412_2302_b200 import alexnet as A
+    seed, B, n = BASE + 6, 4, 10
+    rng = np.random.default_rng(9)
+    img = rng.integers(0, 256, size=(n, 256, 256, 3), dtype=np.uint8)
+    lab = rng.integers(0, 1000, size=(n,), dtype=np.int32)
+    w = synth.init_params(seed, variance_preserving=True)
+    order = O.loader_order(n, B, 99, True, 4)
+
+    def run(use_loader):
+        net = make(B, seed=seed)
+        net.set_params(w)
+        ld = A.Loader(img, lab, batch=B, depth=3, seed=99, shuffle=True, pin=True) if use_loader else None
+        losses = []
+        for s in range(4):
+            if use_loader:
+                bi, bl, idx = ld.next()
+                assert idx == s
+                net.load_batch_async(0, bi, bl, s)
+            else:
+                net.load_batch_async(0, torch.from_numpy(img[order[s]]).pin_memory(), torch.from_numpy(lab[order[s]]).pin_memory(), s)
+            losses.append(net.train_step(0, want_loss=True))      # returns after the step: the slot's copy is done
+            if use_loader:
+                ld.release()
+        p = net.get_params(0, 0)
+        if ld:
+            ld.close()
+        net.close()
+        return losses, p
+
+    l1, p1 = run(True)
+    l2, p2 = run(False)
+    assert l1 == l2 and np.array_equal(p1, p2)
