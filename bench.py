@@ -142,7 +142,9 @@ def run_ours(args, rank, world, local_rank):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     seed = synth.BASE_SEED + 3
-    net = AlexNet(batch=BATCH, replicas=1, seed=seed, mean_image=synth.mean_image(seed), device=str(dev))
+    from paper_1412_2302_b200.alexnet import FLAG_FUSED_FC_UPDATE
+    # the FC weight-gradient kernel applies the momentum update in its epilogue (bit-identical parameters, see the tests)
+    net = AlexNet(batch=BATCH, replicas=1, seed=seed, mean_image=synth.mean_image(seed), device=str(dev), flags=FLAG_FUSED_FC_UPDATE)
     net.set_params(synth.init_params(seed))
     stream = multi.rank_stream(rank)
     host = [(torch.from_numpy(synth.images(seed, stream, i, BATCH)).pin_memory(),

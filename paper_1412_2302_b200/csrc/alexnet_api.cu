@@ -269,13 +269,15 @@ int make_tm(alexnet* h, CUtensorMap* tm, const void* ptr, uint64_t cols, uint64_
 
 // output tensor map of the staged epilogue: {columns, rows, splits}, box = {128 bytes of columns, 32 rows, 1}
 int make_tm_out(alexnet* h, CUtensorMap* tm, const void* ptr, bool f32, uint64_t cols, uint64_t rows, uint64_t nz,
-                uint64_t row_pitch_bytes, uint64_t z_pitch_bytes) {
+                uint64_t row_pitch_bytes, uint64_t z_pitch_bytes, bool narrow_plain = false) {
+    // narrow_plain: bf16 box of 32 columns (64 bytes) without swizzle, the bf16 copy written by the fused FC update
     cuuint64_t dims[3] = {cols, rows, nz};
     cuuint64_t strides[2] = {row_pitch_bytes, z_pitch_bytes};
-    cuuint32_t box[3] = {f32 ? 32u : 64u, 32u, 1u};
+    cuuint32_t box[3] = {(f32 || narrow_plain) ? 32u : 64u, 32u, 1u};
     cuuint32_t es[3] = {1, 1, 1};
     CUresult r = h->encode(tm, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, (void*)ptr, dims, strides,
-                           box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                           box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, narrow_plain ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_NONE,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return fail(h, ALEXNET_ERR_CUDA, "cuTensorMapEncodeTiled (output) failed with code " + std::to_string((int)r));
     return ALEXNET_OK;
@@ -292,7 +294,8 @@ void finish_plan(const alexnet* h, Plan& P) {
     p.splits = (p.steps_total + per - 1) / per;
     p.steps_per_split = per;
     p.tiles_total = p.m_tiles * p.n_tiles * p.groups * p.taps_grid * p.splits;
-    P.smem = tc::smem_bytes(p.mode, p.BN, stages);
+    if (p.fuse_update) p.stages = stages = 2;      // the reduction is two k-steps long; the epilogue tiles need the room
+    P.smem = tc::smem_bytes(p.mode, p.BN, stages, p.fuse_update != 0);
     P.grid = std::min(p.tiles_total, h->sm_count);   // persistent: one CTA per SM walks the tile list
     P.valid = true;
 }
@@ -505,7 +508,7 @@ int plan_fc_bwd(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* w
     finish_plan(h, P);
     return ALEXNET_OK;
 }
-int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x, float* gout) {
+int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x, float* gout, float* w, float* v, bf16* shadow) {
     memset(&P, 0, sizeof(P));
     tc::GemmParams& p = P.p;
     const int B = h->B;
@@ -519,6 +522,14 @@ int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x,
     if ((rc = make_tm(h, &p.tmB, x, f.K, B, (uint64_t)f.K * 2, 64))) return rc;
     p.tma_store = 1;
     if ((rc = make_tm_out(h, &p.tmOut, gout, true, (uint64_t)f.K, (uint64_t)f.N, 1, (uint64_t)f.K * 4, (uint64_t)f.K * 4 * f.N))) return rc;
+    if (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) {
+        p.fuse_update = 1;
+        p.BN = 128; p.n_tiles = f.K / 128;   // narrower tiles leave room for four {w, v} buffers per epilogue warp
+        p.upd_lr = h->cfg.lr; p.upd_mu = h->cfg.momentum; p.upd_d = h->cfg.lr * h->cfg.weight_decay;
+        if ((rc = make_tm_out(h, &p.tmW, w, true, (uint64_t)f.K, (uint64_t)f.N, 1, (uint64_t)f.K * 4, (uint64_t)f.K * 4 * f.N))) return rc;
+        if ((rc = make_tm_out(h, &p.tmV, v, true, (uint64_t)f.K, (uint64_t)f.N, 1, (uint64_t)f.K * 4, (uint64_t)f.K * 4 * f.N))) return rc;
+        if ((rc = make_tm_out(h, &p.tmS, shadow, false, (uint64_t)f.K, (uint64_t)f.N, 1, (uint64_t)f.K * 2, (uint64_t)f.K * 2 * f.N, true))) return rc;
+    }
     finish_plan(h, P);
     return ALEXNET_OK;
 }
@@ -547,7 +558,7 @@ int build_plans(alexnet* h, int r) {
         const FcL& f = L.fc[l];
         if ((rc = plan_fc_fwd(h, R.fc_fwd[l], f, fx[l], R.shadow + f.w_off))) return rc;
         if ((rc = plan_fc_bwd(h, R.fc_bwd[l], f, fdy[l], R.shadow + f.w_off))) return rc;
-        if ((rc = plan_fc_wg(h, R.fc_wg[l], f, fdy[l], fx[l], R.g + f.w_off))) return rc;
+        if ((rc = plan_fc_wg(h, R.fc_wg[l], f, fdy[l], fx[l], R.g + f.w_off, R.w + f.w_off, R.v + f.w_off, R.shadow + f.w_off))) return rc;
     }
     return ALEXNET_OK;
 }
@@ -723,12 +734,15 @@ void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
     kn::mean_kernel<<<1, 256, 0, st>>>(R.loss_n, h->B, R.loss);
     h->launches += 2;
 }
-void op_update(alexnet* h, int r, cudaStream_t st) {
+void op_update(alexnet* h, int r, cudaStream_t st, bool full = false) {
     Replica& R = h->rep[r];
     const long long nd = (h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES) ? h->L.n_total : h->L.n_weights;
     // all conv filters precede the FC weights in the internal order
+    // with the fused FC update the FC weights (a contiguous range of the internal order) are already up to date
+    const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0 && !full;
     kn::sgd_update_kernel<<<1184, 256, 0, st>>>(R.w, R.v, R.g, R.shadow, h->L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum,
-                                                h->cfg.weight_decay, R.wt, h->L.tjobs, h->L.fc[0].w_off / 4);
+                                                h->cfg.weight_decay, R.wt, h->L.tjobs, h->L.fc[0].w_off / 4,
+                                                fused ? h->L.fc[0].w_off / 4 : 0, fused ? h->L.n_weights / 4 : 0);
     h->launches++;
 }
 void op_average(alexnet* h, cudaStream_t st) {
@@ -759,9 +773,12 @@ void forward(alexnet* h, int r, int slot, cudaStream_t st, bool eval) {
 void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
     Replica& R = h->rep[r];
     forward(h, r, slot, st, false);
-    op_fc_wg(h, r, 2, true, st); op_fc_bwd(h, r, 2, st);
-    op_fc_wg(h, r, 1, false, st); op_fc_bwd(h, r, 1, st);
-    op_fc_wg(h, r, 0, false, st); op_fc_bwd(h, r, 0, st);
+    // the data gradient reads the layer's weights, so it comes first when the weight-gradient kernel updates them in place
+    const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0;
+    for (int l = 2; l >= 0; --l) {
+        if (fused) { op_fc_bwd(h, r, l, st); op_fc_wg(h, r, l, l == 2, st); }
+        else { op_fc_wg(h, r, l, l == 2, st); op_fc_bwd(h, r, l, st); }
+    }
     op_pool_bwd(h, r, 2, st);
     op_conv_wg(h, r, 4, slot, st); op_conv_bwd(h, r, 4, st);
     op_conv_wg(h, r, 3, slot, st); op_conv_bwd(h, r, 3, st);
@@ -1173,7 +1190,7 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
         else if (op <= ALEXNET_OP_POOL5_FWD) op_pool_fwd(h, replica, op - ALEXNET_OP_POOL1_FWD, st);
         else if (op <= ALEXNET_OP_POOL5_BWD) op_pool_bwd(h, replica, op - ALEXNET_OP_POOL1_BWD, st);
         else if (op == ALEXNET_OP_SOFTMAX) op_softmax(h, replica, slot, st);
-        else if (op == ALEXNET_OP_UPDATE) op_update(h, replica, st);
+        else if (op == ALEXNET_OP_UPDATE) op_update(h, replica, st, true);
         else if (op == ALEXNET_OP_AVERAGE) op_average(h, st);
         else if (op == ALEXNET_OP_PREPROCESS) op_preprocess(h, replica, slot, R.slot_step[slot], st);
     }

@@ -38,6 +38,12 @@ constexpr long long kWaitBudgetCycles = 400000000LL;  // ~0.2 s at 2 GHz
 struct GemmParams {
     CUtensorMap tmA, tmB, tmOut;   // tmOut: output as {columns, rows, splits}, box {128 bytes, 32, 1}, when tma_store
     int tma_store;
+    // MODE_MNMN with fuse_update: the tile is an FC weight gradient and the epilogue applies the momentum update to the
+    // weights in place instead of storing the gradient: tmW / tmV = fp32 weights and momentum ({32, 32, 1} boxes, 128-byte
+    // swizzle), tmS = bf16 copy of the weights ({32, 32, 1} boxes, no swizzle); upd_d = lr * weight decay
+    CUtensorMap tmW, tmV, tmS;
+    int fuse_update;
+    float upd_lr, upd_mu, upd_d;
     int mode, epi;
     int m_tiles, n_tiles, groups, taps_grid, splits;  // tile decomposition (m fastest)
     int tiles_total;
@@ -121,6 +127,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
@@ -169,6 +180,7 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
@@ -330,8 +342,11 @@ constexpr int kABytes = 128 * 128;  // 128 rows x 64 bf16, or 2 boxes of 64 x 64
 __host__ __device__ inline int b_stage_bytes(int mode, int BN) {
     return mode == MODE_KK ? BN * 128 : ((BN + 63) / 64) * 8192;
 }
-inline size_t smem_bytes(int mode, int BN, int stages) {
-    return 1024 + (size_t)stages * (kABytes + b_stage_bytes(mode, BN)) + 4 * kEpiStageBytes + 256;
+// per epilogue warp of a fused-update kernel: kUpdBufs {w tile, v tile} pairs of 4 KB each and two 2 KB bf16 tiles
+constexpr int kUpdBufs = 4;
+constexpr uint32_t kUpdWarpBytes = kUpdBufs * 8192 + 2 * 2048;
+inline size_t smem_bytes(int mode, int BN, int stages, bool fuse_update = false) {
+    return 1024 + (size_t)stages * (kABytes + b_stage_bytes(mode, BN)) + 4 * kEpiStageBytes + (fuse_update ? 4 * kUpdWarpBytes : 0) + 512;
 }
 
 // position of a CTA in the tile list; tiles are numbered with m fastest, then
@@ -370,7 +385,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     // epilogue staging (4 warps x kEpiStageBytes), then barriers: full[8] @0, empty[8] @64, acc_full[2] @128,
     // acc_empty[2] @144, tmem slot @160, abort flag @168
     const uint32_t epi_stage0 = base + stages * stage_bytes;
-    const uint32_t bar_base = epi_stage0 + 4u * kEpiStageBytes;
+    const uint32_t upd0 = epi_stage0 + 4u * kEpiStageBytes;                     // fused update: per-warp tiles
+    const uint32_t bar_base = upd0 + (p.fuse_update ? 4u * kUpdWarpBytes : 0u);  // ... + per-warp load barriers [4][3] @176
     uint8_t* gen = smem_raw + (bar_base - raw);
     volatile int* abort_flag = (volatile int*)(gen + 168);
     volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 160);
@@ -385,6 +401,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         *abort_flag = 0;
         for (int s = 0; s < stages; ++s) { mbar_init(full0 + 8u * s, 1); mbar_init(empty0 + 8u * s, 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(accf0 + 8u * s, 1); mbar_init(acce0 + 8u * s, 128); }
+        for (int s = 0; s < 4 * kUpdBufs; ++s) mbar_init(bar_base + 176u + 8u * s, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&p.tmA);
         tma_prefetch_desc(&p.tmB);
@@ -487,6 +504,80 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         TileCursor tc; tc.init(p);
         int ab = 0; uint32_t aph = 0;
         bool ok = true;
+        if (p.fuse_update) {
+            // FC weight gradient consumed in place: for every 32 x 32 slab of the tile this warp loads the weights and the
+            // momentum by TMA (two slabs ahead of the arithmetic), applies v <- mu v - d w - lr g, w <- w + v to the
+            // accumulator values and stores w, v and the bf16 copy of w by TMA.  A buffer (of kUpdBufs = 4) is reloaded
+            // only after the stores issued from it two slabs earlier have finished reading (wait_group.read 1).
+            const uint32_t ureg = upd0 + (uint32_t)quad * kUpdWarpBytes, ub0 = bar_base + 176u + (uint32_t)quad * (8u * kUpdBufs);
+            TileCursor tp = tc;                      // prefetch cursor
+            int tile = blockIdx.x, c = 0, q = 0;     // tile, column and count of the slab being processed
+            int ptile = blockIdx.x, pc = 0, pq = 0;  // the same for the slab whose loads are issued next
+            auto issue_loads = [&]() {
+                const uint32_t bar = ub0 + 8u * (uint32_t)(pq % kUpdBufs), dst = ureg + (uint32_t)(pq % kUpdBufs) * 8192u;
+                const int x = tp.n_tile * p.BN + pc, y = tp.m_tile * 128 + quad * 32;
+                mbar_expect_tx(bar, 8192u);
+                tma_load_3d(dst, &p.tmW, x, y, 0, bar);
+                tma_load_3d(dst + 4096u, &p.tmV, x, y, 0, bar);
+                ++pq; pc += 32;
+                if (pc == p.BN) { pc = 0; ptile += gridDim.x; tp.next(p); }
+            };
+            if (lane == 0) {
+                if (ptile < p.tiles_total) issue_loads();
+                if (ptile < p.tiles_total) issue_loads();
+            }
+            __syncwarp();
+            while (tile < p.tiles_total) {
+                if (lane == 0) { bulk_wait_read_1(); if (ptile < p.tiles_total) issue_loads(); }
+                __syncwarp();
+                if (c == 0) {
+                    if (!(ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag))) break;
+                    tc_fence_after();
+                }
+                uint32_t g[32];
+                tmem_ld32(tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * p.BN + c), g);
+                tmem_ld_wait();
+                if (!(ok = mbar_wait(ub0 + 8u * (uint32_t)(q % kUpdBufs), (uint32_t)((q / kUpdBufs) & 1), abort_flag))) break;
+                const uint32_t buf = ureg + (uint32_t)(q % kUpdBufs) * 8192u, rowp = buf + (uint32_t)lane * 128u;
+                const uint32_t sbuf = ureg + (uint32_t)kUpdBufs * 8192u + (uint32_t)(q & 1) * 2048u;
+                uint32_t sh[16];
+                #pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t ch = (uint32_t)((j ^ (lane & 7)) << 4);
+                    float4 w4, v4;
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(w4.x), "=f"(w4.y), "=f"(w4.z), "=f"(w4.w) : "r"(rowp + ch));
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v4.x), "=f"(v4.y), "=f"(v4.z), "=f"(v4.w) : "r"(rowp + 4096u + ch));
+                    kn::sgd_step(w4.x, v4.x, __uint_as_float(g[4 * j]), p.upd_d, p.upd_lr, p.upd_mu);
+                    kn::sgd_step(w4.y, v4.y, __uint_as_float(g[4 * j + 1]), p.upd_d, p.upd_lr, p.upd_mu);
+                    kn::sgd_step(w4.z, v4.z, __uint_as_float(g[4 * j + 2]), p.upd_d, p.upd_lr, p.upd_mu);
+                    kn::sgd_step(w4.w, v4.w, __uint_as_float(g[4 * j + 3]), p.upd_d, p.upd_lr, p.upd_mu);
+                    st_shared_v4(rowp + ch, __float_as_uint(w4.x), __float_as_uint(w4.y), __float_as_uint(w4.z), __float_as_uint(w4.w));
+                    st_shared_v4(rowp + 4096u + ch, __float_as_uint(v4.x), __float_as_uint(v4.y), __float_as_uint(v4.z), __float_as_uint(v4.w));
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(w4.x, w4.y), hi = __floats2bfloat162_rn(w4.z, w4.w);
+                    sh[2 * j] = *(uint32_t*)&lo; sh[2 * j + 1] = *(uint32_t*)&hi;
+                }
+                #pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    st_shared_v4(sbuf + (uint32_t)lane * 64u + 16u * j, sh[4 * j], sh[4 * j + 1], sh[4 * j + 2], sh[4 * j + 3]);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    const int x = tc.n_tile * p.BN + c, y = tc.m_tile * 128 + quad * 32;
+                    tma_store_3d(&p.tmW, buf, x, y, 0);
+                    tma_store_3d(&p.tmV, buf + 4096u, x, y, 0);
+                    tma_store_3d(&p.tmS, sbuf, x, y, 0);
+                    bulk_commit();
+                }
+                ++q; c += 32;
+                if (c == p.BN) {
+                    tc_fence_before();
+                    mbar_arrive(acce0 + 8u * ab);
+                    if (++ab == 2) { ab = 0; aph ^= 1u; }
+                    c = 0; tile += gridDim.x; tc.next(p);
+                }
+            }
+            if (lane == 0) bulk_wait_all();
+        } else
         for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
             const int m0 = tc.m_tile * 128, n0 = tc.n_tile * p.BN, g = tc.g;
             const int s_begin = tc.z * per;
@@ -530,7 +621,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             mbar_arrive(acce0 + 8u * ab);
             if (++ab == 2) { ab = 0; aph ^= 1u; }
         }
-        if (p.tma_store && lane == 0) bulk_wait_all();
+        if (!p.fuse_update && p.tma_store && lane == 0) bulk_wait_all();
     }
     tc_fence_before();
     __syncthreads();

@@ -321,3 +321,25 @@ def test_training_from_the_loader_thread_equals_direct_feeding():
     l1, p1 = run(True)
     l2, p2 = run(False)
     assert l1 == l2 and np.array_equal(p1, p2)
+
+
+def test_fused_fc_update_gives_the_same_parameters():
+    """ALEXNET_FLAG_FUSED_FC_UPDATE: the FC weight-gradient kernel applies the momentum update in its epilogue.  Parameters
+    and momentum after three steps must equal those of the separate update pass (same arithmetic, same order)."""
+    from paper_1412_2302_b200 import alexnet as A
+    seed, B = BASE + 8, 8
+    w = synth.init_params(seed, variance_preserving=True, bias=0.1)
+    res = []
+    for flags in (0, A.FLAG_FUSED_FC_UPDATE):
+        net = make(B, seed=seed, flags=flags)
+        net.set_params(w)
+        losses = []
+        for step in range(3):
+            load(net, 0, seed, step, B)
+            losses.append(net.train_step(0, want_loss=True))
+        res.append((losses, net.get_params(0, 0), net.get_params(0, 1)))
+        net.close()
+    (l0, w0, v0), (l1, w1, v1) = res
+    assert l0 == l1
+    assert np.array_equal(w0, w1) and np.array_equal(v0, v1)
+    assert not np.array_equal(w0, w)
