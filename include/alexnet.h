@@ -50,10 +50,13 @@ enum {                                /* alexnet_config_t.flags */
     ALEXNET_FLAG_LRN_ALPHA_DIV_N = 1, /* s = k + (alpha/n) * sum a^2 instead of alpha * sum a^2 */
     ALEXNET_FLAG_WD_ON_BIASES = 2,    /* weight decay also on biases */
     ALEXNET_FLAG_INVERTED_DROPOUT = 4, /* kept units scaled by 1/(1-p) */
-    ALEXNET_FLAG_FUSED_FC_UPDATE = 8   /* the FC weight-gradient kernel applies the momentum update to the FC weights in its
+    ALEXNET_FLAG_FUSED_FC_UPDATE = 8,  /* the FC weight-gradient kernel applies the momentum update to the FC weights in its
                                         * epilogue (same arithmetic, bit-identical parameters) and never stores those
                                         * gradients: get_params(which = 2) is then meaningless for fc6.W / fc7.W / fc8.W,
                                         * and alexnet_run_op of an FC weight-gradient operation updates the weights */
+    ALEXNET_FLAG_NO_CTA_PAIRS = 16,    /* convolution forward / backward-data never run as clusters of two CTAs */
+    ALEXNET_FLAG_ALL_CTA_PAIRS = 32    /* ... always do (default: per layer, where the cost model expects a gain);
+                                        * results do not depend on either flag beyond fp32 summation order */
 };
 
 typedef struct {

@@ -9,10 +9,25 @@
 #include <cstdio>
 #include <cstring>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "kernels.cuh"
 #include "tc_gemm.cuh"
+
+// Every kernel is launched with programmatic stream serialization: its blocks may become resident while the kernel
+// before it in the stream drains, and run their set-up; each kernel waits (griddepcontrol.wait) before it touches
+// global memory, so the data dependencies of the stream order are kept.
+template <typename... KArgs, typename... Args>
+void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = grid; lc.blockDim = block; lc.dynamicSmemBytes = smem; lc.stream = st;
+    cudaLaunchAttribute at{};
+    at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at.val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = &at; lc.numAttrs = 1;
+    cudaLaunchKernelEx(&lc, kernel, std::forward<Args>(args)...);
+}
 
 namespace {
 
@@ -304,21 +319,24 @@ void finish_plan(const alexnet* h, Plan& P) {
 // groups, a kh x kw filter over `chunks` 64-channel chunks: the (row halves, BN) pair with the lowest
 // modelled time.  Per weight stage the tensor pipe needs MH*kk*BN/2 cycles; TMA brings about 64 bytes
 // per cycle per SM from L2; tiles are dealt to the SMs in rounds.
-struct ConvShape { int MH, BN, acc_stages, epi_sets; };
+struct ConvShape { int MH, BN, acc_stages, epi_sets, cg; };
 ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, int kh, int kw, int chunks, int kk) {
-    ConvShape best{1, N <= 256 ? N : 128, 1, 1};
+    ConvShape best{1, N <= 256 ? N : 128, 1, 1, 1};
     double best_t = 1e30;
     const int a_rows = kw > 1 ? 136 : 128;
     const size_t budget = 227 * 1024 - 2048 - 4 * tc::kEpiStageBytes;
+    const int cg_lo = (h->cfg.flags & ALEXNET_FLAG_ALL_CTA_PAIRS) ? 2 : 1, cg_hi = (h->cfg.flags & ALEXNET_FLAG_NO_CTA_PAIRS) ? 1 : 2;
+    for (int cg = cg_lo; cg <= cg_hi; ++cg)
     for (int MH = 1; MH <= 4; MH *= 2) {
         for (int BN = 16; BN <= 256 && BN <= N; BN += 16) {
             if (N % BN) continue;
             if (MH * BN > 512) continue;
             const size_t g_tiles = kw <= 3 ? kw : 2;     // weight tiles per group (see finish_conv_plan)
-            if (2 * (size_t)MH * a_rows * 128 + 2 * g_tiles * BN * 128 > budget) continue;
+            if (2 * (size_t)MH * a_rows * 128 + 2 * g_tiles * (BN / cg) * 128 > budget) continue;
             const int acc = 2 * MH * BN <= 512 ? 2 : 1;
-            const long long tiles = ((M + 128 * MH - 1) / (128 * MH)) * (N / BN) * groups;
-            const long long rounds = (tiles + h->sm_count - 1) / h->sm_count;
+            const long long tiles = ((M + 128 * MH * cg - 1) / (128 * MH * cg)) * (N / BN) * groups;
+            const int slots = h->sm_count / cg;
+            const long long rounds = (tiles + slots - 1) / slots;
             // per filter row and chunk: the pipe needs kw*kk*MH*BN/2 cycles; each issuer warp pays about 330 cycles per
             // weight group plus 50 per instruction; all issuers together get about one instruction per 40 cycles
             // dispatched (measured: 4 issuers of N = 64 are slower than one of N = 192); TMA brings about 72 B/cycle,
@@ -326,20 +344,23 @@ ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, in
             const int ngroups = kw <= 3 ? 1 : (kw + 1) / 2;
             const double n_mma = (double)kw * kk;
             const double mma = std::max(std::max(n_mma * MH * BN / 2.0, ngroups * 330.0 + n_mma * 50.0), n_mma * MH * 40.0);
-            const bool shallow = 3 * (size_t)MH * a_rows * 128 + 2 * g_tiles * BN * 128 > budget;
-            const double tma = ((double)MH * a_rows * 128 + (double)kw * BN * 128) / 72.0;
-            double tile_t = (double)kh * chunks * (std::max(mma, tma) + (shallow ? 600.0 : 0.0)) + 800.0;
+            const bool shallow = 3 * (size_t)MH * a_rows * 128 + 2 * g_tiles * (BN / cg) * 128 > budget;
+            const double tma = ((double)MH * a_rows * 128 + (double)kw * (BN / cg) * 128) / 72.0;
+            // a CTA pair issues one instruction for both SMs: measured, its issuers run at about 100 cycles per instruction
+            // where two issuers of one CTA (N = 128) hold each other up at about 150; worth a tenth of the main loop
+            const double pair_gain = cg == 2 ? 0.9 : 1.0;
+            double tile_t = (double)kh * chunks * (std::max(mma, tma) * pair_gain + (shallow ? 600.0 : 0.0)) + 800.0;
             // epilogue per 16 columns and row half: about 450 cycles through the staged TMA store (single staging tile per warp), about 1000 with direct
             // stores (tiles whose 64-column slabs would not fit the group's channel range)
             const bool staged = BN % 64 == 0 || (groups == 1 && N == BN);
             const double epi = MH * (BN / 16) * (staged ? 450.0 : 1000.0);
             // a second set of epilogue warps (each takes every other row half) when the epilogue is the longer side
             for (int E = 1; E <= (MH >= 2 && staged ? 2 : 1); ++E) {
-                if (E == 2 && 2 * (size_t)MH * a_rows * 128 + 2 * g_tiles * BN * 128 + 4 * tc::kEpiStageBytes > budget) continue;
+                if (E == 2 && 2 * (size_t)MH * a_rows * 128 + 2 * g_tiles * (BN / cg) * 128 + 4 * tc::kEpiStageBytes > budget) continue;
                 double tt = tile_t;
                 if (acc == 1) tt += epi / E; else tt = std::max(tt, epi / E + 300.0);
                 const double t = rounds * tt + (E == 2 ? 1.0 : 0.0);     // ties go to the smaller block
-                if (t < best_t) { best_t = t; best = ConvShape{MH, BN, acc, E}; }
+                if (t < best_t) { best_t = t; best = ConvShape{MH, BN, acc, E, cg}; }
             }
         }
     }
@@ -353,7 +374,8 @@ void finish_conv_plan(const alexnet* h, Plan& P) {
     c.asteps_per_split = per;
     c.tiles_total = c.m_tiles * c.n_tiles * c.groups * c.splits;
     if (c.cpg < 1) c.cpg = 1;
-    const size_t a_bytes = (size_t)c.MH * c.cpg * c.a_box_rows * 128, b_bytes = (size_t)c.BN * 128;
+    if (c.cg < 1) c.cg = 1;
+    const size_t a_bytes = (size_t)c.MH * c.cpg * c.a_box_rows * 128, b_bytes = (size_t)(c.BN / c.cg) * 128;
     if (c.epi_sets < 1) c.epi_sets = 1;
     const size_t budget = 227 * 1024 - 2048 - 4 * c.epi_sets * tc::kEpiStageBytes;
     c.tpg = c.cpg > 1 ? c.cpg : (c.kw <= 3 ? c.kw : 2);   // weight tiles travel in groups: a filter row (2 + 2 + 1 taps of a five-tap row, which keeps
@@ -369,7 +391,7 @@ void finish_conv_plan(const alexnet* h, Plan& P) {
     }
     P.conv = true;
     P.smem = tc::conv_smem_bytes(c);
-    P.grid = std::min(c.tiles_total, h->sm_count);
+    P.grid = c.cg * std::min(c.tiles_total, h->sm_count / c.cg);     // persistent: CTAs (or CTA pairs) walk the tile list
     P.valid = true;
 }
 
@@ -394,8 +416,8 @@ int plan_conv_fwd(alexnet* h, Plan& P, const ConvL& c, const bf16* in, const bf1
     const int gp = c.gin.Wp;
     p.kh = p.kw = c.k; p.chunks = (c.cig + 63) / 64; p.kk = c.cig == 48 ? 3 : 4;
     const ConvShape sh = choose_conv_shape(h, M, c.cog, c.groups, p.kh, p.kw, p.chunks, p.kk);
-    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages; p.epi_sets = sh.epi_sets;
-    p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH - 1) / (128 * p.MH));
+    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages; p.epi_sets = sh.epi_sets; p.cg = sh.cg;
+    p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH * p.cg - 1) / (128 * p.MH * p.cg));
     p.n_tiles = c.cog / p.BN; p.groups = c.groups; p.splits = 1;
     p.asteps_total = p.kh * p.chunks;
     p.a_box_rows = p.kw > 1 ? 136 : 128;
@@ -407,7 +429,7 @@ int plan_conv_fwd(alexnet* h, Plan& P, const ConvL& c, const bf16* in, const bf1
     p.relu = 1; p.mask_scale = 1.f; p.bias = bias; p.mask = nullptr; p.out = out; p.status = h->status;
     int rc;
     if ((rc = make_tm(h, &p.tmA, in, c.cin, M, (uint64_t)c.cin * 2, p.a_box_rows))) return rc;
-    if ((rc = make_tm(h, &p.tmB, wsh, c.cig, (uint64_t)c.taps * c.cout, (uint64_t)c.cig * 2, p.BN))) return rc;
+    if ((rc = make_tm(h, &p.tmB, wsh, c.cig, (uint64_t)c.taps * c.cout, (uint64_t)c.cig * 2, p.BN / p.cg))) return rc;
     if ((rc = conv_out_map(h, p, out, c.cout, M))) return rc;
     finish_conv_plan(h, P);
     return ALEXNET_OK;
@@ -419,8 +441,8 @@ int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf1
     const int gp = c.gin.Wp;
     p.kh = p.kw = c.k; p.chunks = c.cog / 64; p.kk = 4;
     const ConvShape sh = choose_conv_shape(h, M, c.cig, c.groups, p.kh, p.kw, p.chunks, p.kk);
-    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages; p.epi_sets = sh.epi_sets;
-    p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH - 1) / (128 * p.MH));
+    p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages; p.epi_sets = sh.epi_sets; p.cg = sh.cg;
+    p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH * p.cg - 1) / (128 * p.MH * p.cg));
     p.n_tiles = c.cig / p.BN; p.groups = c.groups; p.splits = 1;
     p.asteps_total = p.kh * p.chunks;
     p.a_box_rows = p.kw > 1 ? 136 : 128;
@@ -433,7 +455,7 @@ int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf1
     p.relu = 0; p.mask_scale = 1.f; p.bias = nullptr; p.mask = mask; p.out = dx; p.status = h->status;
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, p.a_box_rows))) return rc;
-    if ((rc = make_tm(h, &p.tmB, wt, c.cog, (uint64_t)c.taps * c.cin, (uint64_t)c.cog * 2, p.BN))) return rc;
+    if ((rc = make_tm(h, &p.tmB, wt, c.cog, (uint64_t)c.taps * c.cin, (uint64_t)c.cog * 2, p.BN / p.cg))) return rc;
     if ((rc = conv_out_map(h, p, dx, c.cin, M))) return rc;
     finish_conv_plan(h, P);
     return ALEXNET_OK;
@@ -472,7 +494,7 @@ int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* ws
     tc::ConvParams& p = P.c;
     const int B = h->B;
     p.kh = p.kw = 1; p.cpg = 2; p.chunks = f.K / 64 / p.cpg; p.kk = 4;   // K is a multiple of 128 in all three layers
-    p.MH = 1; p.BN = fc_fwd_bn(f); p.acc_stages = 2;
+    p.MH = 1; p.BN = fc_fwd_bn(f); p.acc_stages = 2; p.cg = 1;
     p.M_total = B; p.m_tiles = (B + 127) / 128; p.n_tiles = (f.N + p.BN - 1) / p.BN;
     p.groups = 1; p.splits = fc_fwd_splits(f, B);
     p.asteps_total = p.chunks;
@@ -575,9 +597,20 @@ void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
         }
     }
     if (h->prof) cudaEventRecord(h->prof_ev[h->prof_used], st);
-    if (P.wgrad) tc::wgrad_kernel<<<P.grid, tc::wgrad_threads(P.w), P.smem, st>>>(P.w);
-    else if (P.conv) tc::conv_kernel<<<P.grid, tc::conv_threads(P.c), P.smem, st>>>(P.c);
-    else tc::gemm_kernel<<<P.grid, tc::kThreads, P.smem, st>>>(P.p);
+    if (P.wgrad) launch_k(tc::wgrad_kernel, P.grid, tc::wgrad_threads(P.w), P.smem, st, P.w);
+    else if (P.conv && P.c.cg == 2) {
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3(P.grid); lc.blockDim = dim3(tc::conv_threads(P.c)); lc.dynamicSmemBytes = P.smem; lc.stream = st;
+        cudaLaunchAttribute at[2] = {};
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[1].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at; lc.numAttrs = 2;
+        cudaLaunchKernelEx(&lc, tc::conv_kernel<2>, P.c);
+    }
+    else if (P.conv) launch_k(tc::conv_kernel<1>, P.grid, tc::conv_threads(P.c), P.smem, st, P.c);
+    else launch_k(tc::gemm_kernel, P.grid, tc::kThreads, P.smem, st, P.p);
     if (h->prof) {
         cudaEventRecord(h->prof_ev[h->prof_used + 1], st);
         h->prof_kind.push_back(P.conv ? 0 : P.wgrad ? 1 : 2);
@@ -587,23 +620,23 @@ void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
 }
 void colsum(alexnet* h, const bf16* dy, long long rows, int C, float* db, cudaStream_t st) {
     if (C % 8) {
-        kn::colsum_scalar_kernel<<<nblk(C, 128), 128, 0, st>>>(dy, (int)rows, C, db);
+        launch_k(kn::colsum_scalar_kernel, nblk(C, 128), 128, 0, st, dy, (int)rows, C, db);
         h->launches++;
         return;
     }
     int splits = (int)std::min<long long>(256, std::max<long long>(1, rows / 256));
     dim3 grid((C + 63) / 64, splits);
-    kn::colsum_kernel<<<grid, 256, 0, st>>>(dy, rows, C, h->cs_partial);
-    kn::colsum_final_kernel<<<nblk(C, 128), 128, 0, st>>>(h->cs_partial, splits, C, db);
+    launch_k(kn::colsum_kernel, grid, 256, 0, st, dy, rows, C, h->cs_partial);
+    launch_k(kn::colsum_final_kernel, nblk(C, 128), 128, 0, st, h->cs_partial, splits, C, db);
     h->launches += 2;
 }
 void refresh_shadows(alexnet* h, int r, bool whole, cudaStream_t st) {
     Replica& R = h->rep[r];
     if (whole) {
-        kn::shadow_kernel<<<1184, 256, 0, st>>>(R.w, R.shadow, h->L.n_total / 4);
+        launch_k(kn::shadow_kernel, 1184, 256, 0, st, R.w, R.shadow, h->L.n_total / 4);
         h->launches++;
     }
-    kn::conv_transpose_shadow_kernel<<<592, 256, 0, st>>>(R.shadow, R.wt, h->L.tjobs);
+    launch_k(kn::conv_transpose_shadow_kernel, 592, 256, 0, st, R.shadow, R.wt, h->L.tjobs);
     h->launches++;
 }
 
@@ -615,7 +648,7 @@ void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
     const Plan& P = R.conv_wg[l][slot];
     launch_gemm(h, P, st);     // weight-gradient partials per row split, and the bias-gradient partials
     const long long total = (long long)c.taps * c.cout * c.cig;
-    kn::wgrad_reduce_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.w.splits, P.w.split_stride, total, R.g + c.w_off, l == 0,
+    launch_k(kn::wgrad_reduce_kernel, nblk(total, 256), 256, 0, st, h->ws, P.w.splits, P.w.split_stride, total, R.g + c.w_off, l == 0,
                                                               h->cs_partial, c.cout, R.g + c.b_off);
     h->launches++;
 }
@@ -634,7 +667,7 @@ void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool ev
         scale = (h->cfg.flags & ALEXNET_FLAG_INVERTED_DROPOUT) ? 1.f : 1.f - h->cfg.dropout_p;
     }
     const uint64_t key = kn::stream_key(h->cfg.seed, 2 + l, r, step);
-    kn::fc_reduce_fwd_kernel<<<nblk(total, 256), 256, 0, st>>>(h->ws, P.c.splits, P.c.split_stride, R.w + f.b_off, h->B, f.N,
+    launch_k(kn::fc_reduce_fwd_kernel, nblk(total, 256), 256, 0, st, h->ws, P.c.splits, P.c.split_stride, R.w + f.b_off, h->B, f.N,
                                                                 l < 2, drop, key, h->thr24, scale, outs[l],
                                                                 l == 2 ? R.z : nullptr, keeps[l]);
     h->launches++;
@@ -648,7 +681,7 @@ void op_fc_bwd(alexnet* h, int r, int l, cudaStream_t st) {
     bf16* outs[3] = {R.dp5, R.df6, R.df7};
     // the data gradient of layer l is the output gradient of layer l-1: its column sums are that layer's bias gradient
     float* db = l > 0 ? R.g + h->L.fc[l - 1].b_off : nullptr;
-    kn::fc_reduce_bwd_kernel<<<nblk(f.K, 32), 1024, 0, st>>>(h->ws, P.p.splits, P.p.split_stride, masks[l], h->drop_scale, h->B, f.K,
+    launch_k(kn::fc_reduce_bwd_kernel, nblk(f.K, 32), 1024, 0, st, h->ws, P.p.splits, P.p.split_stride, masks[l], h->drop_scale, h->B, f.K,
                                                            outs[l], db);
     h->launches++;
 }
@@ -666,7 +699,7 @@ void op_lrn_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     R.n_stale[which] = false;
     const Grid& g = h->L.conv[which].gout;
     const long long rows = (long long)h->B * g.Hp * g.Wp;
-    kn::lrn_fwd_kernel<<<nblk(rows * (g.C / 8), 256), 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.n2 : R.n1,
+    launch_k(kn::lrn_fwd_kernel, nblk(rows * (g.C / 8), 256), 256, 0, st, which ? R.a2 : R.a1, which ? R.n2 : R.n1,
                                                                    (unsigned)(rows * (g.C / 8)), (unsigned)(g.C / 8),
                                                                    h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
     h->launches++;
@@ -675,7 +708,7 @@ void op_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
     const Grid& g = h->L.conv[which].gout;
     const long long rows = (long long)h->B * g.Hp * g.Wp;
-    kn::lrn_bwd_kernel<<<nblk(rows * (g.C / 8), 256), 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.dn2 : R.dn1,
+    launch_k(kn::lrn_bwd_kernel, nblk(rows * (g.C / 8), 256), 256, 0, st, which ? R.a2 : R.a1, which ? R.dn2 : R.dn1,
                                                                    which ? R.da2 : R.da1, (unsigned)(rows * (g.C / 8)),
                                                                    (unsigned)(g.C / 8), h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
     h->launches++;
@@ -689,7 +722,7 @@ void op_pool_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     bf16* y[3] = {R.p1, R.p2, R.p5};
     uint8_t* a[3] = {R.arg1, R.arg2, R.arg5};
     const dim3 grid(nblk((long long)g.Wo * (g.C / 8), 256), g.Ho, h->B);
-    kn::pool_fwd_kernel<<<grid, 256, 0, st>>>(x[which], y[which], a[which], g.C / 8, g.Hpi, g.Wpi, g.Ho, g.Wo, g.Hpo, g.Wpo);
+    launch_k(kn::pool_fwd_kernel, grid, 256, 0, st, x[which], y[which], a[which], g.C / 8, g.Hpi, g.Wpi, g.Ho, g.Wo, g.Hpo, g.Wpo);
     h->launches++;
 }
 void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
@@ -701,7 +734,7 @@ void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     const bf16* relu[3] = {nullptr, nullptr, R.a5};
     bf16* dx[3] = {R.dn1, R.dn2, R.da5};
     const dim3 grid(nblk((long long)g.Wpi * (g.C / 8), 256), g.Hpi, h->B);
-    kn::pool_bwd_kernel<<<grid, 256, 0, st>>>(dy[which], a[which], relu[which], dx[which], g.C / 8, g.Hpi, g.Wpi,
+    launch_k(kn::pool_bwd_kernel, grid, 256, 0, st, dy[which], a[which], relu[which], dx[which], g.C / 8, g.Hpi, g.Wpi,
                                               g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo, g.Wpo);
     h->launches++;
 }
@@ -711,7 +744,7 @@ void op_lrn_pool_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     const int cpr = g.C / 8;
     const dim3 grid((g.Ho + 1) / 2, h->B);
     const size_t smem = (size_t)5 * g.Wi * cpr * 16;
-    kn::lrn_pool_fwd_kernel<<<grid, 256, smem, st>>>(which ? R.a2 : R.a1, which ? R.p2 : R.p1, which ? R.arg2 : R.arg1, cpr, g.Hpi,
+    launch_k(kn::lrn_pool_fwd_kernel, grid, 256, smem, st, which ? R.a2 : R.a1, which ? R.p2 : R.p1, which ? R.arg2 : R.arg1, cpr, g.Hpi,
                                                      g.Wpi, g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta,
                                                      h->cfg.lrn_k);
     h->launches++;
@@ -722,7 +755,7 @@ void op_pool_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     const PoolGeo& g = kPool[which];
     const int cpr = g.C / 8, ppb = 256 / cpr;
     const dim3 grid((g.Wpi + ppb - 1) / ppb, g.Hpi, h->B);
-    kn::pool_lrn_bwd_kernel<<<grid, 256, 0, st>>>(which ? R.a2 : R.a1, which ? R.dp2 : R.dp1, which ? R.arg2 : R.arg1,
+    launch_k(kn::pool_lrn_bwd_kernel, grid, 256, 0, st, which ? R.a2 : R.a1, which ? R.dp2 : R.dp1, which ? R.arg2 : R.arg1,
                                                   which ? R.da2 : R.da1, cpr, ppb, g.Hpi, g.Wpi, g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo,
                                                   g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
     h->launches++;
@@ -730,8 +763,8 @@ void op_pool_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
 }
 void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
     Replica& R = h->rep[r];
-    kn::softmax_xent_kernel<<<h->B, 256, 0, st>>>(R.z, R.labels[slot], R.dz, R.loss_n, h->B, 1000);
-    kn::mean_kernel<<<1, 256, 0, st>>>(R.loss_n, h->B, R.loss);
+    launch_k(kn::softmax_xent_kernel, h->B, 256, 0, st, R.z, R.labels[slot], R.dz, R.loss_n, h->B, 1000);
+    launch_k(kn::mean_kernel, 1, 256, 0, st, R.loss_n, h->B, R.loss);
     h->launches += 2;
 }
 void op_update(alexnet* h, int r, cudaStream_t st, bool full = false) {
@@ -740,14 +773,14 @@ void op_update(alexnet* h, int r, cudaStream_t st, bool full = false) {
     // all conv filters precede the FC weights in the internal order
     // with the fused FC update the FC weights (a contiguous range of the internal order) are already up to date
     const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0 && !full;
-    kn::sgd_update_kernel<<<1184, 256, 0, st>>>(R.w, R.v, R.g, R.shadow, h->L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum,
+    launch_k(kn::sgd_update_kernel, 1184, 256, 0, st, R.w, R.v, R.g, R.shadow, h->L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum,
                                                 h->cfg.weight_decay, R.wt, h->L.tjobs, h->L.fc[0].w_off / 4,
                                                 fused ? h->L.fc[0].w_off / 4 : 0, fused ? h->L.n_weights / 4 : 0);
     h->launches++;
 }
 void op_average(alexnet* h, cudaStream_t st) {
     Replica &A = h->rep[0], &Bq = h->rep[1];
-    kn::replica_average_kernel<<<1184, 256, 0, st>>>(A.w, Bq.w, A.v, Bq.v, A.shadow, Bq.shadow, h->L.n_total / 4);
+    launch_k(kn::replica_average_kernel, 1184, 256, 0, st, A.w, Bq.w, A.v, Bq.v, A.shadow, Bq.shadow, h->L.n_total / 4);
     h->launches++;
     refresh_shadows(h, 0, false, st);
     refresh_shadows(h, 1, false, st);
@@ -755,7 +788,7 @@ void op_average(alexnet* h, cudaStream_t st) {
 void op_preprocess(alexnet* h, int r, int slot, uint64_t step, cudaStream_t st, bool eval = false) {
     Replica& R = h->rep[r];
     const long long total = (long long)h->B * 57 * 57 * 4;
-    kn::preprocess_kernel<<<nblk(total, 256), 256, 0, st>>>(R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
+    launch_k(kn::preprocess_kernel, nblk(total, 256), 256, 0, st, R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
                                                             kn::stream_key(h->cfg.seed, 1, r, step), eval ? 1 : 0);
     h->launches++;
 }
@@ -803,6 +836,7 @@ int poll_status(alexnet* h) {  // after a synchronisation
 
 // N(0, std^2) init from the hash (stream 6), identical in every replica; written at internal positions
 __global__ void init_kernel(float* arena, const kn::ParamSegs segs, uint64_t key, float std_) {
+    kn::pdl_sync();
     const long long stride = (long long)gridDim.x * blockDim.x;
     const long long total = 60965224;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
@@ -927,7 +961,8 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     if (!fn || qres != cudaDriverEntryPointSuccess) { delete h; return ALEXNET_ERR_CUDA; }
     h->encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
     CKC(cudaFuncSetAttribute(tc::gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    CKC(cudaFuncSetAttribute(tc::conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CKC(cudaFuncSetAttribute(tc::conv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CKC(cudaFuncSetAttribute(tc::conv_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(kn::lrn_pool_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
     {
@@ -948,7 +983,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
             R.consumed_valid[s] = false; R.slot_step[s] = 0;
         }
         if (cfg->init_std > 0.f) {
-            init_kernel<<<1184, 256, 0, h->cs>>>(R.w, h->L.segs, kn::stream_key(cfg->seed, 6, 0, 0), cfg->init_std);
+            launch_k(init_kernel, 1184, 256, 0, h->cs, R.w, h->L.segs, kn::stream_key(cfg->seed, 6, 0, 0), cfg->init_std);
             h->launches++;
         }
         refresh_shadows(h, r, true, h->cs);
@@ -1029,7 +1064,7 @@ int alexnet_eval_batch(alexnet_t* h, int replica, const uint8_t* images, const i
     forward(h, replica, s, h->cs, true);
     int32_t* counts = (int32_t*)(h->status + 4);    // two counters in the status block
     CK(cudaMemsetAsync(counts, 0, 2 * sizeof(int32_t), h->cs));
-    kn::topk_count_kernel<<<h->B, 256, 0, h->cs>>>(R.z, R.labels[s], 1000, counts);
+    launch_k(kn::topk_count_kernel, h->B, 256, 0, h->cs, R.z, R.labels[s], 1000, counts);
     h->launches++;
     CK(cudaEventRecord(R.consumed[s], h->cs));
     R.consumed_valid[s] = true;
@@ -1060,7 +1095,7 @@ int alexnet_get_params(alexnet_t* h, int replica, int which, float* host_out, si
         return fail(h, ALEXNET_ERR_ARG, "get_params: bad argument");
     Replica& R = h->rep[replica];
     const float* src = which == 0 ? R.w : which == 1 ? R.v : R.g;
-    kn::params_gather_kernel<<<1184, 256, 0, h->cs>>>(src, h->canon_tmp, h->L.segs, kCanonCount);
+    launch_k(kn::params_gather_kernel, 1184, 256, 0, h->cs, src, h->canon_tmp, h->L.segs, kCanonCount);
     h->launches++;
     CK(cudaMemcpyAsync(host_out, h->canon_tmp, n * sizeof(float), cudaMemcpyDeviceToHost, h->cs));
     CK(cudaStreamSynchronize(h->cs));
@@ -1075,7 +1110,7 @@ int alexnet_set_params(alexnet_t* h, int replica, int which, const float* host_i
     float* dst = which == 0 ? R.w : R.v;
     CK(cudaMemcpyAsync(h->canon_tmp, host_in, n * sizeof(float), cudaMemcpyHostToDevice, h->cs));
     CK(cudaMemsetAsync(dst, 0, h->L.n_total * sizeof(float), h->cs));
-    kn::params_scatter_kernel<<<1184, 256, 0, h->cs>>>(dst, h->canon_tmp, h->L.segs, kCanonCount);
+    launch_k(kn::params_scatter_kernel, 1184, 256, 0, h->cs, dst, h->canon_tmp, h->L.segs, kCanonCount);
     h->launches++;
     if (which == 0) refresh_shadows(h, replica, true, h->cs);
     CK(cudaStreamSynchronize(h->cs));
@@ -1301,8 +1336,8 @@ extern "C" int alexnet_bias_grad_noalloc(const void* dev_dy, int64_t rows, int32
     cudaStream_t st = (cudaStream_t)stream;
     int splits = (int)std::min<int64_t>(kNoAllocSplits, std::max<int64_t>(1, rows / 256));
     dim3 grid((channels + 63) / 64, splits);
-    kn::colsum_kernel<<<grid, 256, 0, st>>>((const bf16*)dev_dy, (long long)rows, channels, scratch);
-    kn::colsum_final_kernel<<<(channels + 127) / 128, 128, 0, st>>>(scratch, splits, channels, dev_db);
+    launch_k(kn::colsum_kernel, grid, 256, 0, st, (const bf16*)dev_dy, (long long)rows, channels, scratch);
+    launch_k(kn::colsum_final_kernel, (channels + 127) / 128, 128, 0, st, scratch, splits, channels, dev_db);
     e = cudaGetLastError();
     if (e != cudaSuccess) { put_err(err, err_len, cudaGetErrorString(e)); return ALEXNET_ERR_CUDA; }
     return ALEXNET_OK;

@@ -11,6 +11,13 @@
 
 namespace kn {
 
+// Programmatic dependent launch: every kernel of the step lets the next launch of its stream start its blocks early
+// (they become resident as the SMs drain) and itself waits here, before its first access to global memory, until the
+// kernels before it have completed and their writes are visible.  Without the launch attribute both are no-ops.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_sync() { pdl_trigger(); pdl_wait(); }
+
 // ---------------------------------------------------------------- counter hash
 // SplitMix64 finaliser over key + golden*(idx+1); key = finalise(seed ^ stream<<56 ^ replica<<48 ^ step).
 __host__ __device__ __forceinline__ uint64_t mix64(uint64_t z) {
@@ -47,6 +54,7 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 __global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* __restrict__ mean,
                                   __nv_bfloat16* __restrict__ out, int32_t* __restrict__ cf_out,
                                   int B, uint64_t key, int eval_mode) {
+    pdl_sync();
     // one thread per (n, by, bx, dy): 12 output values (4 dx * 3 colours) = 24 bytes
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long total = (long long)B * 57 * 57 * 4;
@@ -113,6 +121,7 @@ __device__ __forceinline__ uint4 lrn_fwd8(const uint4* ap, bool has_l, bool has_
 }
 __global__ void __launch_bounds__(256) lrn_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ b,
                                                       unsigned total, unsigned cpr, float alpha, float beta, float k) {
+    pdl_sync();
     const unsigned t = blockIdx.x * 256u + threadIdx.x;
     if (t >= total) return;
     const unsigned ch = t % cpr;
@@ -147,6 +156,7 @@ __device__ __forceinline__ uint4 lrn_bwd8(const float* fa, const float* fg, floa
 __global__ void __launch_bounds__(256) lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ g,
                                                       __nv_bfloat16* __restrict__ da, unsigned total, unsigned cpr,
                                                       float alpha, float beta, float k) {
+    pdl_sync();
     const unsigned t = blockIdx.x * 256u + threadIdx.x;
     if (t >= total) return;
     const unsigned ch = t % cpr;
@@ -170,6 +180,7 @@ __global__ void __launch_bounds__(256) lrn_bwd_kernel(const __nv_bfloat16* __res
 __global__ void __launch_bounds__(256) pool_fwd_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
                                                        uint8_t* __restrict__ arg, int cpr, int Hpi, int Wpi,
                                                        int Ho, int Wo, int Hpo, int Wpo) {
+    pdl_sync();
     const unsigned i = blockIdx.x * 256u + threadIdx.x;
     if (i >= (unsigned)(Wo * cpr)) return;
     const int ox = i / cpr, ch = i - ox * cpr;
@@ -216,6 +227,7 @@ __device__ __forceinline__ void pool_bwd8(const __nv_bfloat16* __restrict__ dy, 
 __global__ void __launch_bounds__(256) pool_bwd_kernel(const __nv_bfloat16* __restrict__ dy, const uint8_t* __restrict__ arg,
                                                        const __nv_bfloat16* __restrict__ relu_src, __nv_bfloat16* __restrict__ dx,
                                                        int cpr, int Hpi, int Wpi, int Hi, int Wi, int Ho, int Wo, int Hpo, int Wpo) {
+    pdl_sync();
     const unsigned i = blockIdx.x * 256u + threadIdx.x;
     if (i >= (unsigned)(Wpi * cpr)) return;
     const int x = i / cpr, ch = i - x * cpr;
@@ -242,6 +254,7 @@ __global__ void __launch_bounds__(256) pool_bwd_kernel(const __nv_bfloat16* __re
 __global__ void __launch_bounds__(256) lrn_pool_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ y,
                                                            uint8_t* __restrict__ arg, int cpr, int Hpi, int Wpi, int Hi, int Wi,
                                                            int Ho, int Wo, int Hpo, int Wpo, float alpha, float beta, float k) {
+    pdl_sync();
     extern __shared__ uint4 nrm[];            // [row][x][chunk]
     const int n = blockIdx.y, oy0 = 2 * blockIdx.x;
     const int iy0 = 2 * oy0, nrows = min(5, Hi - iy0);
@@ -284,6 +297,7 @@ __global__ void __launch_bounds__(256) pool_lrn_bwd_kernel(const __nv_bfloat16* 
                                                            const uint8_t* __restrict__ arg, __nv_bfloat16* __restrict__ da,
                                                            int cpr, int ppb, int Hpi, int Wpi, int Hi, int Wi, int Ho, int Wo,
                                                            int Hpo, int Wpo, float alpha, float beta, float k) {
+    pdl_sync();
     __shared__ float4 edge[256];      // tt of the two lowest and two highest channels of every thread, for its neighbours
     const int px = threadIdx.x / cpr, ch = threadIdx.x - px * cpr;
     const int x = blockIdx.x * ppb + px, y = blockIdx.y, n = blockIdx.z;
@@ -346,6 +360,7 @@ __global__ void fc_reduce_fwd_kernel(const float* __restrict__ ws, int splits, l
                                      int use_dropout, uint64_t key, uint32_t thr24, float scale,
                                      __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32,
                                      uint8_t* __restrict__ keep_out) {
+    pdl_sync();
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= (long long)B * N) return;
     const int n = (int)(t % N);
@@ -371,6 +386,7 @@ __global__ void fc_reduce_fwd_kernel(const float* __restrict__ ws, int splits, l
 __global__ void __launch_bounds__(1024) fc_reduce_bwd_kernel(const float* __restrict__ ws, int splits, long long split_stride,
                                                              const __nv_bfloat16* __restrict__ mask, float scale, int B, int K,
                                                              __nv_bfloat16* __restrict__ out, float* __restrict__ db) {
+    pdl_sync();
     __shared__ float red[32][33];
     const int c = blockIdx.x * 32 + (threadIdx.x & 31), rl = threadIdx.x >> 5;
     float acc = 0.f;
@@ -400,6 +416,7 @@ __global__ void __launch_bounds__(1024) fc_reduce_bwd_kernel(const float* __rest
 __global__ void wgrad_reduce_kernel(const float* __restrict__ ws, int splits, long long split_stride,
                                     long long total, float* __restrict__ g, int conv1_pad_mask,
                                     const float* __restrict__ bias_partial, int cout, float* __restrict__ db) {
+    pdl_sync();
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= total) return;
     float v = 0.f;
@@ -420,6 +437,7 @@ __global__ void wgrad_reduce_kernel(const float* __restrict__ ws, int splits, lo
 // db[c] = sum over rows of dy[row][c] (bf16 in, fp32 out), two stages: grid (ceil(C/64), row_splits)
 // writes partial[split][C]; colsum_final_kernel adds the splits in a fixed order.
 __global__ void colsum_kernel(const __nv_bfloat16* __restrict__ dy, long long rows, int C, float* __restrict__ partial) {
+    pdl_sync();
     // block: 256 threads = 32 row-lanes x 8 column-chunks (8 channels each) -> 64 columns per block
     __shared__ float red[32][65];
     const int cc = threadIdx.x & 7, rl = threadIdx.x >> 3;
@@ -446,6 +464,7 @@ __global__ void colsum_kernel(const __nv_bfloat16* __restrict__ dy, long long ro
     }
 }
 __global__ void colsum_final_kernel(const float* __restrict__ partial, int splits, int C, float* __restrict__ db) {
+    pdl_sync();
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= C) return;
     float s = 0.f;
@@ -454,6 +473,7 @@ __global__ void colsum_final_kernel(const float* __restrict__ partial, int split
 }
 // same for a row pitch that is not a multiple of 8 elements (the 1000-wide logits gradient)
 __global__ void colsum_scalar_kernel(const __nv_bfloat16* __restrict__ dy, int rows, int C, float* __restrict__ db) {
+    pdl_sync();
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= C) return;
     float s = 0.f;
@@ -465,6 +485,7 @@ __global__ void colsum_scalar_kernel(const __nv_bfloat16* __restrict__ dy, int r
 // one block per sample: p = softmax(z), loss_n = -log p[label], dz = (p - onehot)/B as bf16
 __global__ void softmax_xent_kernel(const float* __restrict__ z, const int32_t* __restrict__ labels,
                                     __nv_bfloat16* __restrict__ dz, float* __restrict__ loss_n, int B, int N) {
+    pdl_sync();
     __shared__ float red[32];
     const int n = blockIdx.x, tid = threadIdx.x;
     const float* zr = z + (size_t)n * N;
@@ -492,6 +513,7 @@ __global__ void softmax_xent_kernel(const float* __restrict__ z, const int32_t* 
     if (tid == 0) loss_n[n] = -(zr[lab] - mx - logf(sum));
 }
 __global__ void mean_kernel(const float* __restrict__ v, int n, float* __restrict__ out) {
+    pdl_sync();
     __shared__ float red[32];
     float s = 0.f;
     for (int i = threadIdx.x; i < n; i += blockDim.x) s += v[i];
@@ -509,6 +531,7 @@ __global__ void mean_kernel(const float* __restrict__ v, int n, float* __restric
 // logits with a smaller class index; the sample counts for top-k when rank < k.  counts[0] += top-1, counts[1] += top-5
 // (integer atomics: the result does not depend on the order).
 __global__ void topk_count_kernel(const float* __restrict__ z, const int32_t* __restrict__ labels, int N, int32_t* __restrict__ counts) {
+    pdl_sync();
     __shared__ int red[32];
     const int n = blockIdx.x, lab = labels[n];
     const float* zr = z + (size_t)n * N;
@@ -548,6 +571,7 @@ __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, 
                                   __nv_bfloat16* __restrict__ shadow, long long n4, long long n_decay4,
                                   float lr, float mu, float wd, __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs,
                                   long long conv_end4, long long skip_begin4, long long skip_end4) {
+    pdl_sync();
     // vectors [0, n4) except [skip_begin4, skip_end4): the FC weights, when the FC weight-gradient kernel has already
     // updated them in its epilogue
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -588,6 +612,7 @@ __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, 
 __global__ void replica_average_kernel(float* __restrict__ wa, float* __restrict__ wb, float* __restrict__ va,
                                        float* __restrict__ vb, __nv_bfloat16* __restrict__ sa,
                                        __nv_bfloat16* __restrict__ sb, long long n4) {
+    pdl_sync();
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
         const float4 a = ((float4*)wa)[i], b = ((float4*)wb)[i];
@@ -602,6 +627,7 @@ __global__ void replica_average_kernel(float* __restrict__ wa, float* __restrict
     }
 }
 __global__ void shadow_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ shadow, long long n4) {
+    pdl_sync();
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
         const float4 wv = ((const float4*)w)[i];
@@ -612,6 +638,7 @@ __global__ void shadow_kernel(const float* __restrict__ w, __nv_bfloat16* __rest
 
 __global__ void conv_transpose_shadow_kernel(const __nv_bfloat16* __restrict__ shadow, __nv_bfloat16* __restrict__ wt,
                                              const TransposeJobs jobs) {
+    pdl_sync();
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (int q = 0; q < jobs.n; ++q) {
         const TransposeJob J = jobs.j[q];
@@ -651,6 +678,7 @@ __device__ __forceinline__ long long canon_to_internal(const ParamSeg& S, long l
 }
 __global__ void params_gather_kernel(const float* __restrict__ arena, float* __restrict__ canon, const ParamSegs segs,
                                      long long total) {
+    pdl_sync();
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
         int s = 0;
@@ -660,6 +688,7 @@ __global__ void params_gather_kernel(const float* __restrict__ arena, float* __r
 }
 __global__ void params_scatter_kernel(float* __restrict__ arena, const float* __restrict__ canon, const ParamSegs segs,
                                       long long total) {
+    pdl_sync();
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
         int s = 0;

@@ -156,6 +156,51 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\t"
                  "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar) : "memory");
 }
+// ---- CTA pairs (cta_group::2): one instruction of the leader CTA (cluster rank 0) multiplies a 256-row A (128 rows
+// from each CTA's shared memory) by an N-column B (N/2 columns from each CTA) into 128 TMEM lanes of each CTA.
+__device__ __forceinline__ uint32_t cluster_ctarank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+// shared::cluster address of the same shared-memory offset in the CTA of the given cluster rank
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+    uint32_t r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank)); return r;
+}
+// all threads of all CTAs of the cluster
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void fence_acq_rel_cluster() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+// load into this CTA's shared memory, completion counted on a barrier of either CTA of the pair (cluster address)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t cluster_bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+template <int CG>
+__device__ __forceinline__ void umma_cg(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+    if (CG == 1) { umma(d_tmem, adesc, bdesc, idesc, accum); return; }
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\telect.sync _|q, 0xffffffff;\n\t"
+        "@q tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum) : "memory");
+}
+// completion of the issuing thread's MMAs arrives on the barrier at this shared-memory offset in both CTAs of the pair
+template <int CG>
+__device__ __forceinline__ void umma_commit_cg(uint32_t bar) {
+    if (CG == 1) { umma_commit(bar); return; }
+    const uint16_t both = 3;
+    asm volatile("{\n\t.reg .pred q;\n\telect.sync _|q, 0xffffffff;\n\t"
+                 "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
+                 ::"r"(bar), "h"(both) : "memory");
+}
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -198,8 +243,8 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     d |= (uint64_t)2 << 61;
     return d;
 }
-// instruction descriptor: bf16 x bf16 -> fp32, M = 128
-__device__ __forceinline__ uint32_t instr_desc(int N, int a_mn, int b_mn) {
+// instruction descriptor: bf16 x bf16 -> fp32, M = 128 (256 for a CTA pair: 128 rows per CTA)
+__device__ __forceinline__ uint32_t instr_desc(int N, int a_mn, int b_mn, int M = 128) {
     uint32_t d = 0;
     d |= 1u << 4;                 // D format fp32
     d |= 1u << 7;                 // A bf16
@@ -207,7 +252,7 @@ __device__ __forceinline__ uint32_t instr_desc(int N, int a_mn, int b_mn) {
     d |= (uint32_t)a_mn << 15;    // A major (0 = K)
     d |= (uint32_t)b_mn << 16;    // B major
     d |= (uint32_t)(N >> 3) << 17;
-    d |= (uint32_t)(128 >> 4) << 24;
+    d |= (uint32_t)(M >> 4) << 24;
     return d;
 }
 
@@ -376,6 +421,7 @@ struct TileCursor {
 };
 
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+    kn::pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -411,6 +457,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    kn::pdl_wait();        // barriers, TMEM and descriptors are set up; global memory is touched from here on
     const int per = p.steps_per_split;
 
     if (warp == 0) {
@@ -660,7 +707,8 @@ struct ConvParams {
     int tma_store;
     int m_tiles, n_tiles, groups, splits;   // tile decomposition (m fastest, then n, group, k split)
     int tiles_total;
-    int MH;             // 128-row halves per tile (1, 2 or 4)
+    int cg;             // 1, or 2: CTA pairs (clusters of two) work on tiles of 2 x MH halves with cta_group::2 instructions
+    int MH;             // 128-row halves per tile and CTA (1, 2 or 4)
     int BN, kk;         // MMA N (multiple of 16, <= 256); K=16 MMAs per weight stage (<= 4)
     int kh, kw;         // filter rows; taps per filter row
     int cpg;            // 64-channel chunks per A stage: 1 for convolutions; 2 for FC layers (kw = 1), whose A stage then holds
@@ -690,7 +738,7 @@ struct ConvParams {
 constexpr int kConvMaxThreads = 32 * 12;
 inline int conv_threads(const ConvParams& p) { return 32 * (2 + p.MH + 4 * p.epi_sets); }
 inline size_t conv_smem_bytes(const ConvParams& p) {
-    return 1024 + (size_t)p.a_stages * p.MH * p.cpg * p.a_box_rows * 128 + (size_t)p.b_stages * p.tpg * p.BN * 128 + 4 * p.epi_sets * kEpiStageBytes + 512;
+    return 1024 + (size_t)p.a_stages * p.MH * p.cpg * p.a_box_rows * 128 + (size_t)p.b_stages * p.tpg * (p.BN / p.cg) * 128 + 4 * p.epi_sets * kEpiStageBytes + 512;
 }
 
 // tile cursor shared by the roles (m fastest, then n tile, group, split)
@@ -702,11 +750,13 @@ struct ConvCursor {
         g = r % q.groups;
         z = r / q.groups;
     }
-    __device__ __forceinline__ void init(const ConvParams& q) {
-        m_tile = blockIdx.x % q.m_tiles; rest = blockIdx.x / q.m_tiles; decode(q);
+    int stride;      // tile-list stride: CTAs of the grid, or CTA pairs
+    __device__ __forceinline__ void init(const ConvParams& q, int first, int step) {
+        stride = step;
+        m_tile = first % q.m_tiles; rest = first / q.m_tiles; decode(q);
     }
     __device__ __forceinline__ void next(const ConvParams& q) {
-        m_tile += gridDim.x;
+        m_tile += stride;
         if (m_tile >= q.m_tiles) {
             do { m_tile -= q.m_tiles; ++rest; } while (m_tile >= q.m_tiles);
             decode(q);
@@ -715,7 +765,7 @@ struct ConvCursor {
 };
 
 // MMAs of one filter row (KW taps x KK K=16 steps) on one accumulator, fully unrolled; descriptors in 16-byte units
-template <int KW, int KK>
+template <int KW, int KK, int CG>
 __device__ __forceinline__ void issue_row(uint32_t d, uint64_t ad, uint64_t bd, uint32_t b_tile16, const int* tap_off,
                                           uint32_t idesc, uint32_t accum) {
     #pragma unroll
@@ -723,17 +773,27 @@ __device__ __forceinline__ void issue_row(uint32_t d, uint64_t ad, uint64_t bd, 
         const uint64_t a_tap = ad + (uint64_t)(tap_off[kx] * 8);      // one row = 128 bytes = 8 units
         #pragma unroll
         for (int j = 0; j < KK; ++j)
-            umma(d, a_tap + (uint64_t)(2 * j), bd + (uint64_t)(kx * b_tile16 + 2 * j), idesc, (kx == 0 && j == 0) ? accum : 1u);
+            umma_cg<CG>(d, a_tap + (uint64_t)(2 * j), bd + (uint64_t)(kx * b_tile16 + 2 * j), idesc, (kx == 0 && j == 0) ? accum : 1u);
     }
 }
 
+// CG = 2: the CTAs of a pair (cluster of two) share one tile list.  A tile is 2 x MH x 128 rows; CTA `rank` owns the
+// halves rank*MH .. rank*MH+MH-1, loads their halos and BN/2 rows of every weight tile into its own shared memory
+// (completion counted on the leader's barriers), and runs the epilogue of its halves from its own TMEM.  Only the leader
+// (rank 0) issues: one instruction covers half h of both CTAs, and its commits arrive on the barriers of both.
+template <int CG>
 __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_constant__ ConvParams p) {
+    kn::pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     const int MH = p.MH, BN = p.BN;
+    const int rank = CG == 2 ? (int)cluster_ctarank() : 0;
+    const int vb = CG == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // position and stride in the tile list
+    const int vgrid = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int tile_rows = 128 * MH * CG, row0 = rank * 128 * MH;
     const int cpg = p.cpg, gw = cpg > 1 ? cpg : p.kw;            // weight tiles per A stage
-    const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * 128u, a_bytes = a_box_bytes * MH * cpg, b_bytes = (uint32_t)BN * 128u;
+    const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * 128u, a_bytes = a_box_bytes * MH * cpg, b_bytes = (uint32_t)(BN / CG) * 128u;
     const int a_stages = p.a_stages, b_stages = p.b_stages;
     const uint32_t ring_a = base, ring_b = base + a_stages * a_bytes;
     // epilogue staging (4 * epi_sets warps x kEpiStageBytes), then barriers: fullA[8] @0, emptyA[8] @64, fullB[8] @128,
@@ -755,33 +815,39 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         *abort_flag = 0;
         for (int s = 0; s < a_stages; ++s) { mbar_init(fullA + 8u * s, 1); mbar_init(emptyA + 8u * s, MH); }
         for (int s = 0; s < b_stages; ++s) { mbar_init(fullB + 8u * s, 1); mbar_init(emptyB + 8u * s, MH); }
-        for (int s = 0; s < 2; ++s) { mbar_init(accf0 + 8u * s, MH); mbar_init(acce0 + 8u * s, 128 * p.epi_sets); }
+        for (int s = 0; s < 2; ++s) { mbar_init(accf0 + 8u * s, MH); mbar_init(acce0 + 8u * s, 128 * p.epi_sets * CG); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&p.tmA);
         tma_prefetch_desc(&p.tmB);
     }
-    if (warp == 2) tmem_alloc(smem_u32((const void*)tmem_slot), ncols);
+    if (warp == 2) {
+        if (CG == 2) tmem_alloc_pair(smem_u32((const void*)tmem_slot), ncols);
+        else tmem_alloc(smem_u32((const void*)tmem_slot), ncols);
+    }
     tc_fence_before();
     __syncthreads();
+    __syncwarp();
+    if (CG == 2) cluster_sync_all();          // the peer's barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    kn::pdl_wait();        // barriers, TMEM and descriptors are set up; global memory is touched from here on
     const int per = p.asteps_per_split, kw = p.kw;
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producers: lane 0 of warp 0 feeds the ring of
         // activation halos, lane 0 of warp 1 the ring of weight groups, so that neither ring waits for the other
         if (lane == 0) {
-            ConvCursor tc; tc.init(p);
+            ConvCursor tc; tc.init(p, vb, vgrid);
             int sa = 0; uint32_t pha = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
-                const int m0 = tc.m_tile * (128 * MH);
+            for (int tile = vb; tile < p.tiles_total && ok; tile += vgrid, tc.next(p)) {
+                const int m0 = tc.m_tile * tile_rows + row0;
                 const int a_begin = tc.z * per;
                 const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
                 // the reduction order is free: every CTA starts at a different (filter row, chunk) so that the SMs do not
                 // all ask L2 for the same weight tile at the same moment
                 const int a_end = a_begin + nsteps;
-                int a = a_begin + (int)(blockIdx.x % (unsigned)nsteps);
+                int a = a_begin + (int)((unsigned)vb % (unsigned)nsteps);
                 int ky = a / p.chunks, ch = a - ky * p.chunks;
                 const int ky0 = a_begin / p.chunks, ch0 = a_begin - ky0 * p.chunks;
                 const int xa = p.a_x0 + tc.g * p.a_gx;
@@ -790,10 +856,13 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                     {
                         const uint32_t dst = ring_a + sa * a_bytes, fb = fullA + 8u * sa;
                         const int y = m0 + p.halo_shift[ky];
-                        mbar_expect_tx(fb, a_bytes);
+                        if (rank == 0) mbar_expect_tx(fb, a_bytes * CG);
+                        const uint32_t fbc = CG == 2 ? mapa_u32(fb, 0) : fb;
                         for (int c = 0; c < cpg; ++c)
-                            for (int h = 0; h < MH; ++h)
-                                tma_load_2d(dst + (c * MH + h) * a_box_bytes, &p.tmA, xa + (ch * cpg + c) * 64, y + h * p.a_box_rows, fb);
+                            for (int h = 0; h < MH; ++h) {
+                                if (CG == 2) tma_load_2d_pair(dst + (c * MH + h) * a_box_bytes, &p.tmA, xa + (ch * cpg + c) * 64, y + h * p.a_box_rows, fbc);
+                                else tma_load_2d(dst + (c * MH + h) * a_box_bytes, &p.tmA, xa + (ch * cpg + c) * 64, y + h * p.a_box_rows, fb);
+                            }
                     }
                     if (++sa == a_stages) { sa = 0; pha ^= 1u; }
                     if (++a == a_end) { a = a_begin; ky = ky0; ch = ch0; } else if (++ch == p.chunks) { ch = 0; ++ky; }
@@ -802,17 +871,17 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            ConvCursor tc; tc.init(p);
+            ConvCursor tc; tc.init(p, vb, vgrid);
             int sb = 0; uint32_t phb = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
-                const int n0 = tc.n_tile * BN;
+            for (int tile = vb; tile < p.tiles_total && ok; tile += vgrid, tc.next(p)) {
+                const int n0 = tc.n_tile * BN + rank * (BN / CG);       // this CTA's rows of the weight tile
                 const int a_begin = tc.z * per;
                 const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
                 // the reduction order is free: every CTA starts at a different (filter row, chunk) so that the SMs do not
                 // all ask L2 for the same weight tile at the same moment
                 const int a_end = a_begin + nsteps;
-                int a = a_begin + (int)(blockIdx.x % (unsigned)nsteps);
+                int a = a_begin + (int)((unsigned)vb % (unsigned)nsteps);
                 int ky = a / p.chunks, ch = a - ky * p.chunks;
                 const int ky0 = a_begin / p.chunks, ch0 = a_begin - ky0 * p.chunks;
                 const int yb = tc.g * p.b_g_rows + n0;
@@ -823,9 +892,12 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                         if (!(ok = mbar_wait(emptyB + 8u * sb, phb ^ 1u, abort_flag))) break;
                         const uint32_t fb = fullB + 8u * sb, dst = ring_b + sb * g_bytes;
                         const int taps = min(p.tpg, gw - kx0);
-                        mbar_expect_tx(fb, (uint32_t)taps * b_bytes);
-                        for (int t = 0; t < taps; ++t, brow += brow_step, bcol += bcol_step)
-                            tma_load_2d(dst + t * b_bytes, &p.tmB, bcol, brow, fb);
+                        if (rank == 0) mbar_expect_tx(fb, (uint32_t)taps * b_bytes * CG);
+                        const uint32_t fbc = CG == 2 ? mapa_u32(fb, 0) : fb;
+                        for (int t = 0; t < taps; ++t, brow += brow_step, bcol += bcol_step) {
+                            if (CG == 2) tma_load_2d_pair(dst + t * b_bytes, &p.tmB, bcol, brow, fbc);
+                            else tma_load_2d(dst + t * b_bytes, &p.tmB, bcol, brow, fb);
+                        }
                         if (++sb == b_stages) { sb = 0; phb ^= 1u; }
                     }
                     if (++a == a_end) { a = a_begin; ky = ky0; ch = ch0; } else if (++ch == p.chunks) { ch = 0; ++ky; }
@@ -834,21 +906,22 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         }
     } else if (warp <= MH + 1) {
         // ------------------------------------------------------------ MMA issuer of row half h (whole warp)
-        {
+        if (rank == 0) {
             const int h = warp - 2;
-            const uint32_t idesc = instr_desc(BN, 0, 0);
+            const uint32_t idesc = instr_desc(BN, 0, 0, 128 * CG);
             const uint64_t dbase = smem_desc(0, 16, 1024);
             const int kk = p.kk;
             int sa = 0, sb = 0; uint32_t pha = 0, phb = 0;
             int ab = 0; uint32_t aph = 0;
             bool ok = true;
-            int z = blockIdx.x / (p.m_tiles * p.n_tiles * p.groups);     // only the split index matters here
-            int in_split = blockIdx.x - z * (p.m_tiles * p.n_tiles * p.groups);
+            int z = vb / (p.m_tiles * p.n_tiles * p.groups);     // only the split index matters here
+            int in_split = vb - z * (p.m_tiles * p.n_tiles * p.groups);
             const int tiles_per_split = p.m_tiles * p.n_tiles * p.groups;
-            for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x) {
+            for (int tile = vb; tile < p.tiles_total && ok; tile += vgrid) {
                 const int a_begin = z * per;
                 const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
                 if (!(ok = mbar_wait_warp(acce0 + 8u * ab, aph ^ 1u, abort_flag))) break;
+                if (CG == 2) fence_acq_rel_cluster();      // the peer's epilogue arrived from the other CTA
                 tc_fence_after();
                 const uint32_t d = tmem + (uint32_t)(ab * acc_cols + h * BN);
                 uint32_t accum = 0;
@@ -863,26 +936,26 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                         const int taps = min(p.tpg, gw - kx0);
                         const int* toff = p.tap_off + kx0;
                         if (kk == 4) {
-                            if (taps == 3) issue_row<3, 4>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
-                            else if (taps == 2) issue_row<2, 4>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
-                            else issue_row<1, 4>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            if (taps == 3) issue_row<3, 4, CG>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            else if (taps == 2) issue_row<2, 4, CG>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            else issue_row<1, 4, CG>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
                         } else {
-                            if (taps == 3) issue_row<3, 3>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
-                            else if (taps == 2) issue_row<2, 3>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
-                            else issue_row<1, 3>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            if (taps == 3) issue_row<3, 3, CG>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            else if (taps == 2) issue_row<2, 3, CG>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
+                            else issue_row<1, 3, CG>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
                         }
                         accum = 1;
-                        umma_commit(emptyB + 8u * sb);
+                        umma_commit_cg<CG>(emptyB + 8u * sb);
                         if (++sb == b_stages) { sb = 0; phb ^= 1u; }
                     }
                     if (!ok) break;
-                    umma_commit(emptyA + 8u * sa);
+                    umma_commit_cg<CG>(emptyA + 8u * sa);
                     if (++sa == a_stages) { sa = 0; pha ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit(accf0 + 8u * ab);
+                umma_commit_cg<CG>(accf0 + 8u * ab);
                 if (++ab == acc_stages) { ab = 0; aph ^= 1u; }
-                in_split += gridDim.x;
+                in_split += vgrid;
                 while (in_split >= tiles_per_split) { in_split -= tiles_per_split; ++z; }
             }
         }
@@ -891,11 +964,12 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         const int quad = warp & 3;
         const int ew = warp - (MH + 2), eset = ew >> 2, E = p.epi_sets;     // epilogue warp index and its set
         const int r = quad * 32 + lane;          // row within a 128-row half = TMEM lane
-        ConvCursor tc; tc.init(p);
+        ConvCursor tc; tc.init(p, vb, vgrid);
         int ab = 0; uint32_t aph = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < p.tiles_total && ok; tile += gridDim.x, tc.next(p)) {
-            const int m0 = tc.m_tile * (128 * MH), n0 = tc.n_tile * BN, g = tc.g;
+        const uint32_t acce_leader = CG == 2 ? mapa_u32(acce0, 0) : acce0;
+        for (int tile = vb; tile < p.tiles_total && ok; tile += vgrid, tc.next(p)) {
+            const int m0 = tc.m_tile * tile_rows + row0, n0 = tc.n_tile * BN, g = tc.g;
             const int a_begin = tc.z * per;
             const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
             if (!(ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag))) break;
@@ -928,7 +1002,8 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 }
             }
             tc_fence_before();
-            mbar_arrive(acce0 + 8u * ab);
+            if (CG == 2) mbar_arrive_cluster(acce_leader + 8u * ab);
+            else mbar_arrive(acce0 + 8u * ab);
             if (++ab == acc_stages) { ab = 0; aph ^= 1u; }
         }
         if (p.tma_store && lane == 0) bulk_wait_all();
@@ -941,9 +1016,12 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
         while (clock64() - t0 < 2000000LL) { }
         __syncthreads();
     }
+    __syncwarp();
+    if (CG == 2) cluster_sync_all();          // no CTA leaves while its peer may still arrive on its barriers
     if (warp == 2) {
         tc_fence_after();
-        tmem_dealloc(tmem, ncols);
+        if (CG == 2) tmem_dealloc_pair(tmem, ncols);
+        else tmem_dealloc(tmem, ncols);
     }
 }
 
@@ -992,6 +1070,7 @@ inline int wgrad_threads(const WgradParams& p) { return 32 * (5 + p.NI); }
 inline size_t wgrad_smem_bytes(const WgradParams& p) { return 1024 + (size_t)p.stages * (kWgABytes + kWgBBytes) + 4096 + 256; }
 
 __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant__ WgradParams p) {
+    kn::pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -1037,6 +1116,7 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    kn::pdl_wait();        // barriers, TMEM and descriptors are set up; global memory is touched from here on
 
     if (warp == 0) {
         if (lane == 0) {

@@ -25,10 +25,12 @@ def rel(a, b):
     return np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30)
 
 
-@pytest.fixture(scope="module")
-def net():
+# every operation runs three times: tile shapes from the cost model, convolutions on single CTAs only, and
+# convolutions on CTA pairs (cta_group::2) only
+@pytest.fixture(scope="module", params=[0, 16, 32], ids=["auto", "single-cta", "cta-pairs"])
+def net(request):
     from paper_1412_2302_b200.alexnet import AlexNet
-    n = AlexNet(batch=B, replicas=2, seed=SEED, mean_image=synth.mean_image(SEED))
+    n = AlexNet(batch=B, replicas=2, seed=SEED, mean_image=synth.mean_image(SEED), flags=request.param)
     yield n
     n.close()
 
