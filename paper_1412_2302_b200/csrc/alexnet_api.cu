@@ -738,26 +738,33 @@ void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
                                               g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo, g.Wpo);
     h->launches++;
 }
+// fused LRN + pool kernels, instantiated for the two LRN layers: {vectors per pixel, vectors per block, W, H, output rows
+// per block, threads} forward; {vectors per pixel, W, H, pixels per pass, threads} backward
+#define LRN_POOL_FWD_1 kn::lrn_pool_fwd_kernel<12, 6, 55, 55, 3, 352>
+#define LRN_POOL_FWD_2 kn::lrn_pool_fwd_kernel<32, 8, 27, 27, 3, 224>
+#define POOL_LRN_BWD_1 kn::pool_lrn_bwd_kernel<12, 55, 55, 28, 352>
+#define POOL_LRN_BWD_2 kn::pool_lrn_bwd_kernel<32, 27, 27, 9, 288>
 void op_lrn_pool_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
     const PoolGeo& g = kPool[which];
-    const int cpr = g.C / 8;
-    const dim3 grid((g.Ho + 1) / 2, h->B);
-    const size_t smem = (size_t)5 * g.Wi * cpr * 16;
-    launch_k(kn::lrn_pool_fwd_kernel, grid, 256, smem, st, which ? R.a2 : R.a1, which ? R.p2 : R.p1, which ? R.arg2 : R.arg1, cpr, g.Hpi,
-                                                     g.Wpi, g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta,
-                                                     h->cfg.lrn_k);
+    if (which == 0)
+        launch_k(LRN_POOL_FWD_1, dim3((g.Ho + 2) / 3, 2, h->B), 352, (size_t)7 * 55 * 6 * 16, st, R.a1, R.p1, R.arg1, g.Hpi, g.Wpi, g.Hpo,
+                 g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
+    else
+        launch_k(LRN_POOL_FWD_2, dim3((g.Ho + 2) / 3, 4, h->B), 224, (size_t)7 * 27 * 8 * 16, st, R.a2, R.p2, R.arg2, g.Hpi, g.Wpi, g.Hpo,
+                 g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
     h->launches++;
     R.n_stale[which] = true;
 }
 void op_pool_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
     const PoolGeo& g = kPool[which];
-    const int cpr = g.C / 8, ppb = 256 / cpr;
-    const dim3 grid((g.Wpi + ppb - 1) / ppb, g.Hpi, h->B);
-    launch_k(kn::pool_lrn_bwd_kernel, grid, 256, 0, st, which ? R.a2 : R.a1, which ? R.dp2 : R.dp1, which ? R.arg2 : R.arg1,
-                                                  which ? R.da2 : R.da1, cpr, ppb, g.Hpi, g.Wpi, g.Hi, g.Wi, g.Ho, g.Wo, g.Hpo,
-                                                  g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
+    if (which == 0)
+        launch_k(POOL_LRN_BWD_1, dim3((g.Hpi + 1) / 2, h->B), 352, (size_t)2 * 55 * 12 * 32, st, R.a1, R.dp1, R.arg1, R.da1, g.Hpi, g.Wpi,
+                 g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
+    else
+        launch_k(POOL_LRN_BWD_2, dim3((g.Hpi + 1) / 2, h->B), 288, (size_t)2 * 27 * 32 * 32, st, R.a2, R.dp2, R.arg2, R.da2, g.Hpi, g.Wpi,
+                 g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
     h->launches++;
     R.dn_stale[which] = true;
 }
@@ -964,7 +971,9 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     CKC(cudaFuncSetAttribute(tc::conv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::conv_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-    CKC(cudaFuncSetAttribute(kn::lrn_pool_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
+    // (static + dynamic shared memory of both exceeds the 48 KB that need no opt-in)
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 32));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 32));
     {
         int dev = 0;
         CKC(cudaGetDevice(&dev));

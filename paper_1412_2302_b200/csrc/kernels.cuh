@@ -247,110 +247,181 @@ __global__ void __launch_bounds__(256) pool_bwd_kernel(const __nv_bfloat16* __re
 }
 
 // ------------------------------------------------- LRN + pool fused (the training step)
-// Forward: p = maxpool(LRN(a)) without writing the normalised tensor.  One block = one image and two output
-// rows: the (up to five) input rows they cover are normalised once into shared memory as bf16 (the same rounding
-// as lrn_fwd_kernel's output), then pooled from there with pool_fwd_kernel's tie rule.
-// grid: (ceil(Ho/2), B); dynamic shared memory 5 * Wi * cpr * 16 bytes.
-__global__ void __launch_bounds__(256) lrn_pool_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ y,
-                                                           uint8_t* __restrict__ arg, int cpr, int Hpi, int Wpi, int Hi, int Wi,
-                                                           int Ho, int Wo, int Hpo, int Wpo, float alpha, float beta, float k) {
+// Geometry is a template parameter (the network's two LRN layers): CPR 16-byte vectors per pixel, input WI x HI.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d; asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel)); return d;
+}
+// Forward: p = maxpool(LRN(a)) without writing the normalised tensor.  One block = one image, OPR output rows and CV
+// of the CPR channel vectors: the 2*OPR+1 input rows they cover are normalised once into shared memory as bf16 (the
+// same rounding as lrn_fwd_kernel's output; channel neighbours outside the block's range come from global memory),
+// then pooled from there.  The normalised values are non-negative (a is a ReLU output; the sign bit is cleared so that
+// a -0 cannot occur), so bf16 bit patterns order like the values: each candidate becomes the 32-bit key
+// (bits << 16) | (8 - tap) and the window's maximum key carries the largest value and, among equal values, the first
+// tap in scan order - pool_fwd_kernel's tie rule.
+// grid: (ceil(HO / OPR), CPR / CV, B); dynamic shared memory (2*OPR+1) * WI * CV * 16 bytes.
+template <int CPR, int CV, int WI, int HI, int OPR, int NT>
+__global__ void __launch_bounds__(NT) lrn_pool_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ y,
+                                                          uint8_t* __restrict__ arg, int Hpi, int Wpi, int Hpo, int Wpo,
+                                                          float alpha, float beta, float k) {
     pdl_sync();
-    extern __shared__ uint4 nrm[];            // [row][x][chunk]
-    const int n = blockIdx.y, oy0 = 2 * blockIdx.x;
-    const int iy0 = 2 * oy0, nrows = min(5, Hi - iy0);
-    const int row_vecs = Wi * cpr;
-    for (int t = threadIdx.x; t < nrows * row_vecs; t += 256) {
-        const int r = t / row_vecs, q = t - r * row_vecs;
-        const int x = q / cpr, ch = q - x * cpr;
-        nrm[t] = lrn_fwd8((const uint4*)a + ((size_t)(n * Hpi + iy0 + r) * Wpi + x) * cpr + ch, ch > 0, ch < cpr - 1, alpha, beta, k);
+    constexpr int RV = WI * CV, NR = 2 * OPR + 1, WO = (WI - 3) / 2 + 1, HO = (HI - 3) / 2 + 1;
+    extern __shared__ uint4 nrm[];            // [row][x][vector]
+    const int n = blockIdx.z, c0 = blockIdx.y * CV, oy0 = OPR * blockIdx.x, iy0 = 2 * oy0;
+    const int nrows = min(NR, HI - iy0);
+    for (int q = threadIdx.x; q < RV; q += NT) {
+        const int x = q / CV, ch = c0 + q % CV;
+        const uint4* ap = (const uint4*)a + ((size_t)(n * Hpi + iy0) * Wpi + x) * CPR + ch;
+        for (int r = 0; r < nrows; ++r) {
+            uint4 v = lrn_fwd8(ap + (size_t)r * Wpi * CPR, ch > 0, ch < CPR - 1, alpha, beta, k);
+            v.x &= 0x7fff7fffu; v.y &= 0x7fff7fffu; v.z &= 0x7fff7fffu; v.w &= 0x7fff7fffu;
+            nrm[r * RV + q] = v;
+        }
     }
     __syncthreads();
-    const int out_vecs = Wo * cpr;
-    for (int t = threadIdx.x; t < 2 * out_vecs; t += 256) {
-        const int oyl = t / out_vecs, q = t - oyl * out_vecs;
-        const int oy = oy0 + oyl;
-        if (oy >= Ho) break;
-        const int ox = q / cpr, ch = q - ox * cpr;
-        float best[8]; int bi[8];
+    const int orows = min(OPR, HO - oy0);
+    for (int t = threadIdx.x; t < orows * WO * CV; t += NT) {
+        const int oyl = t / (WO * CV), q = t - oyl * (WO * CV);
+        const int ox = q / CV, cv = q - ox * CV;
+        const uint4* src = nrm + (2 * oyl * WI + 2 * ox) * CV + cv;
+        uint32_t best[8];
         #pragma unroll
         for (int ky = 0; ky < 3; ++ky)
             #pragma unroll
             for (int kx = 0; kx < 3; ++kx) {
-                float f[8];
-                unpack8(nrm[((2 * oyl + ky) * Wi + 2 * ox + kx) * cpr + ch], f);
+                const uint4 v = src[(ky * WI + kx) * CV];
+                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                const uint32_t code = 8u - (uint32_t)(ky * 3 + kx);
                 #pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if ((ky == 0 && kx == 0) || f[j] > best[j]) { best[j] = f[j]; bi[j] = ky * 3 + kx; }
+                for (int i = 0; i < 4; ++i) {
+                    const uint32_t lo = prmt(w[i], code, 0x1054u);      // (low bf16 << 16) | code
+                    const uint32_t hi = prmt(w[i], code, 0x3254u);      // (high bf16 << 16) | code
+                    if (ky == 0 && kx == 0) { best[2 * i] = lo; best[2 * i + 1] = hi; }
+                    else { best[2 * i] = max(best[2 * i], lo); best[2 * i + 1] = max(best[2 * i + 1], hi); }
+                }
             }
-        ((uint4*)y)[((size_t)(n * Hpo + oy) * Wpo + ox) * cpr + ch] = pack8(best);
-        uint2 ab;
-        ab.x = bi[0] | (bi[1] << 8) | (bi[2] << 16) | (bi[3] << 24);
-        ab.y = bi[4] | (bi[5] << 8) | (bi[6] << 16) | (bi[7] << 24);
-        ((uint2*)arg)[((size_t)(n * Ho + oy) * Wo + ox) * cpr + ch] = ab;
+        const int oy = oy0 + oyl;
+        uint4 o;
+        o.x = prmt(best[0], best[1], 0x7632u); o.y = prmt(best[2], best[3], 0x7632u);
+        o.z = prmt(best[4], best[5], 0x7632u); o.w = prmt(best[6], best[7], 0x7632u);
+        ((uint4*)y)[((size_t)(n * Hpo + oy) * Wpo + ox) * CPR + c0 + cv] = o;
+        uint2 ab;     // tap = 8 - low byte of the key
+        ab.x = 0x08080808u - prmt(prmt(best[0], best[1], 0x4040u), prmt(best[2], best[3], 0x4040u), 0x5410u);
+        ab.y = 0x08080808u - prmt(prmt(best[4], best[5], 0x4040u), prmt(best[6], best[7], 0x4040u), 0x5410u);
+        ((uint2*)arg)[((size_t)(n * HO + oy) * WO + ox) * CPR + c0 + cv] = ab;
     }
 }
-// Backward: da = LRN'(a, dn) with dn = maxpool'(dp, arg) formed on the fly (rounded to bf16 as pool_bwd_kernel
-// stores it) and passed to the channel neighbours of the same pixel through shared memory.
-// One thread = 8 channels of one pixel of the padded grid; ppb = floor(256 / cpr) pixels per block.
-// grid: (ceil(Wpi / ppb), Hpi, B).
-__global__ void __launch_bounds__(256) pool_lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ dp,
-                                                           const uint8_t* __restrict__ arg, __nv_bfloat16* __restrict__ da,
-                                                           int cpr, int ppb, int Hpi, int Wpi, int Hi, int Wi, int Ho, int Wo,
-                                                           int Hpo, int Wpo, float alpha, float beta, float k) {
+// Backward: da = LRN'(a, dn) with dn = maxpool'(dp, arg) formed in shared memory.  One block = one image and the two
+// input rows 2j, 2j+1.  The pooling windows that reach these rows lie in the window rows j-1 (its last filter row) and
+// j (its first two); windows of one row and one column parity do not overlap, so four passes (window row x parity),
+// each thread adding the eight gradients of one window vector to the fp32 pixels its argmax codes name, form dn
+// without atomics and in a fixed order.  Then one thread = 8 channels of one pixel (PPB pixels at a time): dn rounded
+// to bf16 (as pool_bwd_kernel stores it), s^-beta, tt = dn a s^(-beta-1), the tt of the two channels on either side
+// from the neighbouring threads through shared memory, and da with the ReLU mask of the convolution that produced a.
+// Pad pixels of the grid get zero.  grid: (ceil(Hpi / 2), B); dynamic shared memory 2 * WI * CPR * 32 bytes.
+template <int CPR, int WI, int HI, int PPB, int NT>
+__global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ dp,
+                                                          const uint8_t* __restrict__ arg, __nv_bfloat16* __restrict__ da,
+                                                          int Hpi, int Wpi, int Hpo, int Wpo, float alpha, float beta, float k) {
     pdl_sync();
-    __shared__ float4 edge[256];      // tt of the two lowest and two highest channels of every thread, for its neighbours
-    const int px = threadIdx.x / cpr, ch = threadIdx.x - px * cpr;
-    const int x = blockIdx.x * ppb + px, y = blockIdx.y, n = blockIdx.z;
-    const bool active = px < ppb && x < Wpi;
-    const bool valid = active && y < Hi && x < Wi;         // pad pixels of the grid: da = 0
-    const size_t t = ((size_t)(n * Hpi + y) * Wpi + x) * cpr + ch;
-    // this thread's 8 channels: dn (bf16-rounded, as pool_bwd_kernel stores it), s^-beta and tt = dn a s^(-beta-1);
-    // s needs a of channels c0-2 .. c0+9, read from the neighbouring 16-byte vectors
-    float fa[24], g8[8], sp[8], tt[8];
-    if (valid) {
-        float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        pool_bwd8(dp, arg, acc, n, y, x, ch, cpr, Ho, Wo, Hpo, Wpo);
-        unpack8(pack8(acc), g8);
-        const uint4* ap = (const uint4*)a + t;
-        const uint4 zero = make_uint4(0, 0, 0, 0);
-        unpack8(ch > 0 ? __ldg(ap - 1) : zero, fa);
-        unpack8(__ldg(ap), fa + 8);
-        unpack8(ch < cpr - 1 ? __ldg(ap + 1) : zero, fa + 16);
-        float sq[12];
-        #pragma unroll
-        for (int i = 0; i < 12; ++i) sq[i] = fa[6 + i] * fa[6 + i];
-        #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float ss = (sq[i] + sq[i + 1]) + (sq[i + 2] + sq[i + 3]) + sq[i + 4];
-            float rs;
-            pow_neg(fmaf(alpha, ss, k), beta, sp[i], rs);
-            tt[i] = g8[i] * fa[8 + i] * sp[i] * rs;
-        }
-    } else {
-        #pragma unroll
-        for (int i = 0; i < 8; ++i) tt[i] = 0.f;
+    static_assert(PPB * CPR <= NT, "one thread per vector of PPB pixels");
+    constexpr int RV = WI * CPR, WO = (WI - 3) / 2 + 1, HO = (HI - 3) / 2 + 1;
+    __shared__ float4 edge[2][NT];    // tt of the two lowest and two highest channels of every thread, for its neighbours
+    extern __shared__ float dn[];     // [2 rows][WI][CPR * 8]
+    const int j = blockIdx.x, n = blockIdx.y, y0 = 2 * j;
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    if (y0 >= HI) {                   // pad rows of the grid
+        for (int row = 0; row < 2 && y0 + row < Hpi; ++row)
+            for (int i = threadIdx.x; i < Wpi * CPR; i += NT) ((uint4*)da)[(size_t)(n * Hpi + y0 + row) * Wpi * CPR + i] = zero4;
+        return;
     }
-    edge[threadIdx.x] = make_float4(tt[0], tt[1], tt[6], tt[7]);
+    for (int i = threadIdx.x; i < 4 * RV; i += NT) ((float4*)dn)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();
-    if (!active) return;
-    if (!valid) { ((uint4*)da)[t] = make_uint4(0, 0, 0, 0); return; }
-    // tt of channels c0-2, c0-1 (left neighbour's two highest) and c0+8, c0+9 (right neighbour's two lowest)
-    float te[12];
-    const float4 l = ch > 0 ? edge[threadIdx.x - 1] : make_float4(0, 0, 0, 0);
-    const float4 r = ch < cpr - 1 ? edge[threadIdx.x + 1] : make_float4(0, 0, 0, 0);
-    te[0] = l.z; te[1] = l.w; te[10] = r.x; te[11] = r.y;
-    #pragma unroll
-    for (int i = 0; i < 8; ++i) te[2 + i] = tt[i];
-    const float c2 = 2.f * alpha * beta;
-    float o[8];
-    #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float acc = (te[i] + te[i + 1]) + (te[i + 2] + te[i + 3]) + te[i + 4];
-        const float am = fa[8 + i];
-        const float v = fmaf(g8[i], sp[i], -c2 * am * acc);
-        o[i] = am > 0.f ? v : 0.f;
+    #pragma unroll 1
+    for (int pass = 0; pass < 4; ++pass) {
+        const int oy = j - 1 + (pass >> 1), par = pass & 1;
+        if (oy >= 0 && oy < HO) {
+            for (int t = threadIdx.x; t < ((WO + 1 - par) / 2) * CPR; t += NT) {
+                const int ox = 2 * (t / CPR) + par, ch = t % CPR;
+                const uint2 ab = __ldg((const uint2*)arg + ((size_t)(n * HO + oy) * WO + ox) * CPR + ch);
+                float f[8];
+                unpack8(__ldg((const uint4*)dp + ((size_t)(n * Hpo + oy) * Wpo + ox) * CPR + ch), f);
+                float* base = dn + (2 * ox) * (CPR * 8) + ch * 8;
+                const int r0 = 2 * oy - y0;            // window row 0 relative to the block's first row: -2 or 0
+                #pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int tap = (int)(((q < 4 ? ab.x : ab.y) >> (8 * (q & 3))) & 0xFFu);
+                    const int ky = (tap * 11) >> 5, kx = tap - 3 * ky;
+                    const int row = r0 + ky;
+                    if ((unsigned)row < 2u) base[(row * WI + kx) * (CPR * 8) + q] += f[q];
+                }
+            }
+        }
+        __syncthreads();
     }
-    ((uint4*)da)[t] = pack8(o);
+    const int px = threadIdx.x / CPR, ch = threadIdx.x - px * CPR;
+    int it = 0;
+    #pragma unroll 1
+    for (int row = 0; row < 2; ++row) {
+        const int yy = y0 + row;
+        if (yy >= Hpi) break;
+        uint4* out_row = (uint4*)da + (size_t)(n * Hpi + yy) * Wpi * CPR;
+        if (yy >= HI) {
+            for (int i = threadIdx.x; i < Wpi * CPR; i += NT) out_row[i] = zero4;
+            continue;
+        }
+        for (int i = threadIdx.x; i < (Wpi - WI) * CPR; i += NT) out_row[WI * CPR + i] = zero4;     // pad columns
+        #pragma unroll 1
+        for (int p0 = 0; p0 < WI; p0 += PPB, ++it) {
+            const int x = p0 + px;
+            const bool valid = px < PPB && x < WI;
+            float fa[24], g8[8], sp[8], tt[8];
+            if (valid) {
+                const float4* gp = (const float4*)(dn + (row * WI + x) * (CPR * 8) + ch * 8);
+                const float4 g0 = gp[0], g1 = gp[1];
+                const float acc[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+                unpack8(pack8(acc), g8);
+                const uint4* ap = (const uint4*)a + ((size_t)(n * Hpi + yy) * Wpi + x) * CPR + ch;
+                unpack8(ch > 0 ? __ldg(ap - 1) : zero4, fa);
+                unpack8(__ldg(ap), fa + 8);
+                unpack8(ch < CPR - 1 ? __ldg(ap + 1) : zero4, fa + 16);
+                float sq[12];
+                #pragma unroll
+                for (int i = 0; i < 12; ++i) sq[i] = fa[6 + i] * fa[6 + i];
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float ss = (sq[i] + sq[i + 1]) + (sq[i + 2] + sq[i + 3]) + sq[i + 4];
+                    float rs;
+                    pow_neg(fmaf(alpha, ss, k), beta, sp[i], rs);
+                    tt[i] = g8[i] * fa[8 + i] * sp[i] * rs;
+                }
+            } else {
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) tt[i] = 0.f;
+            }
+            float4* eb = edge[it & 1];
+            eb[threadIdx.x] = make_float4(tt[0], tt[1], tt[6], tt[7]);
+            __syncthreads();
+            if (valid) {
+                // tt of channels c0-2, c0-1 (left neighbour's two highest) and c0+8, c0+9 (right neighbour's two lowest)
+                float te[12];
+                const float4 l = ch > 0 ? eb[threadIdx.x - 1] : make_float4(0, 0, 0, 0);
+                const float4 r = ch < CPR - 1 ? eb[threadIdx.x + 1] : make_float4(0, 0, 0, 0);
+                te[0] = l.z; te[1] = l.w; te[10] = r.x; te[11] = r.y;
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) te[2 + i] = tt[i];
+                const float c2 = 2.f * alpha * beta;
+                float o[8];
+                #pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float acc = (te[i] + te[i + 1]) + (te[i + 2] + te[i + 3]) + te[i + 4];
+                    const float am = fa[8 + i];
+                    const float v = fmaf(g8[i], sp[i], -c2 * am * acc);
+                    o[i] = am > 0.f ? v : 0.f;
+                }
+                out_row[x * CPR + ch] = pack8(o);
+            }
+        }
+    }
 }
 
 // ------------------------------------------------- split-K reductions (FC, wgrad)
