@@ -326,7 +326,8 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
     static_assert(PPB * CPR <= NT, "one thread per vector of PPB pixels");
     constexpr int RV = WI * CPR, WO = (WI - 3) / 2 + 1, HO = (HI - 3) / 2 + 1;
     __shared__ float4 edge[2][NT];    // tt of the two lowest and two highest channels of every thread, for its neighbours
-    extern __shared__ float dn[];     // [2 rows][WI][CPR * 8]
+    extern __shared__ float dn[];     // [2 planes: channels 0-3 / 4-7 of a vector][2 rows][WI][CPR] float4 (conflict-free reads)
+    constexpr int PLANE = 2 * RV * 4; // floats per plane
     const int j = blockIdx.x, n = blockIdx.y, y0 = 2 * j;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     if (y0 >= HI) {                   // pad rows of the grid
@@ -334,26 +335,37 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
             for (int i = threadIdx.x; i < Wpi * CPR; i += NT) ((uint4*)da)[(size_t)(n * Hpi + y0 + row) * Wpi * CPR + i] = zero4;
         return;
     }
+    // every thread first fetches the (up to four) window vectors it will scatter: window rows j-1 and j, even and odd
+    // columns; the loads are in flight while the tile is cleared
+    static_assert(((WO + 1) / 2) * CPR <= NT, "one thread per window vector of a pass");
+    const int wq = threadIdx.x / CPR, wch = threadIdx.x - wq * CPR;
+    uint4 wdp[4]; uint2 warg[4]; bool has[4];
+    #pragma unroll
+    for (int pass = 0; pass < 4; ++pass) {
+        const int oy = j - 1 + (pass >> 1), ox = 2 * wq + (pass & 1);
+        has[pass] = oy >= 0 && oy < HO && ox < WO;
+        if (has[pass]) {
+            warg[pass] = __ldg((const uint2*)arg + ((size_t)(n * HO + oy) * WO + ox) * CPR + wch);
+            wdp[pass] = __ldg((const uint4*)dp + ((size_t)(n * Hpo + oy) * Wpo + ox) * CPR + wch);
+        }
+    }
     for (int i = threadIdx.x; i < 4 * RV; i += NT) ((float4*)dn)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();
-    #pragma unroll 1
+    #pragma unroll
     for (int pass = 0; pass < 4; ++pass) {
         const int oy = j - 1 + (pass >> 1), par = pass & 1;
-        if (oy >= 0 && oy < HO) {
-            for (int t = threadIdx.x; t < ((WO + 1 - par) / 2) * CPR; t += NT) {
-                const int ox = 2 * (t / CPR) + par, ch = t % CPR;
-                const uint2 ab = __ldg((const uint2*)arg + ((size_t)(n * HO + oy) * WO + ox) * CPR + ch);
-                float f[8];
-                unpack8(__ldg((const uint4*)dp + ((size_t)(n * Hpo + oy) * Wpo + ox) * CPR + ch), f);
-                float* base = dn + (2 * ox) * (CPR * 8) + ch * 8;
-                const int r0 = 2 * oy - y0;            // window row 0 relative to the block's first row: -2 or 0
-                #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const int tap = (int)(((q < 4 ? ab.x : ab.y) >> (8 * (q & 3))) & 0xFFu);
-                    const int ky = (tap * 11) >> 5, kx = tap - 3 * ky;
-                    const int row = r0 + ky;
-                    if ((unsigned)row < 2u) base[(row * WI + kx) * (CPR * 8) + q] += f[q];
-                }
+        if (has[pass]) {
+            const int ox = 2 * wq + par;
+            float f[8];
+            unpack8(wdp[pass], f);
+            float* base = dn + ((2 * ox) * CPR + wch) * 4;
+            const int r0 = 2 * oy - y0;            // window row 0 relative to the block's first row: -2 or 0
+            #pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int tap = (int)(((q < 4 ? warg[pass].x : warg[pass].y) >> (8 * (q & 3))) & 0xFFu);
+                const int ky = (tap * 11) >> 5, kx = tap - 3 * ky;
+                const int row = r0 + ky;
+                if ((unsigned)row < 2u) base[(q >> 2) * PLANE + (row * WI + kx) * (CPR * 4) + (q & 3)] += f[q];
             }
         }
         __syncthreads();
@@ -376,8 +388,8 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
             const bool valid = px < PPB && x < WI;
             float fa[24], g8[8], sp[8], tt[8];
             if (valid) {
-                const float4* gp = (const float4*)(dn + (row * WI + x) * (CPR * 8) + ch * 8);
-                const float4 g0 = gp[0], g1 = gp[1];
+                const float4* gp = (const float4*)dn + (row * WI + x) * CPR + ch;
+                const float4 g0 = gp[0], g1 = gp[PLANE / 4];
                 const float acc[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
                 unpack8(pack8(acc), g8);
                 const uint4* ap = (const uint4*)a + ((size_t)(n * Hpi + yy) * Wpi + x) * CPR + ch;
