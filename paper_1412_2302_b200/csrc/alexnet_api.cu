@@ -326,7 +326,10 @@ ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, in
     const int a_rows = kw > 1 ? 136 : 128;
     const size_t budget = 227 * 1024 - 2048 - 4 * tc::kEpiStageBytes;
     const int cg_lo = (h->cfg.flags & ALEXNET_FLAG_ALL_CTA_PAIRS) ? 2 : 1, cg_hi = (h->cfg.flags & ALEXNET_FLAG_NO_CTA_PAIRS) ? 1 : 2;
-    for (int cg = cg_lo; cg <= cg_hi; ++cg)
+    // a reduction of fewer than four (filter row, chunk) steps per tile (conv1) cannot amortise the accumulator hand-over
+    // across the pair: measured slower in pairs (55 -> 61 us), so such layers stay on single CTAs unless forced
+    const int cg_auto_hi = kh * chunks >= 4 ? 2 : 1;
+    for (int cg = cg_lo; cg <= (cg_lo == 2 ? 2 : std::min(cg_hi, cg_auto_hi)); ++cg)
     for (int MH = 1; MH <= 4; MH *= 2) {
         for (int BN = 16; BN <= 256 && BN <= N; BN += 16) {
             if (N % BN) continue;
