@@ -146,6 +146,8 @@ struct alexnet {
     Layout L;
     int B;
     cudaStream_t cs, ls;   // compute, loader
+    cudaStream_t gs = nullptr;             // second compute stream of the backward pass: conv weight gradients (owned)
+    cudaEvent_t ev_dy[5] = {}, ev_gs_done = nullptr;   // dy of conv layer l is ready on cs; gs has finished its weight gradients
     uint8_t* arena; size_t arena_bytes;
     Replica rep[2];
     float* mean; float* ws; float* cs_partial; float* canon_tmp; int* status;
@@ -823,13 +825,29 @@ void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
         else { op_fc_wg(h, r, l, l == 2, st); op_fc_bwd(h, r, l, st); }
     }
     op_pool_bwd(h, r, 2, st);
-    op_conv_wg(h, r, 4, slot, st); op_conv_bwd(h, r, 4, st);
-    op_conv_wg(h, r, 3, slot, st); op_conv_bwd(h, r, 3, st);
-    op_conv_wg(h, r, 2, slot, st); op_conv_bwd(h, r, 2, st);
+    // The weight gradient of a conv layer and the data gradient that continues the chain both need only the layer's dy.
+    // The chain stays on `st`; the weight gradients (kernel, then split reduction) run on a second stream as soon as
+    // their dy exists, so that their blocks fill the SMs that the chain's kernels leave idle in their last waves.
+    // Nothing on `st` touches the split workspace or the conv gradients meanwhile; `st` joins before it returns.
+    // Per-kernel profiling keeps everything on one stream.
+    const bool two = h->gs != nullptr && !h->prof;
+    cudaStream_t g = two ? h->gs : st;
+    auto dy_ready = [&](int l) {
+        if (!two) return;
+        cudaEventRecord(h->ev_dy[l], st);
+        cudaStreamWaitEvent(h->gs, h->ev_dy[l], 0);
+    };
+    dy_ready(4); op_conv_wg(h, r, 4, slot, g); op_conv_bwd(h, r, 4, st);
+    dy_ready(3); op_conv_wg(h, r, 3, slot, g); op_conv_bwd(h, r, 3, st);
+    dy_ready(2); op_conv_wg(h, r, 2, slot, g); op_conv_bwd(h, r, 2, st);
     op_pool_lrn_bwd(h, r, 1, st);
-    op_conv_wg(h, r, 1, slot, st); op_conv_bwd(h, r, 1, st);
+    dy_ready(1); op_conv_wg(h, r, 1, slot, g); op_conv_bwd(h, r, 1, st);
     op_pool_lrn_bwd(h, r, 0, st);
-    op_conv_wg(h, r, 0, slot, st);
+    dy_ready(0); op_conv_wg(h, r, 0, slot, g);
+    if (two) {
+        cudaEventRecord(h->ev_gs_done, h->gs);
+        cudaStreamWaitEvent(st, h->ev_gs_done, 0);
+    }
 }
 
 int check_status(alexnet* h) {
@@ -982,6 +1000,9 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
         CKC(cudaGetDevice(&dev));
         CKC(cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev));
     }
+    CKC(cudaStreamCreateWithFlags(&h->gs, cudaStreamNonBlocking));
+    for (int l = 0; l < 5; ++l) CKC(cudaEventCreateWithFlags(&h->ev_dy[l], cudaEventDisableTiming));
+    CKC(cudaEventCreateWithFlags(&h->ev_gs_done, cudaEventDisableTiming));
     // pad positions of every grid must be zero from the start; gradients and momentum start at zero
     CKC(cudaMemsetAsync(h->arena, 0, need, h->cs));
     if (host_mean_image) CKC(cudaMemcpyAsync(h->mean, host_mean_image, 256 * 256 * 3 * sizeof(float), cudaMemcpyHostToDevice, h->cs));
@@ -1012,6 +1033,9 @@ int alexnet_destroy(alexnet_t* h) {
     if (!h) return ALEXNET_ERR_ARG;
     cudaStreamSynchronize(h->cs);
     cudaStreamSynchronize(h->ls);
+    if (h->gs) { cudaStreamSynchronize(h->gs); cudaStreamDestroy(h->gs); }
+    for (int l = 0; l < 5; ++l) if (h->ev_dy[l]) cudaEventDestroy(h->ev_dy[l]);
+    if (h->ev_gs_done) cudaEventDestroy(h->ev_gs_done);
     for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
     for (int r = 0; r < h->cfg.replicas; ++r)
         for (int s = 0; s < 2; ++s) { cudaEventDestroy(h->rep[r].ready[s]); cudaEventDestroy(h->rep[r].consumed[s]); }
