@@ -311,7 +311,7 @@ void finish_plan(const alexnet* h, Plan& P) {
     p.splits = (p.steps_total + per - 1) / per;
     p.steps_per_split = per;
     p.tiles_total = p.m_tiles * p.n_tiles * p.groups * p.taps_grid * p.splits;
-    if (p.fuse_update) p.stages = stages = 2;      // the reduction is two k-steps long; the epilogue tiles need the room
+    if (p.fuse_update) p.stages = stages = 1;      // two k-steps per tile, hidden behind the epilogue of the tile before; the epilogue tiles need the room
     P.smem = tc::smem_bytes(p.mode, p.BN, stages, p.fuse_update != 0);
     P.grid = std::min(p.tiles_total, h->sm_count);   // persistent: one CTA per SM walks the tile list
     P.valid = true;

@@ -388,10 +388,10 @@ __host__ __device__ inline int b_stage_bytes(int mode, int BN) {
     return mode == MODE_KK ? BN * 128 : ((BN + 63) / 64) * 8192;
 }
 // per epilogue warp of a fused-update kernel: kUpdBufs {w tile, v tile} pairs of 4 KB each and two 2 KB bf16 tiles
-constexpr int kUpdBufs = 4;
+constexpr int kUpdBufs = 5;
 constexpr uint32_t kUpdWarpBytes = kUpdBufs * 8192 + 2 * 2048;
 inline size_t smem_bytes(int mode, int BN, int stages, bool fuse_update = false) {
-    return 1024 + (size_t)stages * (kABytes + b_stage_bytes(mode, BN)) + 4 * kEpiStageBytes + (fuse_update ? 4 * kUpdWarpBytes : 0) + 512;
+    return 1024 + (size_t)stages * (kABytes + b_stage_bytes(mode, BN)) + (fuse_update ? 4 * kUpdWarpBytes : 4 * kEpiStageBytes) + 512;
 }
 
 // position of a CTA in the tile list; tiles are numbered with m fastest, then
@@ -431,8 +431,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     // epilogue staging (4 warps x kEpiStageBytes), then barriers: full[8] @0, empty[8] @64, acc_full[2] @128,
     // acc_empty[2] @144, tmem slot @160, abort flag @168
     const uint32_t epi_stage0 = base + stages * stage_bytes;
-    const uint32_t upd0 = epi_stage0 + 4u * kEpiStageBytes;                     // fused update: per-warp tiles
-    const uint32_t bar_base = upd0 + (p.fuse_update ? 4u * kUpdWarpBytes : 0u);  // ... + per-warp load barriers [4][3] @176
+    const uint32_t upd0 = epi_stage0 + (p.fuse_update ? 0u : 4u * kEpiStageBytes);   // fused update: per-warp tiles instead of the staging
+    const uint32_t bar_base = upd0 + (p.fuse_update ? 4u * kUpdWarpBytes : 0u);  // ... + per-warp load barriers [4][kUpdBufs] @176
     uint8_t* gen = smem_raw + (bar_base - raw);
     volatile int* abort_flag = (volatile int*)(gen + 168);
     volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 160);
@@ -553,8 +553,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         bool ok = true;
         if (p.fuse_update) {
             // FC weight gradient consumed in place: for every 32 x 32 slab of the tile this warp loads the weights and the
-            // momentum by TMA (two slabs ahead of the arithmetic), applies v <- mu v - d w - lr g, w <- w + v to the
-            // accumulator values and stores w, v and the bf16 copy of w by TMA.  A buffer (of kUpdBufs = 4) is reloaded
+            // momentum by TMA (kUpdBufs - 2 = three slabs ahead of the arithmetic), applies v <- mu v - d w - lr g, w <- w + v to the
+            // accumulator values and stores w, v and the bf16 copy of w by TMA.  A buffer (of kUpdBufs = 5) is reloaded
             // only after the stores issued from it two slabs earlier have finished reading (wait_group.read 1).
             const uint32_t ureg = upd0 + (uint32_t)quad * kUpdWarpBytes, ub0 = bar_base + 176u + (uint32_t)quad * (8u * kUpdBufs);
             TileCursor tp = tc;                      // prefetch cursor
@@ -570,8 +570,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 if (pc == p.BN) { pc = 0; ptile += gridDim.x; tp.next(p); }
             };
             if (lane == 0) {
-                if (ptile < p.tiles_total) issue_loads();
-                if (ptile < p.tiles_total) issue_loads();
+                #pragma unroll 1
+                for (int i = 0; i < kUpdBufs - 2 && ptile < p.tiles_total; ++i) issue_loads();
             }
             __syncwarp();
             while (tile < p.tiles_total) {
