@@ -322,7 +322,7 @@ void finish_plan(const alexnet* h, Plan& P) {
 // modelled time.  Per weight stage the tensor pipe needs MH*kk*BN/2 cycles; TMA brings about 64 bytes
 // per cycle per SM from L2; tiles are dealt to the SMs in rounds.
 struct ConvShape { int MH, BN, acc_stages, epi_sets, cg; };
-ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, int kh, int kw, int chunks, int kk) {
+ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, int kh, int kw, int chunks, int kk, bool masked = false) {
     ConvShape best{1, N <= 256 ? N : 128, 1, 1, 1};
     double best_t = 1e30;
     const int a_rows = kw > 1 ? 136 : 128;
@@ -358,9 +358,12 @@ ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, in
             // epilogue per 16 columns and row half: about 450 cycles through the staged TMA store (single staging tile per warp), about 1000 with direct
             // stores (tiles whose 64-column slabs would not fit the group's channel range)
             const bool staged = BN % 64 == 0 || (groups == 1 && N == BN);
-            const double epi = MH * (BN / 16) * (staged ? 450.0 : 1000.0);
-            // a second set of epilogue warps (each takes every other row half) when the epilogue is the longer side
-            for (int E = 1; E <= (MH >= 2 && staged ? 2 : 1); ++E) {
+            // (a ReLU mask read from global memory in the epilogue adds its load latency: measured, the issuer of a masked
+            // backward-data layer waits a quarter of its time for a free accumulator)
+            const double epi = MH * (BN / 16) * (staged ? (masked ? 1000.0 : 450.0) : 1000.0);
+            // a second set of epilogue warps (the sets alternate over the tile's row halves x 64-column slabs) when the
+            // epilogue is the longer side
+            for (int E = 1; E <= (staged && MH * ((BN + 63) / 64) >= 2 ? 2 : 1); ++E) {
                 if (E == 2 && 2 * (size_t)MH * a_rows * 128 + 2 * g_tiles * (BN / cg) * 128 + 4 * tc::kEpiStageBytes > budget) continue;
                 double tt = tile_t;
                 if (acc == 1) tt += epi / E; else tt = std::max(tt, epi / E + 300.0);
@@ -445,7 +448,7 @@ int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf1
     const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
     const int gp = c.gin.Wp;
     p.kh = p.kw = c.k; p.chunks = c.cog / 64; p.kk = 4;
-    const ConvShape sh = choose_conv_shape(h, M, c.cig, c.groups, p.kh, p.kw, p.chunks, p.kk);
+    const ConvShape sh = choose_conv_shape(h, M, c.cig, c.groups, p.kh, p.kw, p.chunks, p.kk, mask != nullptr);
     p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages; p.epi_sets = sh.epi_sets; p.cg = sh.cg;
     p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH * p.cg - 1) / (128 * p.MH * p.cg));
     p.n_tiles = c.cig / p.BN; p.groups = c.groups; p.splits = 1;

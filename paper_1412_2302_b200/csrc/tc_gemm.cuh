@@ -717,7 +717,7 @@ struct ConvParams {
     int chunks;         // 64-channel chunks
     int asteps_total;   // kh * chunks, split evenly over `splits`
     int asteps_per_split;
-    int epi_sets;       // 1 or 2 sets of four epilogue warps; with two, set e handles the row halves h with h % 2 == e
+    int epi_sets;       // 1 or 2 sets of four epilogue warps; with two, the (row half, column slab) units of a tile alternate between them
     int a_stages, b_stages, acc_stages;   // b_stages counts groups of kw weight tiles (one barrier pair per group)
     int a_box_rows;     // rows per activation box (128, or 136 when kw > 1)
     int a_x0, a_gx;     // A column origin and per-group column stride
@@ -974,8 +974,10 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
             const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
             if (!(ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag))) break;
             tc_fence_after();
+            // with two sets of epilogue warps, the (row half, slab) units of the tile alternate between the sets
+            int unit = 0;
             #pragma unroll 1
-            for (int h = eset; h < MH; h += E) {
+            for (int h = 0; h < MH; ++h) {
                 const int row = m0 + h * 128 + r;
                 const bool row_ok = row < p.M_total;
                 bool pad_row = false;
@@ -987,12 +989,14 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 const uint32_t t0 = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * acc_cols + h * BN);
                 if (p.tma_store) {
                     const int slab = p.epi == EPI_F32 ? 32 : 64;
-                    for (int c = 0; c < BN; c += slab) {
+                    for (int c = 0; c < BN; c += slab, ++unit) {
+                        if (E == 2 && (unit & 1) != eset) continue;
                         epi_slab(p, t0 + (uint32_t)c, pad_row, row_off, n0 + c, g, g * p.out_gx + n0 + c, m0 + h * 128 + quad * 32,
                                  tc.z, epi_stage0 + (uint32_t)ew * kEpiStageBytes, lane);
                     }
                 } else {
-                    for (int c = 0; c < BN; c += 16) {
+                    for (int c = 0; c < BN; c += 16, ++unit) {
+                        if (E == 2 && (unit & 1) != eset) continue;
                         uint32_t v[16];
                         tmem_ld16(t0 + (uint32_t)c, v);
                         tmem_ld_wait();
