@@ -154,6 +154,8 @@ enum {
     ALEXNET_T_DZ, ALEXNET_T_DF7, ALEXNET_T_DF6, ALEXNET_T_DP5, ALEXNET_T_DA5, ALEXNET_T_DA4, ALEXNET_T_DA3,
     ALEXNET_T_DP2, ALEXNET_T_DN2, ALEXNET_T_DA2, ALEXNET_T_DP1, ALEXNET_T_DN1, ALEXNET_T_DA1,
     ALEXNET_T_LOSS, /* [B] per-sample loss */
+    ALEXNET_T_DX0,  /* gradient with respect to the preprocessed image, [B][3][227][227]: written only by
+                     * ALEXNET_OP_CONV1_BWD_DATA (the training step never needs it) */
     ALEXNET_T_COUNT
 };
 size_t alexnet_tensor_size(const alexnet_t* h, int tensor_id);
@@ -177,6 +179,7 @@ enum {
     ALEXNET_OP_POOL1_FWD, ALEXNET_OP_POOL2_FWD, ALEXNET_OP_POOL5_FWD,
     ALEXNET_OP_POOL1_BWD, ALEXNET_OP_POOL2_BWD, ALEXNET_OP_POOL5_BWD,
     ALEXNET_OP_SOFTMAX, ALEXNET_OP_UPDATE, ALEXNET_OP_AVERAGE, ALEXNET_OP_PREPROCESS,
+    ALEXNET_OP_CONV1_BWD_DATA,   /* DA1 -> DX0; not part of the training step (per-layer sweep only) */
     ALEXNET_OP_COUNT
 };
 int alexnet_run_op(alexnet_t* h, int replica, int op, int iters);

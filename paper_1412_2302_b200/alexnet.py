@@ -19,7 +19,7 @@ FLAG_NO_CTA_PAIRS, FLAG_ALL_CTA_PAIRS = 16, 32
 
 TENSORS = ["CROPFLIP", "X0", "A1", "N1", "P1", "ARG1", "A2", "N2", "P2", "ARG2", "A3", "A4", "A5", "P5", "ARG5",
            "F6", "F7", "Z", "M6", "M7", "DZ", "DF7", "DF6", "DP5", "DA5", "DA4", "DA3", "DP2", "DN2", "DA2",
-           "DP1", "DN1", "DA1", "LOSS"]
+           "DP1", "DN1", "DA1", "LOSS", "DX0"]
 T = {n: i for i, n in enumerate(TENSORS)}
 OPS = ["CONV1_FWD", "CONV2_FWD", "CONV3_FWD", "CONV4_FWD", "CONV5_FWD",
        "CONV2_BWD_DATA", "CONV3_BWD_DATA", "CONV4_BWD_DATA", "CONV5_BWD_DATA",
@@ -27,7 +27,7 @@ OPS = ["CONV1_FWD", "CONV2_FWD", "CONV3_FWD", "CONV4_FWD", "CONV5_FWD",
        "FC6_FWD", "FC7_FWD", "FC8_FWD", "FC6_BWD_DATA", "FC7_BWD_DATA", "FC8_BWD_DATA",
        "FC6_BWD_WEIGHT", "FC7_BWD_WEIGHT", "FC8_BWD_WEIGHT",
        "LRN1_FWD", "LRN2_FWD", "LRN1_BWD", "LRN2_BWD", "POOL1_FWD", "POOL2_FWD", "POOL5_FWD",
-       "POOL1_BWD", "POOL2_BWD", "POOL5_BWD", "SOFTMAX", "UPDATE", "AVERAGE", "PREPROCESS"]
+       "POOL1_BWD", "POOL2_BWD", "POOL5_BWD", "SOFTMAX", "UPDATE", "AVERAGE", "PREPROCESS", "CONV1_BWD_DATA"]
 OP = {n: i for i, n in enumerate(OPS)}
 
 EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "alexnet_destroy",

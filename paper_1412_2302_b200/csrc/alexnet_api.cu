@@ -75,7 +75,7 @@ Layout make_layout() {
         c.w_off = off; off = align_up(off + (long long)c.taps * c.cout * c.cig, 64);
         c.canon_w = canon; canon += canon_wcount[l];
         c.canon_b = canon; canon += c.cout;
-        if (l > 0) { c.wt_off = wt; wt = align_up(wt + (long long)c.taps * c.cin * c.cog, 64); }
+        c.wt_off = wt; wt = align_up(wt + (long long)c.taps * c.cin * c.cog, 64);
     }
     const int fcs[3][2] = {{9216, 4096}, {4096, 4096}, {4096, 1000}};
     for (int l = 0; l < 3; ++l) {
@@ -103,10 +103,10 @@ Layout make_layout() {
         L.segs.s[s++] = kn::ParamSeg{f.canon_w, f.w_off, (long long)f.K * f.N, l == 0 ? 3 : 0, 0, 0, 0};
         L.segs.s[s++] = kn::ParamSeg{f.canon_b, f.b_off, f.N, 0, 0, 0, 0};
     }
-    L.tjobs.n = 4;
-    for (int l = 1; l < 5; ++l) {
+    L.tjobs.n = 5;
+    for (int l = 0; l < 5; ++l) {
         const ConvL& c = L.conv[l];
-        L.tjobs.j[l - 1] = kn::TransposeJob{c.w_off, c.wt_off, c.taps, c.cout, c.cig, c.groups, (long long)c.taps * c.cin * c.cog};
+        L.tjobs.j[l] = kn::TransposeJob{c.w_off, c.wt_off, c.taps, c.cout, c.cig, c.groups, (long long)c.taps * c.cin * c.cog};
     }
     return L;
 }
@@ -126,7 +126,7 @@ struct Replica {
     bf16 *a1, *n1, *p1, *a2, *n2, *p2, *a3, *a4, *a5, *p5, *f6, *f7;
     float* z;
     uint8_t *arg1, *arg2, *arg5, *m6, *m7;
-    bf16 *dz, *df7, *df6, *dp5, *da5, *da4, *da3, *dp2, *dn2, *da2, *dp1, *dn1, *da1;
+    bf16 *dz, *df7, *df6, *dp5, *da5, *da4, *da3, *dp2, *dn2, *da2, *dp1, *dn1, *da1, *dx0;
     float *loss_n, *loss;
     // batch slots
     cudaEvent_t ready[2], consumed[2];
@@ -256,6 +256,7 @@ size_t carve(alexnet* h, uint8_t* base) {
         R.da5 = c.take<bf16>(r3 * 256); R.da4 = c.take<bf16>(r3 * 384); R.da3 = c.take<bf16>(r3 * 384);
         R.dp2 = c.take<bf16>(r3 * 256); R.dn2 = c.take<bf16>(r2 * 256); R.da2 = c.take<bf16>(r2 * 256);
         R.dp1 = c.take<bf16>(r2 * 96); R.dn1 = c.take<bf16>(r1 * 96); R.da1 = c.take<bf16>(r1 * 96);
+        R.dx0 = c.take<bf16>(rows(L.conv[0].gin) * 48);
         R.loss_n = c.take<float>(B); R.loss = c.take<float>(16);
     }
     return (c.off + 1023) / 1024 * 1024;
@@ -447,7 +448,7 @@ int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf1
     tc::ConvParams& p = P.c;
     const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
     const int gp = c.gin.Wp;
-    p.kh = p.kw = c.k; p.chunks = c.cog / 64; p.kk = 4;
+    p.kh = p.kw = c.k; p.chunks = (c.cog + 63) / 64; p.kk = 4;      // conv1: 96 channels, the second chunk is half zero fill
     const ConvShape sh = choose_conv_shape(h, M, c.cig, c.groups, p.kh, p.kw, p.chunks, p.kk, mask != nullptr);
     p.MH = sh.MH; p.BN = sh.BN; p.acc_stages = sh.acc_stages; p.epi_sets = sh.epi_sets; p.cg = sh.cg;
     p.M_total = (int)M; p.m_tiles = (int)((M + 128 * p.MH * p.cg - 1) / (128 * p.MH * p.cg));
@@ -570,7 +571,7 @@ int build_plans(alexnet* h, int r) {
     const bf16* in[5] = {nullptr, R.p1, R.p2, R.a3, R.a4};
     bf16* out[5] = {R.a1, R.a2, R.a3, R.a4, R.a5};
     bf16* dyv[5] = {R.da1, R.da2, R.da3, R.da4, R.da5};
-    bf16* dxv[5] = {nullptr, R.dp1, R.dp2, R.da3, R.da4};
+    bf16* dxv[5] = {R.dx0, R.dp1, R.dp2, R.da3, R.da4};
     const bf16* maskv[5] = {nullptr, nullptr, nullptr, R.a3, R.a4};
     int rc;
     for (int l = 0; l < 5; ++l) {
@@ -580,7 +581,7 @@ int build_plans(alexnet* h, int r) {
             if ((rc = plan_conv_fwd(h, R.conv_fwd[l][s], c, x, R.shadow + c.w_off, R.w + c.b_off, out[l]))) return rc;
             if ((rc = plan_conv_wg(h, R.conv_wg[l][s], c, dyv[l], x))) return rc;
         }
-        if (l > 0 && (rc = plan_conv_bwd(h, R.conv_bwd[l], c, dyv[l], R.wt + c.wt_off, maskv[l], dxv[l]))) return rc;
+        if ((rc = plan_conv_bwd(h, R.conv_bwd[l], c, dyv[l], R.wt + c.wt_off, maskv[l], dxv[l]))) return rc;
     }
     const bf16* fx[3] = {R.p5, R.f6, R.f7};
     const bf16* fdy[3] = {R.df6, R.df7, R.dz};
@@ -926,6 +927,7 @@ bool tensor_desc(alexnet* h, int r, int id, Tensor* T) {
         case ALEXNET_T_DN1: grid(R.dn1, g1, 96); return true;
         case ALEXNET_T_DA1: grid(R.da1, g1, 96); return true;
         case ALEXNET_T_LOSS: *T = Tensor{R.loss_n, 7, 0, 0, 0, 0, 0, 1}; return true;
+        case ALEXNET_T_DX0: *T = Tensor{R.dx0, 5, 3, 57, 57, 227, 227, 0}; return true;
     }
     return false;
 }
@@ -1267,6 +1269,7 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
         else if (op == ALEXNET_OP_UPDATE) op_update(h, replica, st, true);
         else if (op == ALEXNET_OP_AVERAGE) op_average(h, st);
         else if (op == ALEXNET_OP_PREPROCESS) op_preprocess(h, replica, slot, R.slot_step[slot], st);
+        else if (op == ALEXNET_OP_CONV1_BWD_DATA) op_conv_bwd(h, replica, 0, st);
     }
     CK(cudaGetLastError());
     return ALEXNET_OK;

@@ -639,7 +639,7 @@ __global__ void topk_count_kernel(const float* __restrict__ z, const int32_t* __
 // transposed bf16 copies of the grouped conv filters for the backward-data pass:
 // wt[tap][g*cig + ci][co'] = wf[tap][g*cog + co'][ci]
 struct TransposeJob { long long src_off, dst_off; int taps, cout, cig, groups; long long count; };
-struct TransposeJobs { TransposeJob j[4]; int n; };
+struct TransposeJobs { TransposeJob j[5]; int n; };
 // one parameter of the momentum update: v <- mu v - d w - lr g (d = lr * weight decay, or 0); w <- w + v.
 // Used by the update kernel and by the FC weight-gradient epilogue that applies the update in place, so that both
 // give bit-identical results.

@@ -63,14 +63,17 @@ def test_conv_forward(net, params, name, tin, tout, shp):
     assert (got >= 0).all()
 
 
-BWD = [("conv2", "DA2", "DP1", None, (96, 27, 27)), ("conv3", "DA3", "DP2", None, (256, 13, 13)),
+# conv1's data gradient (the gradient with respect to the image) is not part of the training step; the per-layer sweep
+# runs it, in the space-to-depth layout of conv1's input
+BWD = [("conv1", "DA1", "DX0", None, (3, 227, 227)), ("conv2", "DA2", "DP1", None, (96, 27, 27)), ("conv3", "DA3", "DP2", None, (256, 13, 13)),
        ("conv4", "DA4", "DA3", "A3", (384, 13, 13)), ("conv5", "DA5", "DA4", "A4", (384, 13, 13))]
 
 
 @pytest.mark.parametrize("name,tdy,tdx,tmask,shp", BWD)
 def test_conv_backward_data(net, params, name, tdy, tdx, tmask, shp):
     c = O.CONV[name]
-    dy = synth.bf16_grid(SEED, 7 + tag(name), (B, c["cout"], shp[1], shp[2]), -1, 1)
+    ho = 55 if name == "conv1" else shp[1]
+    dy = synth.bf16_grid(SEED, 7 + tag(name), (B, c["cout"], ho, ho), -1, 1)
     net.set_tensor(tdy, dy)
     ref = O.conv_bwd_data(dy, params[name + ".W"], (B,) + shp, c["s"], c["p"], c["g"])
     if tmask:
