@@ -365,6 +365,7 @@ ConvShape choose_conv_shape(const alexnet* h, long long M, int N, int groups, in
             // a second set of epilogue warps (the sets alternate over the tile's row halves x 64-column slabs) when the
             // epilogue is the longer side
             for (int E = 1; E <= (staged && MH * ((BN + 63) / 64) >= 2 ? 2 : 1); ++E) {
+                if (32 * (2 + MH + 4 * E) > tc::kConvMaxThreads) continue;     // warps: 2 producers, MH issuers, 4 E epilogue
                 if (E == 2 && 2 * (size_t)MH * a_rows * 128 + 2 * g_tiles * (BN / cg) * 128 + 4 * tc::kEpiStageBytes > budget) continue;
                 double tt = tile_t;
                 if (acc == 1) tt += epi / E; else tt = std::max(tt, epi / E + 300.0);

@@ -2,7 +2,7 @@
 """Per-layer roofline sweep: every operation of the training step timed on its
 own through the C ABI (alexnet_run_op), at AlexNet shapes.
 
-    python -m paper_1412_2302_b200.layer_sweep [--batch 256] [--iters 20] [--json out.json]
+    python -m paper_1412_2302_b200.layer_sweep [--batch 256] [--iters 20] [--burst 1] [--json out.json]
 
 Tensor-core operations (convolution and FC forward, backward-data,
 backward-weight) are reported in TFLOP/s of algorithmic work (2 x MACs of the
@@ -11,7 +11,9 @@ bf16 peak; the other operations in GB/s of algorithmic bytes against the
 measured HBM copy bandwidth.  Each timed run is preceded by a write of a buffer
 larger than L2, so no operand is L2-resident from the run before; tensors hold
 the values of a real training step.  An operation's time covers all the kernels
-it launches (e.g. the split-K reduction after a weight-gradient GEMM).
+it launches (e.g. the split-K reduction after a weight-gradient GEMM).  With --burst N > 1 a timed run is N
+back-to-back launches of the operation and the time is divided by N: the launches overlap their set-up and tails as
+the kernels of a training step do (programmatic dependent launch), and operands stay in L2 from the launch before.
 """
 from __future__ import annotations
 
@@ -57,6 +59,7 @@ def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--batch", type=int, default=256)
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--burst", type=int, default=1)
     ap.add_argument("--json", default=None)
     ap.add_argument("--ops", default=None, help="comma-separated subset of operation names")
     args = ap.parse_args(argv)
@@ -92,11 +95,11 @@ def main(argv=None):
                 flush.fill_(1)
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(cs)
-                net.run_op(name)
+                net.run_op(name, iters=args.burst)
                 e1.record(cs)
                 ts.append((e0, e1))
             net.sync()
-            ms = float(np.median([a.elapsed_time(b) for a, b in ts]))
+            ms = float(np.median([a.elapsed_time(b) for a, b in ts])) / args.burst
             layer = name.split("_")[0]
             if layer in MACS:
                 tf = 2.0 * MACS[layer] * B / (ms * 1e-3) / 1e12
@@ -117,7 +120,8 @@ def main(argv=None):
             net.eval_batch(0, dimg, dlab)
         eval_ms = (time.perf_counter() - t0) * 1e3 / args.iters
     net.close()
-    print(f"# batch {B}, median of {args.iters} runs, L2 flushed before each; peaks ({kind}): "
+    print(f"# batch {B}, median of {args.iters} runs" + (f" of {args.burst} back-to-back launches" if args.burst > 1 else "")
+          + f", L2 flushed before each; peaks ({kind}): "
           f"{tf_peak:.0f} TFLOP/s bf16 burst, {hbm_peak:.0f} GB/s HBM")
     print(f"{'operation':<20}{'ms':>9}{'TFLOP/s':>10}{'GB/s':>9}{'of peak':>9}")
     for r in rows:
