@@ -33,6 +33,9 @@ FLOP_PER_IMAGE = 4.1356e9          # 3 x 1.4488 GFLOP forward-equivalents minus 
 # algorithmic FLOP per image of the three tensor-core kernels (2 x MACs of the dense layers, no padding counted):
 # conv_kernel = conv forward (5 layers) + conv backward-data (conv2-5) + FC forward; wgrad_kernel = conv
 # weight gradients; gemm_kernel = FC backward-data + FC weight gradients
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over each kernel's launches of one batch-128 training
+# step (one ncu capture of this build's kernels; the summary is kept with the other profiles)
+NCU_DRAM_BYTES_PER_LAUNCH = {"conv_kernel": 34.7e6, "wgrad_kernel": 59.9e6, "gemm_kernel": 170.5e6}
 KERNELS = ("conv_kernel", "wgrad_kernel", "gemm_kernel")
 KERNEL_FLOP = (1.3315e9 + 1.1207e9 + 0.1173e9, 1.3315e9, 0.2346e9)
 N_POOL = 4                          # distinct synthetic batches cycled through
@@ -231,7 +234,7 @@ def run_ours(args, rank, world, local_rank):
             "config": {"workload": "full AlexNet train step, batch 128 per GPU, fresh uint8 256x256x3 batch per step loaded "
                                    "and preprocessed on a side stream overlapped with the previous step (config 3)",
                        "global_batch": BATCH * world, "precision": "bf16 operands, fp32 accumulate, fp32 master weights",
-                       "l2": "each step streams >1.3 GB of parameters/momentum/gradients, far above the 126 MB L2",
+                       "l2": "each step streams >1 GB of parameters, momentum and bf16 copies, far above the 126 MB L2",
                        "parallelism": "independent replicas per GPU" if world > 1 else "single GPU"},
             "e2e": {"value": imgs / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": BATCH * 196608 + BATCH * 4,
                     "d2h_bytes_per_step": 4,
@@ -239,7 +242,9 @@ def run_ours(args, rank, world, local_rank):
             "gpu_launches": launches,
             "clocks": clocks,
             "roofline": {"bound": "tensor", "kernel": "tc::" + dom, "achieved": achieved, "peak": tf_peak, "unit": "TFLOP/s",
-                         "frac": achieved / tf_peak, "traffic": None, "peak_kind": f"bf16 sustained, {kind}",
+                         "frac": achieved / tf_peak, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(dom),
+                         "traffic_unit": "bytes per launch (dram read + write, ncu, average over the kernel's launches of one step)",
+                         "peak_kind": f"bf16 sustained, {kind}",
                          "launches_per_step": per_kernel[dom]["launches_per_step"],
                          "ms_per_step": per_kernel[dom]["ms_per_step"], "all_tensor_kernels": per_kernel},
         }
