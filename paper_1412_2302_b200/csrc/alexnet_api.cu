@@ -750,31 +750,31 @@ void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
 }
 // fused LRN + pool kernels, instantiated for the two LRN layers: {vectors per pixel, vectors per block, W, H, output rows
 // per block, threads} forward; {vectors per pixel, W, H, pixels per pass, threads} backward
-#define LRN_POOL_FWD_1 kn::lrn_pool_fwd_kernel<12, 6, 55, 55, 3, 352>
-#define LRN_POOL_FWD_2 kn::lrn_pool_fwd_kernel<32, 8, 27, 27, 3, 224>
-#define POOL_LRN_BWD_1 kn::pool_lrn_bwd_kernel<12, 55, 55, 28, 352>
-#define POOL_LRN_BWD_2 kn::pool_lrn_bwd_kernel<32, 27, 27, 9, 288>
+// (the last parameter: exponent beta = 0.75 known at compile time)
+#define LRN_POOL_FWD_1(B75) kn::lrn_pool_fwd_kernel<12, 6, 55, 55, 3, 352, B75>
+#define LRN_POOL_FWD_2(B75) kn::lrn_pool_fwd_kernel<32, 8, 27, 27, 3, 224, B75>
+#define POOL_LRN_BWD_1(B75) kn::pool_lrn_bwd_kernel<12, 55, 55, 28, 352, B75>
+#define POOL_LRN_BWD_2(B75) kn::pool_lrn_bwd_kernel<32, 27, 27, 9, 288, B75>
 void op_lrn_pool_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
     const PoolGeo& g = kPool[which];
-    if (which == 0)
-        launch_k(LRN_POOL_FWD_1, dim3((g.Ho + 2) / 3, 2, h->B), 352, (size_t)7 * 55 * 6 * 16, st, R.a1, R.p1, R.arg1, g.Hpi, g.Wpi, g.Hpo,
-                 g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
-    else
-        launch_k(LRN_POOL_FWD_2, dim3((g.Ho + 2) / 3, 4, h->B), 224, (size_t)7 * 27 * 8 * 16, st, R.a2, R.p2, R.arg2, g.Hpi, g.Wpi, g.Hpo,
-                 g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
+    const bool b75 = h->cfg.lrn_beta == 0.75f;
+    const dim3 grid((g.Ho + 2) / 3, which == 0 ? 2 : 4, h->B);
+    const size_t smem = which == 0 ? (size_t)7 * 55 * 6 * 16 : (size_t)7 * 27 * 8 * 16;
+    auto k = which == 0 ? (b75 ? LRN_POOL_FWD_1(true) : LRN_POOL_FWD_1(false)) : (b75 ? LRN_POOL_FWD_2(true) : LRN_POOL_FWD_2(false));
+    launch_k(k, grid, which == 0 ? 352 : 224, smem, st, which ? R.a2 : R.a1, which ? R.p2 : R.p1, which ? R.arg2 : R.arg1, g.Hpi, g.Wpi,
+             g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
     h->launches++;
     R.n_stale[which] = true;
 }
 void op_pool_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
     const PoolGeo& g = kPool[which];
-    if (which == 0)
-        launch_k(POOL_LRN_BWD_1, dim3((g.Hpi + 1) / 2, h->B), 352, (size_t)2 * 55 * 12 * 32, st, R.a1, R.dp1, R.arg1, R.da1, g.Hpi, g.Wpi,
-                 g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
-    else
-        launch_k(POOL_LRN_BWD_2, dim3((g.Hpi + 1) / 2, h->B), 288, (size_t)2 * 27 * 32 * 32, st, R.a2, R.dp2, R.arg2, R.da2, g.Hpi, g.Wpi,
-                 g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
+    const bool b75 = h->cfg.lrn_beta == 0.75f;
+    const size_t smem = which == 0 ? (size_t)2 * 55 * 12 * 32 : (size_t)2 * 27 * 32 * 32;
+    auto k = which == 0 ? (b75 ? POOL_LRN_BWD_1(true) : POOL_LRN_BWD_1(false)) : (b75 ? POOL_LRN_BWD_2(true) : POOL_LRN_BWD_2(false));
+    launch_k(k, dim3((g.Hpi + 1) / 2, h->B), which == 0 ? 352 : 288, smem, st, which ? R.a2 : R.a1, which ? R.dp2 : R.dp1,
+             which ? R.arg2 : R.arg1, which ? R.da2 : R.da1, g.Hpi, g.Wpi, g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
     h->launches++;
     R.dn_stale[which] = true;
 }
@@ -999,8 +999,10 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     CKC(cudaFuncSetAttribute(tc::conv_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     // (static + dynamic shared memory of both exceeds the 48 KB that need no opt-in)
-    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 32));
-    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 32));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 32));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 32));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 32));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 32));
     {
         int dev = 0;
         CKC(cudaGetDevice(&dev));

@@ -95,12 +95,19 @@ __global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* 
 __device__ __forceinline__ float rsqrt_fast(float x) { float y; asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 __device__ __forceinline__ float sqrt_fast(float x) { float y; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
 // s^-beta and 1/s; the exponent 0.75 of the paper's network costs two special-function instructions
-__device__ __forceinline__ void pow_neg(float s, float beta, float& sp, float& rs) {
-    if (beta == 0.75f) { const float r = rsqrt_fast(s); sp = r * sqrt_fast(r); rs = r * r; }
+// B75: the exponent is known to be 0.75 at compile time (the fused kernels of the training step are instantiated both ways,
+// so that their inner loops carry no test of beta)
+template <bool B75>
+__device__ __forceinline__ void pow_neg_t(float s, float beta, float& sp, float& rs) {
+    if (B75) { const float r = rsqrt_fast(s); sp = r * sqrt_fast(r); rs = r * r; }
     else { sp = exp2f(-beta * __log2f(s)); rs = __fdividef(1.f, s); }
 }
+__device__ __forceinline__ void pow_neg(float s, float beta, float& sp, float& rs) {
+    if (beta == 0.75f) pow_neg_t<true>(s, beta, sp, rs); else pow_neg_t<false>(s, beta, sp, rs);
+}
 // b_c = a_c * (k + alpha * sum_{c' in [c-2,c+2] clipped} a_c'^2)^(-beta); one thread = 8 channels of one pixel.
-__device__ __forceinline__ uint4 lrn_fwd8(const uint4* ap, bool has_l, bool has_r, float alpha, float beta, float k) {
+template <bool B75>
+__device__ __forceinline__ uint4 lrn_fwd8_t(const uint4* ap, bool has_l, bool has_r, float alpha, float beta, float k) {
     const uint4 zero = make_uint4(0, 0, 0, 0);
     float f[24];
     unpack8(has_l ? __ldg(ap - 1) : zero, f);
@@ -114,10 +121,13 @@ __device__ __forceinline__ uint4 lrn_fwd8(const uint4* ap, bool has_l, bool has_
     for (int i = 0; i < 8; ++i) {
         const float ss = (sq[i] + sq[i + 1]) + (sq[i + 2] + sq[i + 3]) + sq[i + 4];
         float sp, rs;
-        pow_neg(fmaf(alpha, ss, k), beta, sp, rs);
+        pow_neg_t<B75>(fmaf(alpha, ss, k), beta, sp, rs);
         o[i] = f[8 + i] * sp;
     }
     return pack8(o);
+}
+__device__ __forceinline__ uint4 lrn_fwd8(const uint4* ap, bool has_l, bool has_r, float alpha, float beta, float k) {
+    return beta == 0.75f ? lrn_fwd8_t<true>(ap, has_l, has_r, alpha, beta, k) : lrn_fwd8_t<false>(ap, has_l, has_r, alpha, beta, k);
 }
 __global__ void __launch_bounds__(256) lrn_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ b,
                                                       unsigned total, unsigned cpr, float alpha, float beta, float k) {
@@ -259,7 +269,7 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 // (bits << 16) | (8 - tap) and the window's maximum key carries the largest value and, among equal values, the first
 // tap in scan order - pool_fwd_kernel's tie rule.
 // grid: (ceil(HO / OPR), CPR / CV, B); dynamic shared memory (2*OPR+1) * WI * CV * 16 bytes.
-template <int CPR, int CV, int WI, int HI, int OPR, int NT>
+template <int CPR, int CV, int WI, int HI, int OPR, int NT, bool B75>
 __global__ void __launch_bounds__(NT) lrn_pool_fwd_kernel(const __nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ y,
                                                           uint8_t* __restrict__ arg, int Hpi, int Wpi, int Hpo, int Wpo,
                                                           float alpha, float beta, float k) {
@@ -272,7 +282,7 @@ __global__ void __launch_bounds__(NT) lrn_pool_fwd_kernel(const __nv_bfloat16* _
         const int x = q / CV, ch = c0 + q % CV;
         const uint4* ap = (const uint4*)a + ((size_t)(n * Hpi + iy0) * Wpi + x) * CPR + ch;
         for (int r = 0; r < nrows; ++r) {
-            uint4 v = lrn_fwd8(ap + (size_t)r * Wpi * CPR, ch > 0, ch < CPR - 1, alpha, beta, k);
+            uint4 v = lrn_fwd8_t<B75>(ap + (size_t)r * Wpi * CPR, ch > 0, ch < CPR - 1, alpha, beta, k);
             v.x &= 0x7fff7fffu; v.y &= 0x7fff7fffu; v.z &= 0x7fff7fffu; v.w &= 0x7fff7fffu;
             nrm[r * RV + q] = v;
         }
@@ -318,7 +328,7 @@ __global__ void __launch_bounds__(NT) lrn_pool_fwd_kernel(const __nv_bfloat16* _
 // to bf16 (as pool_bwd_kernel stores it), s^-beta, tt = dn a s^(-beta-1), the tt of the two channels on either side
 // from the neighbouring threads through shared memory, and da with the ReLU mask of the convolution that produced a.
 // Pad pixels of the grid get zero.  grid: (ceil(Hpi / 2), B); dynamic shared memory 2 * WI * CPR * 32 bytes.
-template <int CPR, int WI, int HI, int PPB, int NT>
+template <int CPR, int WI, int HI, int PPB, int NT, bool B75>
 __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ dp,
                                                           const uint8_t* __restrict__ arg, __nv_bfloat16* __restrict__ da,
                                                           int Hpi, int Wpi, int Hpo, int Wpo, float alpha, float beta, float k) {
@@ -403,7 +413,7 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
                 for (int i = 0; i < 8; ++i) {
                     const float ss = (sq[i] + sq[i + 1]) + (sq[i + 2] + sq[i + 3]) + sq[i + 4];
                     float rs;
-                    pow_neg(fmaf(alpha, ss, k), beta, sp[i], rs);
+                    pow_neg_t<B75>(fmaf(alpha, ss, k), beta, sp[i], rs);
                     tt[i] = g8[i] * fa[8 + i] * sp[i] * rs;
                 }
             } else {
