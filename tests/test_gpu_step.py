@@ -119,9 +119,11 @@ def test_conv1_block_batch2():
     net.close()
 
 
-@pytest.mark.parametrize("vp", [True, False])
-def test_full_step_batch32(vp):
-    seed, B = BASE + 2, 32
+# batch 32 (two initialisations) and ragged batches whose grids fill a fraction of a tile (1), a few tiles (5) and an odd
+# number of CTA-pair tiles (17)
+@pytest.mark.parametrize("B,vp", [(32, True), (32, False), (1, True), (5, True), (17, True)])
+def test_full_step(B, vp):
+    seed = BASE + 2
     net = make(B, seed=seed)
     w = synth.init_params(seed, variance_preserving=vp, bias=0.1 if vp else 0.0)
     net.set_params(w)
