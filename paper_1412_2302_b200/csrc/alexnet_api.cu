@@ -771,7 +771,7 @@ void op_pool_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
     const PoolGeo& g = kPool[which];
     const bool b75 = h->cfg.lrn_beta == 0.75f;
-    const size_t smem = which == 0 ? (size_t)2 * 55 * 12 * 32 : (size_t)2 * 27 * 32 * 32;
+    const size_t smem = which == 0 ? (size_t)2 * 55 * 12 * 48 : (size_t)2 * 27 * 32 * 48;     // gradient tile (fp32) + two rows of a
     auto k = which == 0 ? (b75 ? POOL_LRN_BWD_1(true) : POOL_LRN_BWD_1(false)) : (b75 ? POOL_LRN_BWD_2(true) : POOL_LRN_BWD_2(false));
     launch_k(k, dim3((g.Hpi + 1) / 2, h->B), which == 0 ? 352 : 288, smem, st, which ? R.a2 : R.a1, which ? R.dp2 : R.dp1,
              which ? R.arg2 : R.arg1, which ? R.da2 : R.da1, g.Hpi, g.Wpi, g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
@@ -999,10 +999,10 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     CKC(cudaFuncSetAttribute(tc::conv_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     // (static + dynamic shared memory of both exceeds the 48 KB that need no opt-in)
-    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 32));
-    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 32));
-    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 32));
-    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 32));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 48));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 48));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 48));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 48));
     {
         int dev = 0;
         CKC(cudaGetDevice(&dev));

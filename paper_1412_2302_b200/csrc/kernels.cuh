@@ -327,7 +327,7 @@ __global__ void __launch_bounds__(NT) lrn_pool_fwd_kernel(const __nv_bfloat16* _
 // without atomics and in a fixed order.  Then one thread = 8 channels of one pixel (PPB pixels at a time): dn rounded
 // to bf16 (as pool_bwd_kernel stores it), s^-beta, tt = dn a s^(-beta-1), the tt of the two channels on either side
 // from the neighbouring threads through shared memory, and da with the ReLU mask of the convolution that produced a.
-// Pad pixels of the grid get zero.  grid: (ceil(Hpi / 2), B); dynamic shared memory 2 * WI * CPR * 32 bytes.
+// Pad pixels of the grid get zero.  grid: (ceil(Hpi / 2), B); dynamic shared memory 2 * WI * CPR * 48 bytes.
 template <int CPR, int WI, int HI, int PPB, int NT, bool B75>
 __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ dp,
                                                           const uint8_t* __restrict__ arg, __nv_bfloat16* __restrict__ da,
@@ -338,6 +338,7 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
     __shared__ float4 edge[2][NT];    // tt of the two lowest and two highest channels of every thread, for its neighbours
     extern __shared__ float dn[];     // [2 planes: channels 0-3 / 4-7 of a vector][2 rows][WI][CPR] float4 (conflict-free reads)
     constexpr int PLANE = 2 * RV * 4; // floats per plane
+    uint4* const as = (uint4*)(dn + 2 * PLANE);     // then the block's two rows of a, [2][WI][CPR] vectors
     const int j = blockIdx.x, n = blockIdx.y, y0 = 2 * j;
     const uint4 zero4 = make_uint4(0, 0, 0, 0);
     if (y0 >= HI) {                   // pad rows of the grid
@@ -359,11 +360,22 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
             wdp[pass] = __ldg((const uint4*)dp + ((size_t)(n * Hpo + oy) * Wpo + ox) * CPR + wch);
         }
     }
+    // the two rows of a travel to shared memory asynchronously, behind the scatter passes (the LRN part then reads a and
+    // its channel neighbours from there instead of waiting for global memory three times per vector)
+    for (int i = threadIdx.x; i < 2 * RV; i += NT) {
+        const int row = i / RV, q = i - row * RV;
+        if (y0 + row < HI) {
+            const uint4* src = (const uint4*)a + (size_t)(n * Hpi + y0 + row) * Wpi * CPR + q;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(as + i)), "l"(src) : "memory");
+        }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
     for (int i = threadIdx.x; i < 4 * RV; i += NT) ((float4*)dn)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncthreads();
     #pragma unroll
     for (int pass = 0; pass < 4; ++pass) {
         const int oy = j - 1 + (pass >> 1), par = pass & 1;
+        if (pass == 3) asm volatile("cp.async.wait_group 0;" ::: "memory");     // before the last barrier of the passes
         if (has[pass]) {
             const int ox = 2 * wq + par;
             float f[8];
@@ -402,10 +414,10 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
                 const float4 g0 = gp[0], g1 = gp[PLANE / 4];
                 const float acc[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
                 unpack8(pack8(acc), g8);
-                const uint4* ap = (const uint4*)a + ((size_t)(n * Hpi + yy) * Wpi + x) * CPR + ch;
-                unpack8(ch > 0 ? __ldg(ap - 1) : zero4, fa);
-                unpack8(__ldg(ap), fa + 8);
-                unpack8(ch < CPR - 1 ? __ldg(ap + 1) : zero4, fa + 16);
+                const uint4* ap = as + (row * WI + x) * CPR + ch;
+                unpack8(ch > 0 ? ap[-1] : zero4, fa);
+                unpack8(ap[0], fa + 8);
+                unpack8(ch < CPR - 1 ? ap[1] : zero4, fa + 16);
                 float sq[12];
                 #pragma unroll
                 for (int i = 0; i < 12; ++i) sq[i] = fa[6 + i] * fa[6 + i];
