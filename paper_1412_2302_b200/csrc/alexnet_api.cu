@@ -388,7 +388,7 @@ void finish_conv_plan(const alexnet* h, Plan& P) {
     const size_t a_bytes = (size_t)c.MH * c.cpg * c.a_box_rows * 128, b_bytes = (size_t)(c.BN / c.cg) * 128;
     if (c.epi_sets < 1) c.epi_sets = 1;
     const size_t budget = 227 * 1024 - 2048 - 4 * c.epi_sets * tc::kEpiStageBytes;
-    c.tpg = c.cpg > 1 ? c.cpg : (c.kw <= 3 ? c.kw : 2);   // weight tiles travel in groups: a filter row (2 + 2 + 1 taps of a five-tap row, which keeps
+    c.tpg = c.b_res ? c.kh * c.kw : c.cpg > 1 ? c.cpg : (c.kw <= 3 ? c.kw : 2);   // weight tiles travel in groups: a filter row (2 + 2 + 1 taps of a five-tap row, which keeps
                                                           // four groups in flight), or the chunks of an FC stage
     const size_t g_bytes = b_bytes * c.tpg;
     if (c.kw == 1) {
@@ -441,6 +441,9 @@ int plan_conv_fwd(alexnet* h, Plan& P, const ConvL& c, const bf16* in, const bf1
     if ((rc = make_tm(h, &p.tmA, in, c.cin, M, (uint64_t)c.cin * 2, p.a_box_rows))) return rc;
     if ((rc = make_tm(h, &p.tmB, wsh, c.cig, (uint64_t)c.taps * c.cout, (uint64_t)c.cig * 2, p.BN / p.cg))) return rc;
     if ((rc = conv_out_map(h, p, out, c.cout, M))) return rc;
+    // a layer whose whole filter is one n tile of one chunk (conv1: 9 taps x 96 rows x 128 bytes = 108 KB) keeps it in
+    // shared memory for all the tiles of a CTA; the halo ring gets two stages
+    p.b_res = (p.cg == 1 && p.groups == 1 && p.n_tiles == 1 && p.chunks == 1 && (size_t)p.kh * p.kw * p.BN * 128 <= 112 * 1024) ? 1 : 0;
     finish_conv_plan(h, P);
     return ALEXNET_OK;
 }

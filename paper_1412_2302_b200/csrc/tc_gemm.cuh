@@ -707,6 +707,8 @@ struct ConvParams {
     int tma_store;
     int m_tiles, n_tiles, groups, splits;   // tile decomposition (m fastest, then n, group, k split)
     int tiles_total;
+    int b_res;          // 1: all kh*kw weight tiles of the layer fit in one group slot and stay there for the whole CTA (one
+                        // n tile, one group, one chunk, no split: conv1), loaded once instead of once per tile
     int cg;             // 1, or 2: CTA pairs (clusters of two) work on tiles of 2 x MH halves with cta_group::2 instructions
     int MH;             // 128-row halves per tile and CTA (1, 2 or 4)
     int BN, kk;         // MMA N (multiple of 16, <= 256); K=16 MMAs per weight stage (<= 4)
@@ -870,7 +872,13 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (lane == 0 && p.b_res) {
+            // the whole filter, once: tile t = ky * kw + kx
+            if (vb < p.tiles_total) {
+                mbar_expect_tx(fullB, (uint32_t)(p.kh * kw) * b_bytes);
+                for (int t = 0; t < p.kh * kw; ++t) tma_load_2d(ring_b + t * b_bytes, &p.tmB, 0, t * p.b_tap_rows, fullB);
+            }
+        } else if (lane == 0) {
             ConvCursor tc; tc.init(p, vb, vgrid);
             int sb = 0; uint32_t phb = 0;
             bool ok = true;
@@ -917,9 +925,12 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
             int z = vb / (p.m_tiles * p.n_tiles * p.groups);     // only the split index matters here
             int in_split = vb - z * (p.m_tiles * p.n_tiles * p.groups);
             const int tiles_per_split = p.m_tiles * p.n_tiles * p.groups;
+            const bool b_res = p.b_res != 0;
+            if (b_res && vb < p.tiles_total) ok = mbar_wait_warp(fullB, 0u, abort_flag);      // the resident filter has arrived
             for (int tile = vb; tile < p.tiles_total && ok; tile += vgrid) {
                 const int a_begin = z * per;
                 const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
+                int ares = a_begin + (int)((unsigned)vb % (unsigned)nsteps);      // resident filter: the producer's rotation of the filter rows
                 if (!(ok = mbar_wait_warp(acce0 + 8u * ab, aph ^ 1u, abort_flag))) break;
                 if (CG == 2) fence_acq_rel_cluster();      // the peer's epilogue arrived from the other CTA
                 tc_fence_after();
@@ -931,8 +942,8 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                     // the MMAs of a weight group in straight-line code: the fixed cost of a loop trip with a barrier wait
                     // (a few hundred cycles) is paid once per taps*kk instructions
                     for (int kx0 = 0; kx0 < gw; kx0 += p.tpg) {
-                        if (!(ok = mbar_wait_warp(fullB + 8u * sb, phb, abort_flag))) break;
-                        const uint64_t bd = dbase + (uint64_t)((ring_b + sb * g_bytes) >> 4);
+                        if (!b_res && !(ok = mbar_wait_warp(fullB + 8u * sb, phb, abort_flag))) break;
+                        const uint64_t bd = dbase + (uint64_t)((b_res ? ring_b + (uint32_t)(ares * kw) * b_bytes : ring_b + sb * g_bytes) >> 4);
                         const int taps = min(p.tpg, gw - kx0);
                         const int* toff = p.tap_off + kx0;
                         if (kk == 4) {
@@ -945,9 +956,12 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                             else issue_row<1, 3, CG>(d, ad, bd, b_bytes >> 4, toff, idesc, accum);
                         }
                         accum = 1;
-                        umma_commit_cg<CG>(emptyB + 8u * sb);
-                        if (++sb == b_stages) { sb = 0; phb ^= 1u; }
+                        if (!b_res) {
+                            umma_commit_cg<CG>(emptyB + 8u * sb);
+                            if (++sb == b_stages) { sb = 0; phb ^= 1u; }
+                        }
                     }
+                    if (++ares == a_begin + nsteps) ares = a_begin;
                     if (!ok) break;
                     umma_commit_cg<CG>(emptyA + 8u * sa);
                     if (++sa == a_stages) { sa = 0; pha ^= 1u; }
