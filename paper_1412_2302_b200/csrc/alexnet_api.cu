@@ -756,8 +756,8 @@ void op_pool_bwd(alexnet* h, int r, int which, cudaStream_t st) {
 // (the last parameter: exponent beta = 0.75 known at compile time)
 #define LRN_POOL_FWD_1(B75) kn::lrn_pool_fwd_kernel<12, 6, 55, 55, 3, 352, B75>
 #define LRN_POOL_FWD_2(B75) kn::lrn_pool_fwd_kernel<32, 8, 27, 27, 3, 224, B75>
-#define POOL_LRN_BWD_1(B75) kn::pool_lrn_bwd_kernel<12, 55, 55, 28, 352, B75>
-#define POOL_LRN_BWD_2(B75) kn::pool_lrn_bwd_kernel<32, 27, 27, 9, 288, B75>
+#define POOL_LRN_BWD_1(B75) kn::pool_lrn_bwd_kernel<12, 55, 55, 28, 352, B75, true>
+#define POOL_LRN_BWD_2(B75) kn::pool_lrn_bwd_kernel<32, 27, 27, 9, 288, B75, false>
 void op_lrn_pool_fwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
     const PoolGeo& g = kPool[which];
@@ -774,7 +774,7 @@ void op_pool_lrn_bwd(alexnet* h, int r, int which, cudaStream_t st) {
     Replica& R = h->rep[r];
     const PoolGeo& g = kPool[which];
     const bool b75 = h->cfg.lrn_beta == 0.75f;
-    const size_t smem = which == 0 ? (size_t)2 * 55 * 12 * 48 : (size_t)2 * 27 * 32 * 48;     // gradient tile (fp32) + two rows of a
+    const size_t smem = which == 0 ? (size_t)2 * 55 * 12 * 48 : (size_t)2 * 27 * 32 * 32;     // gradient tile (fp32) (+ two rows of a: LRN1)
     auto k = which == 0 ? (b75 ? POOL_LRN_BWD_1(true) : POOL_LRN_BWD_1(false)) : (b75 ? POOL_LRN_BWD_2(true) : POOL_LRN_BWD_2(false));
     launch_k(k, dim3((g.Hpi + 1) / 2, h->B), which == 0 ? 352 : 288, smem, st, which ? R.a2 : R.a1, which ? R.dp2 : R.dp1,
              which ? R.arg2 : R.arg1, which ? R.da2 : R.da1, g.Hpi, g.Wpi, g.Hpo, g.Wpo, h->alpha_eff, h->cfg.lrn_beta, h->cfg.lrn_k);
@@ -1004,8 +1004,8 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     // (static + dynamic shared memory of both exceeds the 48 KB that need no opt-in)
     CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 48));
     CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 48));
-    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 48));
-    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 48));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 32));
+    CKC(cudaFuncSetAttribute(POOL_LRN_BWD_2(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 27 * 32 * 32));
     {
         int dev = 0;
         CKC(cudaGetDevice(&dev));

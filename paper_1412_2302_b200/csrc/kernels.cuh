@@ -328,7 +328,7 @@ __global__ void __launch_bounds__(NT) lrn_pool_fwd_kernel(const __nv_bfloat16* _
 // to bf16 (as pool_bwd_kernel stores it), s^-beta, tt = dn a s^(-beta-1), the tt of the two channels on either side
 // from the neighbouring threads through shared memory, and da with the ReLU mask of the convolution that produced a.
 // Pad pixels of the grid get zero.  grid: (ceil(Hpi / 2), B); dynamic shared memory 2 * WI * CPR * 48 bytes.
-template <int CPR, int WI, int HI, int PPB, int NT, bool B75>
+template <int CPR, int WI, int HI, int PPB, int NT, bool B75, bool STAGE_A>
 __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ dp,
                                                           const uint8_t* __restrict__ arg, __nv_bfloat16* __restrict__ da,
                                                           int Hpi, int Wpi, int Hpo, int Wpo, float alpha, float beta, float k) {
@@ -362,7 +362,7 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
     }
     // the two rows of a travel to shared memory asynchronously, behind the scatter passes (the LRN part then reads a and
     // its channel neighbours from there instead of waiting for global memory three times per vector)
-    for (int i = threadIdx.x; i < 2 * RV; i += NT) {
+    for (int i = threadIdx.x; STAGE_A && i < 2 * RV; i += NT) {
         const int row = i / RV, q = i - row * RV;
         if (y0 + row < HI) {
             const uint4* src = (const uint4*)a + (size_t)(n * Hpi + y0 + row) * Wpi * CPR + q;
@@ -414,10 +414,17 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
                 const float4 g0 = gp[0], g1 = gp[PLANE / 4];
                 const float acc[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
                 unpack8(pack8(acc), g8);
-                const uint4* ap = as + (row * WI + x) * CPR + ch;
-                unpack8(ch > 0 ? ap[-1] : zero4, fa);
-                unpack8(ap[0], fa + 8);
-                unpack8(ch < CPR - 1 ? ap[1] : zero4, fa + 16);
+                if (STAGE_A) {
+                    const uint4* ap = as + (row * WI + x) * CPR + ch;
+                    unpack8(ch > 0 ? ap[-1] : zero4, fa);
+                    unpack8(ap[0], fa + 8);
+                    unpack8(ch < CPR - 1 ? ap[1] : zero4, fa + 16);
+                } else {
+                    const uint4* ap = (const uint4*)a + ((size_t)(n * Hpi + yy) * Wpi + x) * CPR + ch;
+                    unpack8(ch > 0 ? __ldg(ap - 1) : zero4, fa);
+                    unpack8(__ldg(ap), fa + 8);
+                    unpack8(ch < CPR - 1 ? __ldg(ap + 1) : zero4, fa + 16);
+                }
                 float sq[12];
                 #pragma unroll
                 for (int i = 0; i < 12; ++i) sq[i] = fa[6 + i] * fa[6 + i];
