@@ -148,6 +148,7 @@ struct alexnet {
     cudaStream_t cs, ls;   // compute, loader
     cudaStream_t gs = nullptr;             // second compute stream of the backward pass: conv weight gradients (owned)
     cudaEvent_t ev_dy[5] = {}, ev_gs_done = nullptr;   // dy of conv layer l is ready on cs; gs has finished its weight gradients
+    cudaEvent_t ev_fc[3] = {};             // the data gradient of FC layer l has read the layer's weights (fused FC update)
     uint8_t* arena; size_t arena_bytes;
     Replica rep[2];
     float* mean; float* ws; float* cs_partial; float* canon_tmp; int* status;
@@ -828,8 +829,18 @@ void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
     forward(h, r, slot, st, false);
     // the data gradient reads the layer's weights, so it comes first when the weight-gradient kernel updates them in place
     const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0;
+    // With the fused update the weight-gradient kernel of an FC layer (HBM-bound: it streams the layer's weights and momentum)
+    // goes to the second stream once the layer's data gradient has read the old weights; the chain of small data-gradient
+    // kernels and reductions continues beside it.
+    const bool fork_fc = fused && h->gs != nullptr && !h->prof;
     for (int l = 2; l >= 0; --l) {
-        if (fused) { op_fc_bwd(h, r, l, st); op_fc_wg(h, r, l, l == 2, st); }
+        if (fork_fc) {
+            op_fc_bwd(h, r, l, st);
+            cudaEventRecord(h->ev_fc[l], st);
+            cudaStreamWaitEvent(h->gs, h->ev_fc[l], 0);
+            op_fc_wg(h, r, l, l == 2, h->gs);
+        }
+        else if (fused) { op_fc_bwd(h, r, l, st); op_fc_wg(h, r, l, l == 2, st); }
         else { op_fc_wg(h, r, l, l == 2, st); op_fc_bwd(h, r, l, st); }
     }
     op_pool_bwd(h, r, 2, st);
@@ -1013,6 +1024,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     }
     CKC(cudaStreamCreateWithFlags(&h->gs, cudaStreamNonBlocking));
     for (int l = 0; l < 5; ++l) CKC(cudaEventCreateWithFlags(&h->ev_dy[l], cudaEventDisableTiming));
+    for (int l = 0; l < 3; ++l) CKC(cudaEventCreateWithFlags(&h->ev_fc[l], cudaEventDisableTiming));
     CKC(cudaEventCreateWithFlags(&h->ev_gs_done, cudaEventDisableTiming));
     // pad positions of every grid must be zero from the start; gradients and momentum start at zero
     CKC(cudaMemsetAsync(h->arena, 0, need, h->cs));
@@ -1046,6 +1058,7 @@ int alexnet_destroy(alexnet_t* h) {
     cudaStreamSynchronize(h->ls);
     if (h->gs) { cudaStreamSynchronize(h->gs); cudaStreamDestroy(h->gs); }
     for (int l = 0; l < 5; ++l) if (h->ev_dy[l]) cudaEventDestroy(h->ev_dy[l]);
+    for (int l = 0; l < 3; ++l) if (h->ev_fc[l]) cudaEventDestroy(h->ev_fc[l]);
     if (h->ev_gs_done) cudaEventDestroy(h->ev_gs_done);
     for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
     for (int r = 0; r < h->cfg.replicas; ++r)
