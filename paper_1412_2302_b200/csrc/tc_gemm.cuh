@@ -20,6 +20,11 @@
 // tap t reads the input rows of the output tile shifted by shift[t] rows, so
 // every A tile is a plain 2-D TMA box; out-of-range rows are zero-filled by TMA.
 // Every wait is bounded: on expiry the CTA raises *status and drains.
+// conv_kernel also runs as CTA pairs (clusters of two, tcgen05.mma.cta_group::2: one instruction of the leader covers 128
+// rows of each CTA), and gemm_kernel can apply the momentum update to the FC weights in its weight-gradient epilogue.
+// All kernels are launched with programmatic stream serialization: they let the next launch of the stream start early
+// (griddepcontrol.launch_dependents first thing) and wait for their predecessors (griddepcontrol.wait) after their
+// barriers, tensor memory and descriptors are set up and before they touch global memory.
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
