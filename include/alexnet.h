@@ -106,11 +106,11 @@ int alexnet_load_batch_async(alexnet_t* h, int replica, const uint8_t* images, c
  * updated on different minibatches respectively"): forward, softmax
  * cross-entropy, backward, momentum update
  *   v <- momentum*v - lr*weight_decay*w - lr*g ; w <- w + v   (decay on weights only unless flagged).
- * Runs on the compute stream after the batch's load has finished; part of
- * the backward pass (the convolution weight gradients) runs on a stream the
- * handle owns, forked from and joined into the compute stream inside the
- * call, so work queued on the compute stream afterwards is ordered after
- * the whole step.  If host_loss is non-NULL the mean loss is written there and the call
+ * Runs on the compute stream after the batch's load has finished; the
+ * independent branches of the backward pass (weight gradients) run on
+ * streams the handle owns, forked from and joined into the compute stream
+ * inside the call, so work queued on the compute stream afterwards is
+ * ordered after the whole step.  If host_loss is non-NULL the mean loss is written there and the call
  * synchronises the compute stream; otherwise it is asynchronous.
  * Errors: STATE (no loaded batch), DEVICE_TIMEOUT (latched), CUDA. */
 int alexnet_train_step(alexnet_t* h, int replica, float* host_loss);

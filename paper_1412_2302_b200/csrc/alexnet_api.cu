@@ -113,6 +113,7 @@ Layout make_layout() {
 const long long kCanonCount = 60965224;
 
 // ------------------------------------------------------------------- handle
+constexpr size_t kBiasPartial = 65536;    // floats per conv layer: row splits (<= 148) x output channels (<= 384)
 struct Plan { tc::GemmParams p; tc::ConvParams c; tc::WgradParams w; bool conv, wgrad; int grid; size_t smem; bool valid; };
 
 struct Tensor {  // description of one exportable device tensor
@@ -146,9 +147,15 @@ struct alexnet {
     Layout L;
     int B;
     cudaStream_t cs, ls;   // compute, loader
-    cudaStream_t gs = nullptr;             // second compute stream of the backward pass: conv weight gradients (owned)
-    cudaEvent_t ev_dy[5] = {}, ev_gs_done = nullptr;   // dy of conv layer l is ready on cs; gs has finished its weight gradients
-    cudaEvent_t ev_fc[3] = {};             // the data gradient of FC layer l has read the layer's weights (fused FC update)
+    // The independent branches of the backward pass - the weight gradient (+ update) of FC layer l (branch l) and the weight
+    // gradient + split reduction of conv layer l (branch 3 + l) - each run on a stream of their own (owned by the handle),
+    // forked from the compute stream when their inputs exist and joined before the update.
+    static const int kBranches = 8;
+    cudaStream_t side[kBranches] = {};
+    cudaEvent_t ev_side_done[kBranches] = {};
+    cudaEvent_t ev_fork[kBranches] = {};   // the inputs of branch b are ready on the compute stream
+    size_t ws_conv_off[5] = {};            // floats: each conv layer's split partials have their own region of the workspace
+    float* bias_partial = nullptr;         // [5][kBiasPartial] bias-gradient partials of the conv weight-gradient kernels
     uint8_t* arena; size_t arena_bytes;
     Replica rep[2];
     float* mean; float* ws; float* cs_partial; float* canon_tmp; int* status;
@@ -208,15 +215,19 @@ int fc_bwd_splits(const FcL& f, int B) {
     const int tiles = ((B + 127) / 128) * (f.K / 256);
     return pick_splits(tiles, (f.N + 63) / 64);
 }
-size_t ws_need(const Layout& L, int B) {
+// split-K workspace in floats: one region shared by the FC passes (they follow one another on the compute stream), then one
+// region per conv layer's weight-gradient partials (those kernels run side by side); conv_off receives the conv regions' offsets
+size_t ws_need(const Layout& L, int B, size_t* conv_off = nullptr) {
     size_t need = 0;
-    for (int l = 0; l < 5; ++l) {
-        const ConvL& c = L.conv[l];
-        need = std::max(need, (size_t)conv_wg_splits(c, B) * c.taps * c.cout * c.cig);
-    }
     for (int l = 0; l < 3; ++l) {
         need = std::max(need, (size_t)fc_fwd_splits(L.fc[l], B) * B * L.fc[l].N);
         need = std::max(need, (size_t)fc_bwd_splits(L.fc[l], B) * B * L.fc[l].K);
+    }
+    for (int l = 0; l < 5; ++l) {
+        const ConvL& c = L.conv[l];
+        need = (need + 63) / 64 * 64;
+        if (conv_off) conv_off[l] = need;
+        need += (size_t)conv_wg_splits(c, B) * c.taps * c.cout * c.cig;
     }
     return need;
 }
@@ -228,9 +239,10 @@ size_t carve(alexnet* h, uint8_t* base) {
     const int B = h->B;
     auto rows = [&](const Grid& g) { return (size_t)B * g.Hp * g.Wp; };
     h->mean = c.take<float>(256 * 256 * 3);
-    h->ws_floats = ws_need(L, B);
+    h->ws_floats = ws_need(L, B, h->ws_conv_off);
     h->ws = c.take<float>(h->ws_floats);
     h->cs_partial = c.take<float>(256 * 4096);
+    h->bias_partial = c.take<float>(5 * kBiasPartial);
     h->canon_tmp = c.take<float>(kCanonCount);
     h->status = c.take<int>(16);
     for (int r = 0; r < h->cfg.replicas; ++r) {
@@ -474,7 +486,7 @@ int plan_conv_bwd(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf1
     finish_conv_plan(h, P);
     return ALEXNET_OK;
 }
-int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16* xin) {
+int plan_conv_wg(alexnet* h, Plan& P, int l, const ConvL& c, const bf16* dy, const bf16* xin) {
     memset(&P, 0, sizeof(P));
     tc::WgradParams& p = P.w;
     const long long M = (long long)h->B * c.gin.Hp * c.gin.Wp;
@@ -492,8 +504,8 @@ int plan_conv_wg(alexnet* h, Plan& P, const ConvL& c, const bf16* dy, const bf16
     p.M_total = c.cog; p.n_valid = c.cig; p.ldo = c.cig; p.out_gx = c.cog;
     p.tap_stride = (long long)c.cout * c.cig; p.split_stride = (long long)c.taps * c.cout * c.cig;
     p.epi = tc::EPI_F32; p.mask_scale = 1.f;
-    p.out = h->ws; p.status = h->status;
-    p.bias_partial = h->cs_partial; p.bias_ld = c.cout;
+    p.out = h->ws + h->ws_conv_off[l]; p.status = h->status;
+    p.bias_partial = h->bias_partial + (size_t)l * kBiasPartial; p.bias_ld = c.cout;
     int rc;
     if ((rc = make_tm(h, &p.tmA, dy, c.cout, M, (uint64_t)c.cout * 2, tc::kWgRows))) return rc;
     if ((rc = make_tm(h, &p.tmB, xin, c.cin, M, (uint64_t)c.cin * 2, tc::kWgRows + 8))) return rc;
@@ -584,7 +596,7 @@ int build_plans(alexnet* h, int r) {
         for (int s = 0; s < 2; ++s) {
             const bf16* x = l == 0 ? R.x0[s] : in[l];
             if ((rc = plan_conv_fwd(h, R.conv_fwd[l][s], c, x, R.shadow + c.w_off, R.w + c.b_off, out[l]))) return rc;
-            if ((rc = plan_conv_wg(h, R.conv_wg[l][s], c, dyv[l], x))) return rc;
+            if ((rc = plan_conv_wg(h, R.conv_wg[l][s], l, c, dyv[l], x))) return rc;
         }
         if ((rc = plan_conv_bwd(h, R.conv_bwd[l], c, dyv[l], R.wt + c.wt_off, maskv[l], dxv[l]))) return rc;
     }
@@ -662,8 +674,8 @@ void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
     const Plan& P = R.conv_wg[l][slot];
     launch_gemm(h, P, st);     // weight-gradient partials per row split, and the bias-gradient partials
     const long long total = (long long)c.taps * c.cout * c.cig;
-    launch_k(kn::wgrad_reduce_kernel, nblk(total, 256), 256, 0, st, h->ws, P.w.splits, P.w.split_stride, total, R.g + c.w_off, l == 0,
-                                                              h->cs_partial, c.cout, R.g + c.b_off);
+    launch_k(kn::wgrad_reduce_kernel, nblk(total, 256), 256, 0, st, h->ws + h->ws_conv_off[l], P.w.splits, P.w.split_stride, total,
+             R.g + c.w_off, l == 0, h->bias_partial + (size_t)l * kBiasPartial, c.cout, R.g + c.b_off);
     h->launches++;
 }
 void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool eval = false) {
@@ -829,44 +841,39 @@ void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
     forward(h, r, slot, st, false);
     // the data gradient reads the layer's weights, so it comes first when the weight-gradient kernel updates them in place
     const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0;
-    // With the fused update the weight-gradient kernel of an FC layer (HBM-bound: it streams the layer's weights and momentum)
-    // goes to the second stream once the layer's data gradient has read the old weights; the chain of small data-gradient
-    // kernels and reductions continues beside it.
-    const bool fork_fc = fused && h->gs != nullptr && !h->prof;
+    // Every independent branch of the backward pass runs on its own stream: with the fused update the weight-gradient kernel
+    // of an FC layer (HBM-bound: it streams the layer's weights and momentum) once the layer's data gradient has read the old
+    // weights, and the weight gradient of a conv layer (kernel, then split reduction) once the layer's dy exists.  The chain
+    // of data gradients stays on `st`.  The kernels of the branches fill the SMs that the chain leaves idle (small split
+    // GEMMs and reductions of the FC layers, last rounds and tails of the conv kernels) and overlap HBM-bound with
+    // tensor-bound work; each branch has its own region of the split workspace and of the bias partials.  `st` joins all
+    // branches before it returns.  Per-kernel profiling keeps everything on one stream.
+    const bool fork = h->side[0] != nullptr && !h->prof;
+    bool used[alexnet::kBranches] = {};
+    auto branch = [&](int b) -> cudaStream_t {       // fork branch b from `st` here
+        if (!fork) return st;
+        cudaEventRecord(h->ev_fork[b], st);
+        cudaStreamWaitEvent(h->side[b], h->ev_fork[b], 0);
+        used[b] = true;
+        return h->side[b];
+    };
     for (int l = 2; l >= 0; --l) {
-        if (fork_fc) {
-            op_fc_bwd(h, r, l, st);
-            cudaEventRecord(h->ev_fc[l], st);
-            cudaStreamWaitEvent(h->gs, h->ev_fc[l], 0);
-            op_fc_wg(h, r, l, l == 2, h->gs);
-        }
-        else if (fused) { op_fc_bwd(h, r, l, st); op_fc_wg(h, r, l, l == 2, st); }
+        if (fused) { op_fc_bwd(h, r, l, st); op_fc_wg(h, r, l, l == 2, branch(l)); }
         else { op_fc_wg(h, r, l, l == 2, st); op_fc_bwd(h, r, l, st); }
     }
     op_pool_bwd(h, r, 2, st);
-    // The weight gradient of a conv layer and the data gradient that continues the chain both need only the layer's dy.
-    // The chain stays on `st`; the weight gradients (kernel, then split reduction) run on a second stream as soon as
-    // their dy exists, so that their blocks fill the SMs that the chain's kernels leave idle in their last waves.
-    // Nothing on `st` touches the split workspace or the conv gradients meanwhile; `st` joins before it returns.
-    // Per-kernel profiling keeps everything on one stream.
-    const bool two = h->gs != nullptr && !h->prof;
-    cudaStream_t g = two ? h->gs : st;
-    auto dy_ready = [&](int l) {
-        if (!two) return;
-        cudaEventRecord(h->ev_dy[l], st);
-        cudaStreamWaitEvent(h->gs, h->ev_dy[l], 0);
-    };
-    dy_ready(4); op_conv_wg(h, r, 4, slot, g); op_conv_bwd(h, r, 4, st);
-    dy_ready(3); op_conv_wg(h, r, 3, slot, g); op_conv_bwd(h, r, 3, st);
-    dy_ready(2); op_conv_wg(h, r, 2, slot, g); op_conv_bwd(h, r, 2, st);
+    op_conv_wg(h, r, 4, slot, branch(3 + 4)); op_conv_bwd(h, r, 4, st);
+    op_conv_wg(h, r, 3, slot, branch(3 + 3)); op_conv_bwd(h, r, 3, st);
+    op_conv_wg(h, r, 2, slot, branch(3 + 2)); op_conv_bwd(h, r, 2, st);
     op_pool_lrn_bwd(h, r, 1, st);
-    dy_ready(1); op_conv_wg(h, r, 1, slot, g); op_conv_bwd(h, r, 1, st);
+    op_conv_wg(h, r, 1, slot, branch(3 + 1)); op_conv_bwd(h, r, 1, st);
     op_pool_lrn_bwd(h, r, 0, st);
-    dy_ready(0); op_conv_wg(h, r, 0, slot, g);
-    if (two) {
-        cudaEventRecord(h->ev_gs_done, h->gs);
-        cudaStreamWaitEvent(st, h->ev_gs_done, 0);
-    }
+    op_conv_wg(h, r, 0, slot, branch(3 + 0));
+    for (int b = 0; b < alexnet::kBranches; ++b)
+        if (used[b]) {
+            cudaEventRecord(h->ev_side_done[b], h->side[b]);
+            cudaStreamWaitEvent(st, h->ev_side_done[b], 0);
+        }
 }
 
 int check_status(alexnet* h) {
@@ -1022,10 +1029,11 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
         CKC(cudaGetDevice(&dev));
         CKC(cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, dev));
     }
-    CKC(cudaStreamCreateWithFlags(&h->gs, cudaStreamNonBlocking));
-    for (int l = 0; l < 5; ++l) CKC(cudaEventCreateWithFlags(&h->ev_dy[l], cudaEventDisableTiming));
-    for (int l = 0; l < 3; ++l) CKC(cudaEventCreateWithFlags(&h->ev_fc[l], cudaEventDisableTiming));
-    CKC(cudaEventCreateWithFlags(&h->ev_gs_done, cudaEventDisableTiming));
+    for (int b = 0; b < alexnet::kBranches; ++b) {
+        CKC(cudaStreamCreateWithFlags(&h->side[b], cudaStreamNonBlocking));
+        CKC(cudaEventCreateWithFlags(&h->ev_side_done[b], cudaEventDisableTiming));
+        CKC(cudaEventCreateWithFlags(&h->ev_fork[b], cudaEventDisableTiming));
+    }
     // pad positions of every grid must be zero from the start; gradients and momentum start at zero
     CKC(cudaMemsetAsync(h->arena, 0, need, h->cs));
     if (host_mean_image) CKC(cudaMemcpyAsync(h->mean, host_mean_image, 256 * 256 * 3 * sizeof(float), cudaMemcpyHostToDevice, h->cs));
@@ -1056,10 +1064,11 @@ int alexnet_destroy(alexnet_t* h) {
     if (!h) return ALEXNET_ERR_ARG;
     cudaStreamSynchronize(h->cs);
     cudaStreamSynchronize(h->ls);
-    if (h->gs) { cudaStreamSynchronize(h->gs); cudaStreamDestroy(h->gs); }
-    for (int l = 0; l < 5; ++l) if (h->ev_dy[l]) cudaEventDestroy(h->ev_dy[l]);
-    for (int l = 0; l < 3; ++l) if (h->ev_fc[l]) cudaEventDestroy(h->ev_fc[l]);
-    if (h->ev_gs_done) cudaEventDestroy(h->ev_gs_done);
+    for (int b = 0; b < alexnet::kBranches; ++b) {
+        if (h->side[b]) { cudaStreamSynchronize(h->side[b]); cudaStreamDestroy(h->side[b]); }
+        if (h->ev_side_done[b]) cudaEventDestroy(h->ev_side_done[b]);
+        if (h->ev_fork[b]) cudaEventDestroy(h->ev_fork[b]);
+    }
     for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
     for (int r = 0; r < h->cfg.replicas; ++r)
         for (int s = 0; s < 2; ++s) { cudaEventDestroy(h->rep[r].ready[s]); cudaEventDestroy(h->rep[r].consumed[s]); }
