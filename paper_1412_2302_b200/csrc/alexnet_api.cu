@@ -108,6 +108,11 @@ Layout make_layout() {
         const ConvL& c = L.conv[l];
         L.tjobs.j[l] = kn::TransposeJob{c.w_off, c.wt_off, c.taps, c.cout, c.cig, c.groups, (long long)c.taps * c.cin * c.cog};
     }
+    L.tjobs.tile0[0] = 0;
+    for (int l = 0; l < 5; ++l) {
+        const ConvL& c = L.conv[l];
+        L.tjobs.tile0[l + 1] = L.tjobs.tile0[l] + c.taps * (c.cout / 32) * ((c.cig + 31) / 32);
+    }
     return L;
 }
 const long long kCanonCount = 60965224;
@@ -802,14 +807,17 @@ void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
 }
 void op_update(alexnet* h, int r, cudaStream_t st, bool full = false) {
     Replica& R = h->rep[r];
-    const long long nd = (h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES) ? h->L.n_total : h->L.n_weights;
-    // all conv filters precede the FC weights in the internal order
-    // with the fused FC update the FC weights (a contiguous range of the internal order) are already up to date
+    const Layout& L = h->L;
+    const long long nd = (h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES) ? L.n_total : L.n_weights;
+    // internal order: conv filters, FC weights, biases.  The conv filters (with their transposed bf16 copies) have a tiled
+    // kernel of their own; the one-pass kernel takes the rest, minus the FC weights when the fused FC update has done them.
     const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0 && !full;
-    launch_k(kn::sgd_update_kernel, 1184, 256, 0, st, R.w, R.v, R.g, R.shadow, h->L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum,
-                                                h->cfg.weight_decay, R.wt, h->L.tjobs, h->L.fc[0].w_off / 4,
-                                                fused ? h->L.fc[0].w_off / 4 : 0, fused ? h->L.n_weights / 4 : 0);
-    h->launches++;
+    launch_k(kn::sgd_update_conv_kernel, L.tjobs.tile0[5], 256, 0, st, R.w, R.v, R.g, R.shadow, h->cfg.lr * h->cfg.weight_decay,
+             h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs);
+    launch_k(kn::sgd_update_kernel, fused ? 148 : 1184, 256, 0, st, R.w, R.v, R.g, R.shadow, L.n_total / 4, nd / 4, h->cfg.lr,
+             h->cfg.momentum, h->cfg.weight_decay, R.wt, L.tjobs, (long long)0, (long long)0,
+             (fused ? L.n_weights : L.fc[0].w_off) / 4);
+    h->launches += 2;
 }
 void op_average(alexnet* h, cudaStream_t st) {
     Replica &A = h->rep[0], &Bq = h->rep[1];

@@ -668,7 +668,7 @@ __global__ void topk_count_kernel(const float* __restrict__ z, const int32_t* __
 // transposed bf16 copies of the grouped conv filters for the backward-data pass:
 // wt[tap][g*cig + ci][co'] = wf[tap][g*cog + co'][ci]
 struct TransposeJob { long long src_off, dst_off; int taps, cout, cig, groups; long long count; };
-struct TransposeJobs { TransposeJob j[5]; int n; };
+struct TransposeJobs { TransposeJob j[5]; int n; int tile0[6]; };   // tile0: first 32 x 32 tile of each job in sgd_update_conv_kernel's grid
 // one parameter of the momentum update: v <- mu v - d w - lr g (d = lr * weight decay, or 0); w <- w + v.
 // Used by the update kernel and by the FC weight-gradient epilogue that applies the update in place, so that both
 // give bit-identical results.
@@ -718,6 +718,49 @@ __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, 
                 }
             }
         }
+    }
+}
+// The same update for the conv filters, tiled so that the transposed bf16 copies are written in runs: one block = one tap,
+// 32 output channels and 32 input channels of one layer.  Thread (r, c4) updates the four consecutive input channels
+// 4*c4 .. 4*c4+3 of output channel r (the source order [tap][cout][cig]: 128-byte runs per row), the bf16 values cross a
+// shared-memory tile, and thread (ci, q) writes four consecutive output channels of input channel ci to the transposed copy
+// [tap][cin][cog] (64-byte runs) where the one-pass kernel writes single elements.  Bit-identical to sgd_update_kernel.
+__global__ void __launch_bounds__(256) sgd_update_conv_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g,
+                                                              __nv_bfloat16* __restrict__ shadow, float d, float lr, float mu,
+                                                              __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs) {
+    pdl_sync();
+    __shared__ __nv_bfloat16 tile[32][36];       // [input channel][output channel], padded
+    int q = 0;
+    while (q + 1 < jobs.n && (int)blockIdx.x >= jobs.tile0[q + 1]) ++q;
+    const TransposeJob J = jobs.j[q];
+    const int cog = J.cout / J.groups;
+    const int ci_blocks = (J.cig + 31) / 32, co_blocks = J.cout / 32;     // cout is a multiple of 32 in every layer
+    int t = (int)blockIdx.x - jobs.tile0[q];
+    const int cib = t % ci_blocks; t /= ci_blocks;
+    const int cob = t % co_blocks, tap = t / co_blocks;
+    const int r = threadIdx.x >> 3, c4 = threadIdx.x & 7;
+    const int co = cob * 32 + r, ci = cib * 32 + 4 * c4;
+    if (ci < J.cig) {                            // cig is a multiple of 4
+        const long long e = J.src_off + ((long long)tap * J.cout + co) * J.cig + ci;
+        float4 wv = *(float4*)(w + e), vv = *(float4*)(v + e);
+        const float4 gv = *(const float4*)(g + e);
+        sgd_step(wv.x, vv.x, gv.x, d, lr, mu);
+        sgd_step(wv.y, vv.y, gv.y, d, lr, mu);
+        sgd_step(wv.z, vv.z, gv.z, d, lr, mu);
+        sgd_step(wv.w, vv.w, gv.w, d, lr, mu);
+        *(float4*)(w + e) = wv;
+        *(float4*)(v + e) = vv;
+        const __nv_bfloat162 lo2 = __floats2bfloat162_rn(wv.x, wv.y), hi2 = __floats2bfloat162_rn(wv.z, wv.w);
+        *(uint2*)(shadow + e) = make_uint2(*(const uint32_t*)&lo2, *(const uint32_t*)&hi2);
+        tile[4 * c4][r] = lo2.x; tile[4 * c4 + 1][r] = lo2.y; tile[4 * c4 + 2][r] = hi2.x; tile[4 * c4 + 3][r] = hi2.y;
+    }
+    __syncthreads();
+    const int ci2 = cib * 32 + r, cq = 4 * c4;   // now: thread (input channel r of the tile, four output channels from cq)
+    if (ci2 < J.cig) {
+        const int co0 = cob * 32 + cq, grp = co0 / cog, col = co0 - grp * cog;
+        __nv_bfloat16* dst = wt + J.dst_off + ((long long)tap * J.cig * J.groups + grp * J.cig + ci2) * cog + col;
+        const __nv_bfloat162 a = __halves2bfloat162(tile[r][cq], tile[r][cq + 1]), b = __halves2bfloat162(tile[r][cq + 2], tile[r][cq + 3]);
+        *(uint2*)dst = make_uint2(*(const uint32_t*)&a, *(const uint32_t*)&b);
     }
 }
 // exchange-and-average with both replicas in one HBM: w_a = w_b = (w_a+w_b)/2, same for momentum; refresh both shadows.
