@@ -814,9 +814,8 @@ void op_update(alexnet* h, int r, cudaStream_t st, bool full = false) {
     const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0 && !full;
     launch_k(kn::sgd_update_conv_kernel, L.tjobs.tile0[5], 256, 0, st, R.w, R.v, R.g, R.shadow, h->cfg.lr * h->cfg.weight_decay,
              h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs);
-    launch_k(kn::sgd_update_kernel, fused ? 148 : 1184, 256, 0, st, R.w, R.v, R.g, R.shadow, L.n_total / 4, nd / 4, h->cfg.lr,
-             h->cfg.momentum, h->cfg.weight_decay, R.wt, L.tjobs, (long long)0, (long long)0,
-             (fused ? L.n_weights : L.fc[0].w_off) / 4);
+    launch_k(kn::sgd_update_kernel, fused ? 148 : 1184, 256, 0, st, R.w, R.v, R.g, R.shadow, (fused ? L.n_weights : L.fc[0].w_off) / 4,
+             L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum, h->cfg.weight_decay);
     h->launches += 2;
 }
 void op_average(alexnet* h, cudaStream_t st) {

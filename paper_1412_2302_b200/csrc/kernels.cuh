@@ -677,54 +677,32 @@ __device__ __forceinline__ void sgd_step(float& w, float& v, float g, float d, f
     w += v;
 }
 // v <- mu v - lr wd w [i < n_decay] - lr g ; w <- w + v ; bf16 shadow of w.  22 bytes per parameter.
-// The conv filters of layers 2-5 (the first conv_end4 vectors hold all conv filters) are also written to their
-// transposed bf16 copies for the backward-data pass, so no separate transposition pass is needed after a step.
+// Updates the 16-byte vectors [begin4, n4) of the internal order: everything after the conv filters (which
+// sgd_update_conv_kernel takes), or only the biases when the FC weight-gradient kernel has already updated the FC weights.
 __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g,
-                                  __nv_bfloat16* __restrict__ shadow, long long n4, long long n_decay4,
-                                  float lr, float mu, float wd, __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs,
-                                  long long conv_end4, long long skip_begin4, long long skip_end4) {
+                                  __nv_bfloat16* __restrict__ shadow, long long begin4, long long n4, long long n_decay4,
+                                  float lr, float mu, float wd) {
     pdl_sync();
-    // vectors [0, n4) except [skip_begin4, skip_end4): the FC weights, when the FC weight-gradient kernel has already
-    // updated them in its epilogue
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (int part = 0; part < 2; ++part) {
-        const long long lo = part == 0 ? 0 : max(skip_end4, 0LL), hi = part == 0 ? (skip_end4 > skip_begin4 ? skip_begin4 : n4) : n4;
-        if (part == 1 && skip_end4 <= skip_begin4) break;
-        for (long long i = lo + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < hi; i += stride) {
-            float4 wv = ((float4*)w)[i], vv = ((float4*)v)[i];
-            const float4 gv = ((const float4*)g)[i];
-            const float d = i < n_decay4 ? lr * wd : 0.f;
-            sgd_step(wv.x, vv.x, gv.x, d, lr, mu);
-            sgd_step(wv.y, vv.y, gv.y, d, lr, mu);
-            sgd_step(wv.z, vv.z, gv.z, d, lr, mu);
-            sgd_step(wv.w, vv.w, gv.w, d, lr, mu);
-            ((float4*)w)[i] = wv;
-            ((float4*)v)[i] = vv;
-            __nv_bfloat162 lo2 = __floats2bfloat162_rn(wv.x, wv.y), hi2 = __floats2bfloat162_rn(wv.z, wv.w);
-            ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo2, *(uint32_t*)&hi2);
-            if (i < conv_end4) {
-                const long long e = 4 * i;
-                for (int q = 0; q < jobs.n; ++q) {
-                    const TransposeJob J = jobs.j[q];
-                    const long long sidx = e - J.src_off;          // [tap][cout][cig], four consecutive ci
-                    if (sidx < 0 || sidx >= J.count) continue;
-                    const int cog = J.cout / J.groups;
-                    const int ci = (int)(sidx % J.cig);
-                    const long long r = sidx / J.cig;
-                    const int co = (int)(r % J.cout), tap = (int)(r / J.cout);
-                    const int grp = co / cog, co_ = co - grp * cog;
-                    __nv_bfloat16* dst = wt + J.dst_off + ((long long)tap * J.cig * J.groups + grp * J.cig + ci) * cog + co_;
-                    dst[0] = lo2.x; dst[cog] = lo2.y; dst[2 * cog] = hi2.x; dst[3 * cog] = hi2.y;   // cig is a multiple of 4
-                }
-            }
-        }
+    for (long long i = begin4 + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 wv = ((float4*)w)[i], vv = ((float4*)v)[i];
+        const float4 gv = ((const float4*)g)[i];
+        const float d = i < n_decay4 ? lr * wd : 0.f;
+        sgd_step(wv.x, vv.x, gv.x, d, lr, mu);
+        sgd_step(wv.y, vv.y, gv.y, d, lr, mu);
+        sgd_step(wv.z, vv.z, gv.z, d, lr, mu);
+        sgd_step(wv.w, vv.w, gv.w, d, lr, mu);
+        ((float4*)w)[i] = wv;
+        ((float4*)v)[i] = vv;
+        __nv_bfloat162 lo2 = __floats2bfloat162_rn(wv.x, wv.y), hi2 = __floats2bfloat162_rn(wv.z, wv.w);
+        ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo2, *(uint32_t*)&hi2);
     }
 }
 // The same update for the conv filters, tiled so that the transposed bf16 copies are written in runs: one block = one tap,
 // 32 output channels and 32 input channels of one layer.  Thread (r, c4) updates the four consecutive input channels
 // 4*c4 .. 4*c4+3 of output channel r (the source order [tap][cout][cig]: 128-byte runs per row), the bf16 values cross a
 // shared-memory tile, and thread (ci, q) writes four consecutive output channels of input channel ci to the transposed copy
-// [tap][cin][cog] (64-byte runs) where the one-pass kernel writes single elements.  Bit-identical to sgd_update_kernel.
+// [tap][cin][cog] (64-byte runs; a thread that walked the source order would write single elements).  Same arithmetic as sgd_update_kernel.
 __global__ void __launch_bounds__(256) sgd_update_conv_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g,
                                                               __nv_bfloat16* __restrict__ shadow, float d, float lr, float mu,
                                                               __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs) {
