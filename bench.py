@@ -159,13 +159,29 @@ def run_ours(args, rank, world, local_rank):
         multi.barrier(world)
         torch.cuda.synchronize()
 
+    loss_buf = torch.zeros(2, dtype=torch.float32).pin_memory()
+    loss_ev = [torch.cuda.Event(), torch.cuda.Event()]
+    losses = []
+
     def loop(pool, n, first, want_loss):
-        """n overlapped steps: the load of step i+1 is issued before train_step i."""
+        """n overlapped steps: the load of step i+1 is issued before train_step i.  With want_loss every step's loss is
+        copied to pinned host memory and read by the host: the copy is queued behind the step (alexnet_loss_async) and
+        read one step later, so the host never holds the GPU up."""
         net.load_batch_async(0, *pool[first % N_POOL], first)
         for i in range(first, first + n):
             if i + 1 < first + n:
                 net.load_batch_async(0, *pool[(i + 1) % N_POOL], i + 1)
-            net.train_step(0, want_loss=want_loss)
+            net.train_step(0, want_loss=False)
+            if want_loss:
+                k = (i - first) & 1
+                net.loss_async(0, loss_buf[k:k + 1])
+                loss_ev[k].record(cs)
+                if i > first:
+                    loss_ev[k ^ 1].synchronize()
+                    losses.append(float(loss_buf[k ^ 1]))
+        if want_loss:
+            loss_ev[(n - 1) & 1].synchronize()
+            losses.append(float(loss_buf[(n - 1) & 1]))
 
     def timed(pool, want_loss, first):
         barrier()
@@ -199,8 +215,17 @@ def run_ours(args, rank, world, local_rank):
             if i + 1 < first + n:
                 bi, bl, _ = ld.next()
                 net.load_batch_async(0, bi, bl, i + 1)
-            net.train_step(0, want_loss=True)
-            ld.release()                       # the step has run: the copy out of the oldest held slot is done
+            net.train_step(0, want_loss=False)
+            k = (i - first) & 1
+            net.loss_async(0, loss_buf[k:k + 1])
+            loss_ev[k].record(cs)
+            if i > first:
+                loss_ev[k ^ 1].synchronize()   # step i-1 has run: its loss is on the host and the copy out of its ring slot is done
+                losses.append(float(loss_buf[k ^ 1]))
+                ld.release()
+        loss_ev[(n - 1) & 1].synchronize()
+        losses.append(float(loss_buf[(n - 1) & 1]))
+        ld.release()
 
     loader_loop(3, 0)
     barrier()

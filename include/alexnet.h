@@ -115,6 +115,14 @@ int alexnet_load_batch_async(alexnet_t* h, int replica, const uint8_t* images, c
  * Errors: STATE (no loaded batch), DEVICE_TIMEOUT (latched), CUDA. */
 int alexnet_train_step(alexnet_t* h, int replica, float* host_loss);
 
+/* Queue, on the compute stream, a copy of the mean loss of the replica's most
+ * recent train_step to *loss_out (pinned host memory or device memory, one
+ * float) and return without waiting: the host can read step i's loss while
+ * step i+1 runs.  The value is there once the compute stream has reached this
+ * point (alexnet_sync, or an event the caller records on that stream after
+ * the call); loss_out must stay valid until then.  Errors: ARG, CUDA. */
+int alexnet_loss_async(alexnet_t* h, int replica, float* loss_out);
+
 /* Evaluation of one minibatch, the measurement behind the paper's reported
  * validation errors ("Experiments": top-1 and top-5 error): forward pass only,
  * on the centre 227 x 227 crop without flip, with the dropout masks replaced by

@@ -31,7 +31,7 @@ OPS = ["CONV1_FWD", "CONV2_FWD", "CONV3_FWD", "CONV4_FWD", "CONV5_FWD",
 OP = {n: i for i, n in enumerate(OPS)}
 
 EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "alexnet_destroy",
-           "alexnet_load_batch_async", "alexnet_train_step", "alexnet_replica_average", "alexnet_get_params",
+           "alexnet_load_batch_async", "alexnet_train_step", "alexnet_loss_async", "alexnet_replica_average", "alexnet_get_params",
            "alexnet_set_params", "alexnet_eval_batch", "alexnet_tensor_size", "alexnet_get_tensor", "alexnet_set_tensor", "alexnet_run_op",
            "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error", "alexnet_bias_grad_noalloc", "alexnet_loader_ring_bytes",
            "alexnet_loader_create", "alexnet_loader_next", "alexnet_loader_release", "alexnet_loader_destroy"]
@@ -71,6 +71,7 @@ def load_library():
     L.alexnet_destroy.argtypes = [vp]
     L.alexnet_load_batch_async.argtypes = [vp, i32, vp, vp, u64]
     L.alexnet_train_step.argtypes = [vp, i32, vp]
+    L.alexnet_loss_async.argtypes = [vp, i32, vp]
     L.alexnet_replica_average.argtypes = [vp]
     L.alexnet_eval_batch.argtypes = [vp, i32, vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                                      ctypes.POINTER(ctypes.c_float)]
@@ -170,6 +171,12 @@ class AlexNet:
             return loss.value
         self._ck(self.lib.alexnet_train_step(self.h, replica, None))
         return None
+
+    def loss_async(self, replica, out):
+        """Queue the copy of the last step's mean loss into `out` (one float32, pinned host or device tensor) on the
+        compute stream; the value is there once that stream has reached this point."""
+        self._keep = self._keep[-8:] + [out]
+        self._ck(self.lib.alexnet_loss_async(self.h, replica, _ptr(out)))
 
     def eval_batch(self, replica, images, labels):
         """(top-1 count, top-5 count, mean loss) of one minibatch: forward pass on the centre crop, no dropout mask."""

@@ -1122,6 +1122,14 @@ int alexnet_train_step(alexnet_t* h, int replica, float* host_loss) {
     return ALEXNET_OK;
 }
 
+int alexnet_loss_async(alexnet_t* h, int replica, float* loss_out) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas || !loss_out) return fail(h, ALEXNET_ERR_ARG, "loss_async: bad argument");
+    if (int rc = check_status(h)) return rc;
+    CK(cudaMemcpyAsync(loss_out, h->rep[replica].loss, sizeof(float), cudaMemcpyDefault, h->cs));
+    return ALEXNET_OK;
+}
+
 int alexnet_eval_batch(alexnet_t* h, int replica, const uint8_t* images, const int32_t* labels, int32_t* host_top1,
                        int32_t* host_top5, float* host_loss) {
     if (!h) return ALEXNET_ERR_ARG;

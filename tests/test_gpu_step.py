@@ -345,3 +345,26 @@ def test_fused_fc_update_gives_the_same_parameters():
     assert l0 == l1
     assert np.array_equal(w0, w1) and np.array_equal(v0, v1)
     assert not np.array_equal(w0, w)
+
+
+def test_loss_async_delivers_the_step_loss():
+    """alexnet_loss_async queues the copy of the last step's loss behind the step; after a sync it equals the loss
+    train_step returns when it is asked to wait, and error paths are checked."""
+    from paper_1412_2302_b200 import alexnet as A
+    seed, B = BASE + 9, 4
+    net = make(B, seed=seed)
+    net.set_params(synth.init_params(seed))
+    buf = torch.zeros(1, dtype=torch.float32).pin_memory()
+    load(net, 0, seed, 0, B)
+    blocking = net.train_step(0, want_loss=True)
+    net.loss_async(0, buf)
+    net.sync()
+    assert float(buf[0]) == blocking
+    load(net, 0, seed, 1, B)
+    net.train_step(0, want_loss=False)
+    net.loss_async(0, buf)
+    net.sync()
+    assert np.isfinite(float(buf[0])) and float(buf[0]) != blocking
+    assert net.lib.alexnet_loss_async(net.h, 0, None) == A.ERR_ARG
+    assert net.lib.alexnet_loss_async(net.h, 5, A._ptr(buf)) == A.ERR_ARG
+    net.close()
