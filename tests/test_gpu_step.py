@@ -368,3 +368,26 @@ def test_loss_async_delivers_the_step_loss():
     assert net.lib.alexnet_loss_async(net.h, 0, None) == A.ERR_ARG
     assert net.lib.alexnet_loss_async(net.h, 5, A._ptr(buf)) == A.ERR_ARG
     net.close()
+
+
+def test_multi_stream_step_is_deterministic():
+    """The backward pass forks its independent branches onto streams of their own; the result may not depend on how the
+    kernels interleave: three runs of four steps (fused FC update) give bit-identical parameters and momentum."""
+    from paper_1412_2302_b200 import alexnet as A
+    seed, B = BASE + 10, 16
+    w = synth.init_params(seed)
+    ref = None
+    for _ in range(3):
+        net = make(B, seed=seed, flags=A.FLAG_FUSED_FC_UPDATE)
+        net.set_params(w)
+        for step in range(4):
+            load(net, 0, seed, step, B)
+            net.train_step(0)
+        net.sync()
+        got = (net.get_params(0, 0), net.get_params(0, 1))
+        net.close()
+        if ref is None:
+            ref = got
+        else:
+            assert np.array_equal(ref[0], got[0]) and np.array_equal(ref[1], got[1])
+    assert not np.array_equal(ref[0], w)
