@@ -1,13 +1,17 @@
 /*
  * C ABI of the B200 AlexNet training-step library.
  *
- * The calls follow the paper's statement of the problem: identically
- * initialised model replicas ("Data parallelism": "They are initialized
- * identically"), a loader that brings the next minibatch to the GPU and
- * preprocesses it while the current one trains ("Parallel Data Loading" and
- * its figure), one update per replica on its own minibatch, and the exchange
- * and average of weights, biases and momentum between two replicas ("Data
- * parallelism" and its figure), here with both replicas in one GPU's memory.
+ * The calls follow the paper's statement of the problem: model replicas that
+ * start from the same parameters ("Data parallelism", first paragraph), a
+ * loader that brings the next minibatch to the GPU and preprocesses it while
+ * the current one trains ("Parallel Data Loading" and its figure), one update
+ * per replica on its own minibatch, and the exchange and average of weights,
+ * biases and momentum between replicas ("Data parallelism" and its figure):
+ * with both replicas in one GPU's memory (alexnet_replica_average,
+ * alexnet_update_and_average) or with one replica per GPU and process
+ * (alexnet_param_regions + the caller's all-reduce + alexnet_scale_and_refresh,
+ * or the gradient form alexnet_forward_backward + all-reduce +
+ * alexnet_apply_update).
  *
  * Conventions
  *   - every function returns ALEXNET_OK (0) or a negative error code; nothing
@@ -102,9 +106,9 @@ int alexnet_destroy(alexnet_t* h);
  * consumed returns STATE. */
 int alexnet_load_batch_async(alexnet_t* h, int replica, const uint8_t* images, const int32_t* labels, uint64_t step);
 
-/* One SGD step of `replica` on its oldest loaded batch (paper: "they are
- * updated on different minibatches respectively"): forward, softmax
- * cross-entropy, backward, momentum update
+/* One SGD step of `replica` on its oldest loaded batch (paper, "Data
+ * parallelism": every replica is updated on a minibatch of its own): forward,
+ * softmax cross-entropy, backward, momentum update
  *   v <- momentum*v - lr*weight_decay*w - lr*g ; w <- w + v   (decay on weights only unless flagged).
  * Runs on the compute stream after the batch's load has finished; the
  * independent branches of the backward pass (weight gradients) run on
@@ -142,6 +146,56 @@ int alexnet_eval_batch(alexnet_t* h, int replica, const uint8_t* images, const i
  * one GPU memory: w_a = w_b = (w_a+w_b)/2 and the same for momentum, over all
  * weights and biases.  No-op returning OK when replicas == 1. */
 int alexnet_replica_average(alexnet_t* h);
+
+/* The step in two halves, for callers that combine the gradients or the
+ * parameters of several replicas before or after the update.
+ *
+ * alexnet_forward_backward is alexnet_train_step without the momentum update:
+ * forward, loss, backward on the replica's oldest loaded batch; the gradient of
+ * the mean loss stays in the replica's gradient array (get_params which = 2,
+ * alexnet_param_regions) and is marked pending.  The FC weight gradients are
+ * always stored here, whatever ALEXNET_FLAG_FUSED_FC_UPDATE says.
+ *
+ * alexnet_apply_update applies the update rule of alexnet_train_step to the
+ * pending gradient multiplied by grad_scale (1 for a single replica; 1/R after
+ * the caller has summed the gradients of R replicas into the array): by the
+ * paper's remark that averaging the updated parameters and momenta of
+ * identically starting replicas equals one update on the joint minibatch
+ * ("Data parallelism", last paragraph), this is the gradient form of its
+ * exchange.  Errors: STATE (no pending gradient), ARG, DEVICE_TIMEOUT, CUDA.
+ *
+ * alexnet_update_and_average is steps 1 to 3 of the paper's data-parallel
+ * figure for two replicas in one GPU memory in ONE pass over the parameters:
+ * both pending gradients are applied (each replica's own w, v, g; the same
+ * arithmetic as alexnet_train_step) and w, v of both replicas are replaced by
+ * the averages, 44 bytes of traffic per parameter index instead of 22 + 22 for
+ * two updates and 36 for alexnet_replica_average.  The result is bit-identical
+ * to alexnet_apply_update on both replicas followed by alexnet_replica_average.
+ * Errors: STATE (replicas != 2 or a replica without pending gradient). */
+int alexnet_forward_backward(alexnet_t* h, int replica, float* host_loss);
+int alexnet_apply_update(alexnet_t* h, int replica, float grad_scale);
+int alexnet_update_and_average(alexnet_t* h);
+
+/* One replica per GPU and process: the exchange between GPUs is the caller's
+ * (an all-reduce over NVLink by NCCL, or peer copies); the library exposes what
+ * has to travel and finishes the average.
+ *
+ * alexnet_param_regions returns device pointers to the replica's parameters,
+ * momentum and gradient: three arrays of *n_floats fp32 values each, in the
+ * library's internal order (a fixed permutation of the canonical vector with
+ * zero padding, identical in every process of the same build), owned by the
+ * handle's arena and valid until alexnet_destroy.  Any of the four output
+ * pointers may be NULL.  Work the caller queues on these arrays must be
+ * ordered against the compute stream.
+ *
+ * alexnet_scale_and_refresh multiplies parameters and momentum by `scale`
+ * (1/R after an all-reduce(sum) over R replicas: steps 2 and 3 of the paper's
+ * data-parallel figure) and rebuilds the bf16 copies the tensor-core kernels
+ * read (including the transposed convolution filters); with scale == 1 it only
+ * rebuilds the copies, which is what a caller needs after writing averaged
+ * parameters into the arrays itself.  Asynchronous, on the compute stream. */
+int alexnet_param_regions(alexnet_t* h, int replica, float** dev_w, float** dev_v, float** dev_g, size_t* n_floats);
+int alexnet_scale_and_refresh(alexnet_t* h, int replica, float scale);
 
 /* Read / write a replica's parameters in the canonical order above.
  *   which: 0 = parameters, 1 = momentum, 2 = gradient of the last step (read only)
@@ -191,6 +245,12 @@ enum {
     ALEXNET_OP_POOL1_BWD, ALEXNET_OP_POOL2_BWD, ALEXNET_OP_POOL5_BWD,
     ALEXNET_OP_SOFTMAX, ALEXNET_OP_UPDATE, ALEXNET_OP_AVERAGE, ALEXNET_OP_PREPROCESS,
     ALEXNET_OP_CONV1_BWD_DATA,   /* DA1 -> DX0; not part of the training step (per-layer sweep only) */
+    /* the fused kernels the training step runs for the two LRN layers: A -> P, ARG (normalisation + pooling) and
+     * A, DP, ARG -> DA (pooling gradient + normalisation gradient + ReLU mask) */
+    ALEXNET_OP_LRN1_POOL1_FWD, ALEXNET_OP_LRN2_POOL2_FWD, ALEXNET_OP_POOL1_LRN1_BWD, ALEXNET_OP_POOL2_LRN2_BWD,
+    ALEXNET_OP_UPDATE_AVERAGE,   /* the one-pass update + average of alexnet_update_and_average on whatever the gradient
+                                  * arrays of the two replicas hold */
+    ALEXNET_OP_SCALE_REFRESH,    /* alexnet_scale_and_refresh with scale 1 */
     ALEXNET_OP_COUNT
 };
 int alexnet_run_op(alexnet_t* h, int replica, int op, int iters);
@@ -199,14 +259,16 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters);
 uint64_t alexnet_launch_count(const alexnet_t* h);
 
 /* Optional timing of the tensor-core kernels: while enabled, every launch of
- * one is bracketed by a CUDA event pair on its stream.  profile_read waits for
- * both streams, returns per kernel the summed device time (ms) and the number
- * of launches recorded since the last read, and clears the record.  Index 0 =
- * conv_kernel (convolution forward and backward-data, FC forward), 1 =
- * wgrad_kernel (convolution weight gradients), 2 = gemm_kernel (FC
- * backward-data and weight gradients).  Both arrays have three entries. */
+ * one is bracketed by a CUDA event pair on its stream (and the whole step stays
+ * on the compute stream).  profile_read waits for both streams, returns per
+ * kernel class the summed device time (ms) and the number of launches recorded
+ * since the last read, and clears the record.  Index 0 = conv_kernel on
+ * convolutions (forward and backward-data), 1 = wgrad_kernel (convolution
+ * weight gradients), 2 = gemm_kernel (FC backward-data and weight gradients),
+ * 3 = conv_kernel on the FC forward passes (its 1 x 1 case, HBM-bound at batch
+ * 128).  Both arrays have four entries. */
 int alexnet_profile(alexnet_t* h, int enable);
-int alexnet_profile_read(alexnet_t* h, double* ms3, uint64_t* launches3);
+int alexnet_profile_read(alexnet_t* h, double* ms4, uint64_t* launches4);
 
 /* Bias gradient db[c] = sum over rows of dy[row][c], for callers that cannot
  * allocate device memory when they need it.  (The paper has no counterpart of
@@ -234,7 +296,8 @@ int alexnet_bias_grad_noalloc(const void* dev_dy, int64_t rows, int32_t channels
 
 /* Host half of the paper's loading process ("Parallel Data Loading": a second
  * process loads the next minibatch while the current one trains): a worker
- * pool of `threads` threads (each fills whole batches, in turn) gathers
+ * pool of `threads` threads (every batch is cut into `threads` chunks of
+ * consecutive images, handed out in order) gathers
  * minibatches from a dataset in host memory (for instance a
  * memory-mapped file of uint8 [n][256][256][3] images and int32 labels) into a
  * ring of `depth` staging slots.  Sample j of the stream is dataset entry
@@ -258,6 +321,23 @@ int alexnet_loader_create(const uint8_t* host_images, const int32_t* host_labels
 int alexnet_loader_next(alexnet_loader_t* l, int32_t timeout_ms, const uint8_t** images, const int32_t** labels, uint64_t* batch_index);
 int alexnet_loader_release(alexnet_loader_t* l);
 int alexnet_loader_destroy(alexnet_loader_t* l);
+
+/* Message of the most recent alexnet_create that failed in the calling thread
+ * (there is no handle to ask then); an empty string when none has failed. */
+const char* alexnet_create_error(void);
+
+/* Failure-detection self-test.  Every wait inside the tensor-core kernels is
+ * bounded: when its cycle budget runs out the kernel sets the handle's device
+ * status word, drains and returns, and the host reports DEVICE_TIMEOUT from
+ * then on.  This call launches, on the compute stream, one warp that waits
+ * through the same bounded-wait routine on a barrier that nothing ever arrives
+ * on, with a budget of `budget_cycles` SM clock cycles (clamped to
+ * [1e4, 2e8], i.e. at most about a tenth of a second), so the wait expires by
+ * construction; the GPU context stays usable.  After the next synchronising
+ * call (alexnet_sync, get_params, a train_step that returns its loss) the
+ * handle is latched: every later call returns ALEXNET_ERR_DEVICE_TIMEOUT until
+ * alexnet_destroy, which still succeeds. */
+int alexnet_debug_expire_wait(alexnet_t* h, long long budget_cycles);
 
 /* Wait for both streams; returns a latched DEVICE_TIMEOUT or CUDA error if any. */
 int alexnet_sync(alexnet_t* h);

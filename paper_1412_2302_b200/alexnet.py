@@ -27,14 +27,17 @@ OPS = ["CONV1_FWD", "CONV2_FWD", "CONV3_FWD", "CONV4_FWD", "CONV5_FWD",
        "FC6_FWD", "FC7_FWD", "FC8_FWD", "FC6_BWD_DATA", "FC7_BWD_DATA", "FC8_BWD_DATA",
        "FC6_BWD_WEIGHT", "FC7_BWD_WEIGHT", "FC8_BWD_WEIGHT",
        "LRN1_FWD", "LRN2_FWD", "LRN1_BWD", "LRN2_BWD", "POOL1_FWD", "POOL2_FWD", "POOL5_FWD",
-       "POOL1_BWD", "POOL2_BWD", "POOL5_BWD", "SOFTMAX", "UPDATE", "AVERAGE", "PREPROCESS", "CONV1_BWD_DATA"]
+       "POOL1_BWD", "POOL2_BWD", "POOL5_BWD", "SOFTMAX", "UPDATE", "AVERAGE", "PREPROCESS", "CONV1_BWD_DATA",
+       "LRN1_POOL1_FWD", "LRN2_POOL2_FWD", "POOL1_LRN1_BWD", "POOL2_LRN2_BWD", "UPDATE_AVERAGE", "SCALE_REFRESH"]
 OP = {n: i for i, n in enumerate(OPS)}
 
 EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "alexnet_destroy",
            "alexnet_load_batch_async", "alexnet_train_step", "alexnet_loss_async", "alexnet_replica_average", "alexnet_get_params",
            "alexnet_set_params", "alexnet_eval_batch", "alexnet_tensor_size", "alexnet_get_tensor", "alexnet_set_tensor", "alexnet_run_op",
            "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error", "alexnet_bias_grad_noalloc", "alexnet_loader_ring_bytes",
-           "alexnet_loader_create", "alexnet_loader_next", "alexnet_loader_release", "alexnet_loader_destroy"]
+           "alexnet_loader_create", "alexnet_loader_next", "alexnet_loader_release", "alexnet_loader_destroy",
+           "alexnet_forward_backward", "alexnet_apply_update", "alexnet_update_and_average", "alexnet_param_regions",
+           "alexnet_scale_and_refresh", "alexnet_create_error", "alexnet_debug_expire_wait"]
 
 
 class Config(ctypes.Structure):
@@ -73,6 +76,14 @@ def load_library():
     L.alexnet_train_step.argtypes = [vp, i32, vp]
     L.alexnet_loss_async.argtypes = [vp, i32, vp]
     L.alexnet_replica_average.argtypes = [vp]
+    L.alexnet_forward_backward.argtypes = [vp, i32, vp]
+    L.alexnet_apply_update.argtypes = [vp, i32, ctypes.c_float]
+    L.alexnet_update_and_average.argtypes = [vp]
+    L.alexnet_param_regions.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(sz)]
+    L.alexnet_scale_and_refresh.argtypes = [vp, i32, ctypes.c_float]
+    L.alexnet_create_error.restype = ctypes.c_char_p
+    L.alexnet_create_error.argtypes = []
+    L.alexnet_debug_expire_wait.argtypes = [vp, ctypes.c_longlong]
     L.alexnet_eval_batch.argtypes = [vp, i32, vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                                      ctypes.POINTER(ctypes.c_float)]
     L.alexnet_get_params.argtypes = [vp, i32, i32, vp, sz]
@@ -138,7 +149,7 @@ class AlexNet:
                                      ctypes.c_void_p(self.compute_stream.cuda_stream),
                                      ctypes.c_void_p(self.copy_stream.cuda_stream), ctypes.byref(h))
         if rc != OK:
-            raise AlexNetError(rc, "alexnet_create failed")
+            raise AlexNetError(rc, self.lib.alexnet_create_error().decode() or "alexnet_create failed")
         self.h = h
         self.param_count = int(self.lib.alexnet_param_count())
         self._keep = []
@@ -189,6 +200,39 @@ class AlexNet:
     def replica_average(self):
         self._ck(self.lib.alexnet_replica_average(self.h))
 
+    def forward_backward(self, replica=0, want_loss=False):
+        """train_step without the update: the gradient stays pending (apply_update / update_and_average consume it)."""
+        if want_loss:
+            loss = ctypes.c_float()
+            self._ck(self.lib.alexnet_forward_backward(self.h, replica, ctypes.byref(loss)))
+            return loss.value
+        self._ck(self.lib.alexnet_forward_backward(self.h, replica, None))
+        return None
+
+    def apply_update(self, replica=0, grad_scale=1.0):
+        self._ck(self.lib.alexnet_apply_update(self.h, replica, float(grad_scale)))
+
+    def update_and_average(self):
+        self._ck(self.lib.alexnet_update_and_average(self.h))
+
+    def scale_and_refresh(self, replica=0, scale=1.0):
+        self._ck(self.lib.alexnet_scale_and_refresh(self.h, replica, float(scale)))
+
+    def param_views(self, replica=0):
+        """(w, v, g): fp32 torch views of the replica's parameter, momentum and gradient arrays inside the arena (the
+        library's internal order, zero padded), for collectives between processes; no copy is made."""
+        w, v, g, n = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_size_t()
+        self._ck(self.lib.alexnet_param_regions(self.h, replica, ctypes.byref(w), ctypes.byref(v), ctypes.byref(g), ctypes.byref(n)))
+        base = self.arena.data_ptr()
+        out = []
+        for p in (w, v, g):
+            off = p.value - base
+            out.append(self.arena[off:off + 4 * n.value].view(self._torch.float32))
+        return tuple(out)
+
+    def debug_expire_wait(self, budget_cycles=2_000_000):
+        self._ck(self.lib.alexnet_debug_expire_wait(self.h, int(budget_cycles)))
+
     def sync(self):
         self._ck(self.lib.alexnet_sync(self.h))
 
@@ -221,9 +265,9 @@ class AlexNet:
         self._ck(self.lib.alexnet_profile(self.h, 1 if enable else 0))
 
     def profile_read(self):
-        """Per tensor-core kernel (conv_kernel, wgrad_kernel, gemm_kernel): summed device time in ms and
-        launches since the last read, as two 3-tuples."""
-        ms, n = (ctypes.c_double * 3)(), (ctypes.c_uint64 * 3)()
+        """Per tensor-core kernel class (conv_kernel on convolutions, wgrad_kernel, gemm_kernel, conv_kernel on FC
+        forward): summed device time in ms and launches since the last read, as two 4-tuples."""
+        ms, n = (ctypes.c_double * 4)(), (ctypes.c_uint64 * 4)()
         self._ck(self.lib.alexnet_profile_read(self.h, ms, n))
         return tuple(ms), tuple(int(v) for v in n)
 

@@ -143,6 +143,8 @@ struct Replica {
     bool n_stale[2], dn_stale[2];
     // plans
     Plan conv_fwd[5][2], conv_bwd[5], conv_wg[5][2], fc_fwd[3], fc_bwd[3], fc_wg[3];
+    Plan fc_wg_plain[3];    // the FC weight gradient stored, never fused with the update (alexnet_forward_backward)
+    bool grad_pending;      // forward_backward has left a gradient that no update has consumed yet
 };
 
 }  // namespace
@@ -174,7 +176,8 @@ struct alexnet {
     // optional per-launch timing of the GEMM kernel (event pairs on the launching stream)
     bool prof;
     std::vector<cudaEvent_t> prof_ev;
-    std::vector<int> prof_kind;     // kernel of each recorded pair: 0 conv_kernel, 1 wgrad_kernel, 2 gemm_kernel
+    std::vector<int> prof_kind;     // kernel of each recorded pair: 0 conv_kernel (convolutions), 1 wgrad_kernel, 2 gemm_kernel,
+                                    // 3 conv_kernel (FC forward)
     size_t prof_used;
 };
 
@@ -561,7 +564,8 @@ int plan_fc_bwd(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* w
     finish_plan(h, P);
     return ALEXNET_OK;
 }
-int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x, float* gout, float* w, float* v, bf16* shadow) {
+int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x, float* gout, float* w, float* v, bf16* shadow,
+               bool fuse) {
     memset(&P, 0, sizeof(P));
     tc::GemmParams& p = P.p;
     const int B = h->B;
@@ -575,7 +579,7 @@ int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x,
     if ((rc = make_tm(h, &p.tmB, x, f.K, B, (uint64_t)f.K * 2, 64))) return rc;
     p.tma_store = 1;
     if ((rc = make_tm_out(h, &p.tmOut, gout, true, (uint64_t)f.K, (uint64_t)f.N, 1, (uint64_t)f.K * 4, (uint64_t)f.K * 4 * f.N))) return rc;
-    if (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) {
+    if (fuse) {
         p.fuse_update = 1;
         p.BN = 128; p.n_tiles = f.K / 128;   // narrower tiles leave room for four {w, v} buffers per epilogue warp
         p.upd_lr = h->cfg.lr; p.upd_mu = h->cfg.momentum; p.upd_d = h->cfg.lr * h->cfg.weight_decay;
@@ -611,7 +615,9 @@ int build_plans(alexnet* h, int r) {
         const FcL& f = L.fc[l];
         if ((rc = plan_fc_fwd(h, R.fc_fwd[l], f, fx[l], R.shadow + f.w_off))) return rc;
         if ((rc = plan_fc_bwd(h, R.fc_bwd[l], f, fdy[l], R.shadow + f.w_off))) return rc;
-        if ((rc = plan_fc_wg(h, R.fc_wg[l], f, fdy[l], fx[l], R.g + f.w_off, R.w + f.w_off, R.v + f.w_off, R.shadow + f.w_off))) return rc;
+        const bool fuse = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0;
+        if ((rc = plan_fc_wg(h, R.fc_wg[l], f, fdy[l], fx[l], R.g + f.w_off, R.w + f.w_off, R.v + f.w_off, R.shadow + f.w_off, fuse))) return rc;
+        if ((rc = plan_fc_wg(h, R.fc_wg_plain[l], f, fdy[l], fx[l], R.g + f.w_off, R.w + f.w_off, R.v + f.w_off, R.shadow + f.w_off, false))) return rc;
     }
     return ALEXNET_OK;
 }
@@ -644,7 +650,7 @@ void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
     else launch_k(tc::gemm_kernel, P.grid, tc::kThreads, P.smem, st, P.p);
     if (h->prof) {
         cudaEventRecord(h->prof_ev[h->prof_used + 1], st);
-        h->prof_kind.push_back(P.conv ? 0 : P.wgrad ? 1 : 2);
+        h->prof_kind.push_back(P.conv ? (P.c.kh == 1 && P.c.cpg > 1 ? 3 : 0) : P.wgrad ? 1 : 2);
         h->prof_used += 2;
     }
     h->launches++;
@@ -716,10 +722,10 @@ void op_fc_bwd(alexnet* h, int r, int l, cudaStream_t st) {
                                                            outs[l], db);
     h->launches++;
 }
-void op_fc_wg(alexnet* h, int r, int l, bool with_bias, cudaStream_t st) {
+void op_fc_wg(alexnet* h, int r, int l, bool with_bias, cudaStream_t st, bool plain = false) {
     Replica& R = h->rep[r];
     const FcL& f = h->L.fc[l];
-    launch_gemm(h, R.fc_wg[l], st);
+    launch_gemm(h, plain ? R.fc_wg_plain[l] : R.fc_wg[l], st);
     if (with_bias) {    // in the step only fc8 needs this: fc6 / fc7 get theirs from the data-gradient reduction above them
         const bf16* dyv[3] = {R.df6, R.df7, R.dz};
         colsum(h, dyv[l], h->B, f.N, R.g + f.b_off, st);
@@ -805,7 +811,7 @@ void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
     launch_k(kn::mean_kernel, 1, 256, 0, st, R.loss_n, h->B, R.loss);
     h->launches += 2;
 }
-void op_update(alexnet* h, int r, cudaStream_t st, bool full = false) {
+void op_update(alexnet* h, int r, cudaStream_t st, bool full = false, float gscale = 1.f) {
     Replica& R = h->rep[r];
     const Layout& L = h->L;
     const long long nd = (h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES) ? L.n_total : L.n_weights;
@@ -813,10 +819,28 @@ void op_update(alexnet* h, int r, cudaStream_t st, bool full = false) {
     // kernel of their own; the one-pass kernel takes the rest, minus the FC weights when the fused FC update has done them.
     const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0 && !full;
     launch_k(kn::sgd_update_conv_kernel, L.tjobs.tile0[5], 256, 0, st, R.w, R.v, R.g, R.shadow, h->cfg.lr * h->cfg.weight_decay,
-             h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs);
+             h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs, gscale);
     launch_k(kn::sgd_update_kernel, fused ? 148 : 1184, 256, 0, st, R.w, R.v, R.g, R.shadow, (fused ? L.n_weights : L.fc[0].w_off) / 4,
-             L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum, h->cfg.weight_decay);
+             L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum, h->cfg.weight_decay, gscale);
     h->launches += 2;
+}
+// both replicas: update from each one's own gradient, then average, in one pass; then the transposed conv filters
+void op_update_average(alexnet* h, cudaStream_t st) {
+    Replica &A = h->rep[0], &Bq = h->rep[1];
+    const Layout& L = h->L;
+    const long long nd = (h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES) ? L.n_total : L.n_weights;
+    launch_k(kn::sgd_update_average_kernel, 1184, 256, 0, st, A.w, A.v, A.g, Bq.w, Bq.v, Bq.g, A.shadow, Bq.shadow, L.n_total / 4,
+             nd / 4, h->cfg.lr, h->cfg.momentum, h->cfg.weight_decay);
+    h->launches++;
+    refresh_shadows(h, 0, false, st);
+    refresh_shadows(h, 1, false, st);
+}
+void op_scale_refresh(alexnet* h, int r, float scale, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    if (scale == 1.f) { refresh_shadows(h, r, true, st); return; }
+    launch_k(kn::scale_refresh_kernel, 1184, 256, 0, st, R.w, R.v, R.shadow, h->L.n_total / 4, scale);
+    h->launches++;
+    refresh_shadows(h, r, false, st);
 }
 void op_average(alexnet* h, cudaStream_t st) {
     Replica &A = h->rep[0], &Bq = h->rep[1];
@@ -843,11 +867,10 @@ void forward(alexnet* h, int r, int slot, cudaStream_t st, bool eval) {
     op_fc_fwd(h, r, 0, step, st, eval); op_fc_fwd(h, r, 1, step, st, eval); op_fc_fwd(h, r, 2, step, st, eval);
     op_softmax(h, r, slot, st);
 }
-void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
-    Replica& R = h->rep[r];
+void forward_backward(alexnet* h, int r, int slot, cudaStream_t st, bool plain_fc = false) {
     forward(h, r, slot, st, false);
     // the data gradient reads the layer's weights, so it comes first when the weight-gradient kernel updates them in place
-    const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0;
+    const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0 && !plain_fc;
     // Every independent branch of the backward pass runs on its own stream: with the fused update the weight-gradient kernel
     // of an FC layer (HBM-bound: it streams the layer's weights and momentum) once the layer's data gradient has read the old
     // weights, and the weight gradient of a conv layer (kernel, then split reduction) once the layer's dy exists.  The chain
@@ -866,6 +889,7 @@ void forward_backward(alexnet* h, int r, int slot, cudaStream_t st) {
     };
     for (int l = 2; l >= 0; --l) {
         if (fused) { op_fc_bwd(h, r, l, st); op_fc_wg(h, r, l, l == 2, branch(l)); }
+        else if (plain_fc) { op_fc_wg(h, r, l, l == 2, branch(l), true); op_fc_bwd(h, r, l, st); }
         else { op_fc_wg(h, r, l, l == 2, st); op_fc_bwd(h, r, l, st); }
     }
     op_pool_bwd(h, r, 2, st);
@@ -986,10 +1010,35 @@ inline uint16_t f2bf(float f) {
     return (uint16_t)(u >> 16);
 }
 
+// everything the handle owns: streams, events (null where never created); shared by alexnet_destroy and the failure paths
+// of alexnet_create
+void teardown(alexnet* h) {
+    for (int b = 0; b < alexnet::kBranches; ++b) {
+        if (h->side[b]) { cudaStreamSynchronize(h->side[b]); cudaStreamDestroy(h->side[b]); }
+        if (h->ev_side_done[b]) cudaEventDestroy(h->ev_side_done[b]);
+        if (h->ev_fork[b]) cudaEventDestroy(h->ev_fork[b]);
+    }
+    for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
+    for (int r = 0; r < h->cfg.replicas; ++r)
+        for (int s = 0; s < 2; ++s) {
+            if (h->rep[r].ready[s]) cudaEventDestroy(h->rep[r].ready[s]);
+            if (h->rep[r].consumed[s]) cudaEventDestroy(h->rep[r].consumed[s]);
+        }
+    delete h;
+}
+thread_local std::string g_create_err;
+int create_fail(alexnet* h, int code, const std::string& msg) {
+    g_create_err = msg;
+    if (h) teardown(h);
+    return code;
+}
+
 }  // namespace
 
 // =========================================================================== C ABI
 extern "C" {
+
+const char* alexnet_create_error(void) { return g_create_err.c_str(); }
 
 size_t alexnet_param_count(void) { return (size_t)kCanonCount; }
 
@@ -1002,9 +1051,10 @@ size_t alexnet_workspace_bytes(const alexnet_config_t* cfg) {
 
 int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_bytes, const float* host_mean_image,
                    void* compute_stream, void* copy_stream, alexnet_t** out) {
-    if (!out) return ALEXNET_ERR_ARG;
+    if (!out) return create_fail(nullptr, ALEXNET_ERR_ARG, "alexnet_create: out is NULL");
     *out = nullptr;
-    if (!check_cfg(cfg) || !dev_arena || ((uintptr_t)dev_arena & 1023)) return ALEXNET_ERR_ARG;
+    if (!check_cfg(cfg)) return create_fail(nullptr, ALEXNET_ERR_ARG, "alexnet_create: invalid configuration");
+    if (!dev_arena || ((uintptr_t)dev_arena & 1023)) return create_fail(nullptr, ALEXNET_ERR_ARG, "alexnet_create: arena is NULL or not 1024-byte aligned");
     alexnet* h = new alexnet();
     h->cfg = *cfg; h->B = cfg->batch; h->L = make_layout();
     h->cs = (cudaStream_t)compute_stream; h->ls = (cudaStream_t)copy_stream;
@@ -1012,15 +1062,19 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     h->alpha_eff = (cfg->flags & ALEXNET_FLAG_LRN_ALPHA_DIV_N) ? cfg->lrn_alpha / 5.f : cfg->lrn_alpha;
     h->drop_scale = ((cfg->flags & ALEXNET_FLAG_INVERTED_DROPOUT) && cfg->dropout_p > 0.f) ? 1.f / (1.f - cfg->dropout_p) : 1.f;
     h->thr24 = (uint32_t)floor((double)cfg->dropout_p * 16777216.0);
+    for (int r = 0; r < 2; ++r)
+        for (int s = 0; s < 2; ++s) { h->rep[r].ready[s] = nullptr; h->rep[r].consumed[s] = nullptr; }
+    // nothing is created before the size check: a caller probing arena sizes leaves nothing behind
     const size_t need = carve(h, nullptr);
-    if (arena_bytes < need) { delete h; return ALEXNET_ERR_NOMEM; }
+    if (arena_bytes < need)
+        return create_fail(h, ALEXNET_ERR_NOMEM, "alexnet_create: arena of " + std::to_string(arena_bytes) + " bytes, " + std::to_string(need) + " needed");
     h->arena = (uint8_t*)dev_arena; h->arena_bytes = arena_bytes;
     carve(h, h->arena);
-#define CKC(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { fprintf(stderr, "alexnet_create: %s: %s\n", #call, cudaGetErrorString(e_)); delete h; return ALEXNET_ERR_CUDA; } } while (0)
+#define CKC(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return create_fail(h, ALEXNET_ERR_CUDA, std::string("alexnet_create: ") + #call + ": " + cudaGetErrorString(e_)); } while (0)
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     CKC(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
-    if (!fn || qres != cudaDriverEntryPointSuccess) { delete h; return ALEXNET_ERR_CUDA; }
+    if (!fn || qres != cudaDriverEntryPointSuccess) return create_fail(h, ALEXNET_ERR_CUDA, "alexnet_create: the driver has no cuTensorMapEncodeTiled");
     h->encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
     CKC(cudaFuncSetAttribute(tc::gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::conv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
@@ -1048,6 +1102,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
         Replica& R = h->rep[r];
         R.next_load = R.next_train = R.loaded = R.last_slot = 0;
         R.n_stale[0] = R.n_stale[1] = R.dn_stale[0] = R.dn_stale[1] = false;
+        R.grad_pending = false;
         for (int s = 0; s < 2; ++s) {
             CKC(cudaEventCreateWithFlags(&R.ready[s], cudaEventDisableTiming));
             CKC(cudaEventCreateWithFlags(&R.consumed[s], cudaEventDisableTiming));
@@ -1059,7 +1114,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
         }
         refresh_shadows(h, r, true, h->cs);
         int rc = build_plans(h, r);
-        if (rc) { fprintf(stderr, "alexnet_create: %s\n", h->err.c_str()); delete h; return rc; }
+        if (rc) return create_fail(h, rc, "alexnet_create: " + h->err);
     }
     CKC(cudaStreamSynchronize(h->cs));
     CKC(cudaGetLastError());
@@ -1071,15 +1126,7 @@ int alexnet_destroy(alexnet_t* h) {
     if (!h) return ALEXNET_ERR_ARG;
     cudaStreamSynchronize(h->cs);
     cudaStreamSynchronize(h->ls);
-    for (int b = 0; b < alexnet::kBranches; ++b) {
-        if (h->side[b]) { cudaStreamSynchronize(h->side[b]); cudaStreamDestroy(h->side[b]); }
-        if (h->ev_side_done[b]) cudaEventDestroy(h->ev_side_done[b]);
-        if (h->ev_fork[b]) cudaEventDestroy(h->ev_fork[b]);
-    }
-    for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
-    for (int r = 0; r < h->cfg.replicas; ++r)
-        for (int s = 0; s < 2; ++s) { cudaEventDestroy(h->rep[r].ready[s]); cudaEventDestroy(h->rep[r].consumed[s]); }
-    delete h;
+    teardown(h);
     return ALEXNET_OK;
 }
 
@@ -1100,7 +1147,7 @@ int alexnet_load_batch_async(alexnet_t* h, int replica, const uint8_t* images, c
     return ALEXNET_OK;
 }
 
-int alexnet_train_step(alexnet_t* h, int replica, float* host_loss) {
+static int step_impl(alexnet_t* h, int replica, float* host_loss, bool with_update) {
     if (!h) return ALEXNET_ERR_ARG;
     if (replica < 0 || replica >= h->cfg.replicas) return fail(h, ALEXNET_ERR_ARG, "train_step: bad replica");
     if (int rc = check_status(h)) return rc;
@@ -1108,10 +1155,11 @@ int alexnet_train_step(alexnet_t* h, int replica, float* host_loss) {
     if (R.loaded == 0) return fail(h, ALEXNET_ERR_STATE, "train_step: no loaded batch");
     const int s = R.next_train;
     CK(cudaStreamWaitEvent(h->cs, R.ready[s], 0));
-    forward_backward(h, replica, s, h->cs);
+    forward_backward(h, replica, s, h->cs, !with_update);
     CK(cudaEventRecord(R.consumed[s], h->cs));
     R.consumed_valid[s] = true;
-    op_update(h, replica, h->cs);
+    if (with_update) op_update(h, replica, h->cs);
+    R.grad_pending = !with_update;
     R.last_slot = s; R.next_train ^= 1; R.loaded--;
     CK(cudaGetLastError());
     if (host_loss) {
@@ -1119,6 +1167,64 @@ int alexnet_train_step(alexnet_t* h, int replica, float* host_loss) {
         CK(cudaStreamSynchronize(h->cs));
         return poll_status(h);
     }
+    return ALEXNET_OK;
+}
+
+int alexnet_train_step(alexnet_t* h, int replica, float* host_loss) { return step_impl(h, replica, host_loss, true); }
+int alexnet_forward_backward(alexnet_t* h, int replica, float* host_loss) { return step_impl(h, replica, host_loss, false); }
+
+int alexnet_apply_update(alexnet_t* h, int replica, float grad_scale) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas || !(grad_scale == grad_scale))
+        return fail(h, ALEXNET_ERR_ARG, "apply_update: bad argument");
+    if (int rc = check_status(h)) return rc;
+    Replica& R = h->rep[replica];
+    if (!R.grad_pending) return fail(h, ALEXNET_ERR_STATE, "apply_update: no pending gradient (call alexnet_forward_backward first)");
+    op_update(h, replica, h->cs, true, grad_scale);
+    R.grad_pending = false;
+    CK(cudaGetLastError());
+    return ALEXNET_OK;
+}
+
+int alexnet_update_and_average(alexnet_t* h) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (int rc = check_status(h)) return rc;
+    if (h->cfg.replicas != 2) return fail(h, ALEXNET_ERR_STATE, "update_and_average: needs two replicas");
+    if (!h->rep[0].grad_pending || !h->rep[1].grad_pending)
+        return fail(h, ALEXNET_ERR_STATE, "update_and_average: both replicas need a pending gradient (alexnet_forward_backward)");
+    op_update_average(h, h->cs);
+    h->rep[0].grad_pending = h->rep[1].grad_pending = false;
+    CK(cudaGetLastError());
+    return ALEXNET_OK;
+}
+
+int alexnet_param_regions(alexnet_t* h, int replica, float** dev_w, float** dev_v, float** dev_g, size_t* n_floats) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas) return fail(h, ALEXNET_ERR_ARG, "param_regions: bad replica");
+    Replica& R = h->rep[replica];
+    if (dev_w) *dev_w = R.w;
+    if (dev_v) *dev_v = R.v;
+    if (dev_g) *dev_g = R.g;
+    if (n_floats) *n_floats = (size_t)h->L.n_total;
+    return ALEXNET_OK;
+}
+
+int alexnet_scale_and_refresh(alexnet_t* h, int replica, float scale) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas || !(scale == scale)) return fail(h, ALEXNET_ERR_ARG, "scale_and_refresh: bad argument");
+    if (int rc = check_status(h)) return rc;
+    op_scale_refresh(h, replica, scale, h->cs);
+    CK(cudaGetLastError());
+    return ALEXNET_OK;
+}
+
+int alexnet_debug_expire_wait(alexnet_t* h, long long budget_cycles) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (int rc = check_status(h)) return rc;
+    const long long budget = std::min<long long>(200000000LL, std::max<long long>(10000LL, budget_cycles));
+    launch_k(tc::wait_probe_kernel, 1, 32, 0, h->cs, h->status, budget);
+    h->launches++;
+    CK(cudaGetLastError());
     return ALEXNET_OK;
 }
 
@@ -1292,7 +1398,8 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
     if (!h) return ALEXNET_ERR_ARG;
     if (replica < 0 || replica >= h->cfg.replicas || op < 0 || op >= ALEXNET_OP_COUNT || iters < 1)
         return fail(h, ALEXNET_ERR_ARG, "run_op: bad argument");
-    if (op == ALEXNET_OP_AVERAGE && h->cfg.replicas < 2) return fail(h, ALEXNET_ERR_ARG, "run_op: average needs two replicas");
+    if ((op == ALEXNET_OP_AVERAGE || op == ALEXNET_OP_UPDATE_AVERAGE) && h->cfg.replicas < 2)
+        return fail(h, ALEXNET_ERR_ARG, "run_op: average needs two replicas");
     if (int rc = check_status(h)) return rc;
     Replica& R = h->rep[replica];
     const int slot = R.last_slot;
@@ -1313,6 +1420,10 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
         else if (op == ALEXNET_OP_AVERAGE) op_average(h, st);
         else if (op == ALEXNET_OP_PREPROCESS) op_preprocess(h, replica, slot, R.slot_step[slot], st);
         else if (op == ALEXNET_OP_CONV1_BWD_DATA) op_conv_bwd(h, replica, 0, st);
+        else if (op == ALEXNET_OP_LRN1_POOL1_FWD || op == ALEXNET_OP_LRN2_POOL2_FWD) op_lrn_pool_fwd(h, replica, op - ALEXNET_OP_LRN1_POOL1_FWD, st);
+        else if (op == ALEXNET_OP_POOL1_LRN1_BWD || op == ALEXNET_OP_POOL2_LRN2_BWD) op_pool_lrn_bwd(h, replica, op - ALEXNET_OP_POOL1_LRN1_BWD, st);
+        else if (op == ALEXNET_OP_UPDATE_AVERAGE) op_update_average(h, st);
+        else if (op == ALEXNET_OP_SCALE_REFRESH) op_scale_refresh(h, replica, 1.f, st);
     }
     CK(cudaGetLastError());
     return ALEXNET_OK;
@@ -1330,7 +1441,7 @@ int alexnet_profile_read(alexnet_t* h, double* ms3, uint64_t* launches3) {
     if (!h || !ms3 || !launches3) return ALEXNET_ERR_ARG;
     CK(cudaStreamSynchronize(h->ls));
     CK(cudaStreamSynchronize(h->cs));
-    for (int k = 0; k < 3; ++k) { ms3[k] = 0.0; launches3[k] = 0; }
+    for (int k = 0; k < 4; ++k) { ms3[k] = 0.0; launches3[k] = 0; }
     for (size_t i = 0; i + 1 < h->prof_used; i += 2) {
         float t = 0.f;
         CK(cudaEventElapsedTime(&t, h->prof_ev[i], h->prof_ev[i + 1]));

@@ -679,19 +679,20 @@ __device__ __forceinline__ void sgd_step(float& w, float& v, float g, float d, f
 // v <- mu v - lr wd w [i < n_decay] - lr g ; w <- w + v ; bf16 shadow of w.  22 bytes per parameter.
 // Updates the 16-byte vectors [begin4, n4) of the internal order: everything after the conv filters (which
 // sgd_update_conv_kernel takes), or only the biases when the FC weight-gradient kernel has already updated the FC weights.
+// gscale multiplies the gradient first (1 for a single replica: exact; 1/R for a gradient summed over R replicas).
 __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g,
                                   __nv_bfloat16* __restrict__ shadow, long long begin4, long long n4, long long n_decay4,
-                                  float lr, float mu, float wd) {
+                                  float lr, float mu, float wd, float gscale) {
     pdl_sync();
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long i = begin4 + (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
         float4 wv = ((float4*)w)[i], vv = ((float4*)v)[i];
         const float4 gv = ((const float4*)g)[i];
         const float d = i < n_decay4 ? lr * wd : 0.f;
-        sgd_step(wv.x, vv.x, gv.x, d, lr, mu);
-        sgd_step(wv.y, vv.y, gv.y, d, lr, mu);
-        sgd_step(wv.z, vv.z, gv.z, d, lr, mu);
-        sgd_step(wv.w, vv.w, gv.w, d, lr, mu);
+        sgd_step(wv.x, vv.x, gscale * gv.x, d, lr, mu);
+        sgd_step(wv.y, vv.y, gscale * gv.y, d, lr, mu);
+        sgd_step(wv.z, vv.z, gscale * gv.z, d, lr, mu);
+        sgd_step(wv.w, vv.w, gscale * gv.w, d, lr, mu);
         ((float4*)w)[i] = wv;
         ((float4*)v)[i] = vv;
         __nv_bfloat162 lo2 = __floats2bfloat162_rn(wv.x, wv.y), hi2 = __floats2bfloat162_rn(wv.z, wv.w);
@@ -705,7 +706,7 @@ __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, 
 // [tap][cin][cog] (64-byte runs; a thread that walked the source order would write single elements).  Same arithmetic as sgd_update_kernel.
 __global__ void __launch_bounds__(256) sgd_update_conv_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g,
                                                               __nv_bfloat16* __restrict__ shadow, float d, float lr, float mu,
-                                                              __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs) {
+                                                              __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs, float gscale) {
     pdl_sync();
     __shared__ __nv_bfloat16 tile[32][36];       // [input channel][output channel], padded
     int q = 0;
@@ -722,10 +723,10 @@ __global__ void __launch_bounds__(256) sgd_update_conv_kernel(float* __restrict_
         const long long e = J.src_off + ((long long)tap * J.cout + co) * J.cig + ci;
         float4 wv = *(float4*)(w + e), vv = *(float4*)(v + e);
         const float4 gv = *(const float4*)(g + e);
-        sgd_step(wv.x, vv.x, gv.x, d, lr, mu);
-        sgd_step(wv.y, vv.y, gv.y, d, lr, mu);
-        sgd_step(wv.z, vv.z, gv.z, d, lr, mu);
-        sgd_step(wv.w, vv.w, gv.w, d, lr, mu);
+        sgd_step(wv.x, vv.x, gscale * gv.x, d, lr, mu);
+        sgd_step(wv.y, vv.y, gscale * gv.y, d, lr, mu);
+        sgd_step(wv.z, vv.z, gscale * gv.z, d, lr, mu);
+        sgd_step(wv.w, vv.w, gscale * gv.w, d, lr, mu);
         *(float4*)(w + e) = wv;
         *(float4*)(v + e) = vv;
         const __nv_bfloat162 lo2 = __floats2bfloat162_rn(wv.x, wv.y), hi2 = __floats2bfloat162_rn(wv.z, wv.w);
@@ -757,6 +758,54 @@ __global__ void replica_average_kernel(float* __restrict__ wa, float* __restrict
         __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
         const uint2 s = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
         ((uint2*)sa)[i] = s; ((uint2*)sb)[i] = s;
+    }
+}
+// Momentum update of two replicas and their exchange-and-average in one pass: each replica's own (w, v, g) goes through
+// sgd_step (the update kernels' arithmetic), then w and v of both are replaced by 0.5 * (a + b) (replica_average_kernel's
+// arithmetic) and both bf16 copies are written: six 16-byte loads and six stores per four parameter indices, 44 bytes per
+// index, against 22 + 22 + 36 for the three separate passes, with bit-identical results.
+__device__ __forceinline__ float4 ld_stream(const float* p) {       // read once, do not keep in L1
+    float4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(p));
+    return r;
+}
+__global__ void __launch_bounds__(256) sgd_update_average_kernel(float* __restrict__ wa, float* __restrict__ va, const float* __restrict__ ga,
+                                                                 float* __restrict__ wb, float* __restrict__ vb, const float* __restrict__ gb,
+                                                                 __nv_bfloat16* __restrict__ sa, __nv_bfloat16* __restrict__ sb,
+                                                                 long long n4, long long n_decay4, float lr, float mu, float wd) {
+    pdl_sync();
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 a = ((const float4*)wa)[i], c = ((const float4*)va)[i];
+        float4 b = ((const float4*)wb)[i], e = ((const float4*)vb)[i];
+        const float4 g0 = ld_stream(ga + 4 * i), g1 = ld_stream(gb + 4 * i);
+        const float d = i < n_decay4 ? lr * wd : 0.f;
+        sgd_step(a.x, c.x, g0.x, d, lr, mu); sgd_step(a.y, c.y, g0.y, d, lr, mu);
+        sgd_step(a.z, c.z, g0.z, d, lr, mu); sgd_step(a.w, c.w, g0.w, d, lr, mu);
+        sgd_step(b.x, e.x, g1.x, d, lr, mu); sgd_step(b.y, e.y, g1.y, d, lr, mu);
+        sgd_step(b.z, e.z, g1.z, d, lr, mu); sgd_step(b.w, e.w, g1.w, d, lr, mu);
+        const float4 w = make_float4(0.5f * (a.x + b.x), 0.5f * (a.y + b.y), 0.5f * (a.z + b.z), 0.5f * (a.w + b.w));
+        const float4 v = make_float4(0.5f * (c.x + e.x), 0.5f * (c.y + e.y), 0.5f * (c.z + e.z), 0.5f * (c.w + e.w));
+        ((float4*)wa)[i] = w; ((float4*)wb)[i] = w;
+        ((float4*)va)[i] = v; ((float4*)vb)[i] = v;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(w.x, w.y), hi = __floats2bfloat162_rn(w.z, w.w);
+        const uint2 s = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
+        ((uint2*)sa)[i] = s; ((uint2*)sb)[i] = s;
+    }
+}
+// After an all-reduce(sum) of parameters and momentum over R replicas on R GPUs: w <- scale w, v <- scale v (scale = 1/R:
+// the average) and the bf16 copy of w: 8 bytes read and 10 written per index.
+__global__ void __launch_bounds__(256) scale_refresh_kernel(float* __restrict__ w, float* __restrict__ v,
+                                                            __nv_bfloat16* __restrict__ shadow, long long n4, float scale) {
+    pdl_sync();
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 a = ((const float4*)w)[i], c = ((const float4*)v)[i];
+        a.x *= scale; a.y *= scale; a.z *= scale; a.w *= scale;
+        c.x *= scale; c.y *= scale; c.z *= scale; c.w *= scale;
+        ((float4*)w)[i] = a; ((float4*)v)[i] = c;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+        ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
     }
 }
 __global__ void shadow_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ shadow, long long n4) {

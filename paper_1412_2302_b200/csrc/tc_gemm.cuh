@@ -110,7 +110,7 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // bounded wait: returns false when the cycle budget ran out or another role aborted.  It polls with the
 // non-blocking test_wait first: a thread suspended inside try_wait was seen to resume late, which starves the
 // producer / issuer hand-over of a pipelined ring; only a long wait falls back to the suspending form.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_budget(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget) {
     #pragma unroll 1
     for (int i = 0; i < 4096; ++i)
         if (mbar_test_wait(bar, parity)) return true;
@@ -120,12 +120,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitBudgetCycles) { *abort_flag = 1; return false; }
+        if (clock64() - t0 > budget) { *abort_flag = 1; return false; }
     }
 }
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    return mbar_wait_budget(bar, parity, abort_flag, kWaitBudgetCycles);
+}
 // the same for a whole warp that must take one decision (all lanes wait; any failure fails all)
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                               long long budget = kWaitBudgetCycles) {
+    return __all_sync(0xffffffffu, mbar_wait_budget(bar, parity, abort_flag, budget));
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y, uint32_t bar) {
     asm volatile(
@@ -385,6 +389,22 @@ __device__ __forceinline__ void epi_slab(const P& p, uint32_t tmem_addr, bool pa
     fence_async_smem();
     __syncwarp();
     if (lane == 0) { tma_store_3d(&p.tmOut, stage, x, y, z); bulk_commit(); }
+}
+
+// Failure-detection self-test: one warp waits, through the bounded wait above, on a barrier nothing arrives on.  The
+// wait runs out after `budget` cycles, the warp raises the status word as the GEMM kernels do, and returns.
+__global__ void __launch_bounds__(32) wait_probe_kernel(int* status, long long budget) {
+    kn::pdl_sync();
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    const bool ok = mbar_wait_warp(smem_u32(&bar), 0u, &abort_flag, budget);
+    if (!ok && threadIdx.x == 0 && status) atomicExch(status, 1);
 }
 
 constexpr int kABytes = 128 * 128;  // 128 rows x 64 bf16, or 2 boxes of 64 x 64
@@ -1201,6 +1221,10 @@ __global__ void __launch_bounds__(32 * 7, 1) wgrad_kernel(const __grid_constant_
                     #pragma unroll
                     for (int k = 0; k < 4; ++k) { const float2 f = __bfloat1622float2(hh[k]); acc[2 * k] += f.x; acc[2 * k + 1] += f.y; }
                 }
+                // these were generic-proxy reads of a stage that TMA (the async proxy) overwrites once it is released: without
+                // a proxy fence between the reads and the release the refill may overtake reads still in flight (seen as a
+                // wrong bias partial in a few per cent of the steps, only when other kernels shared the GPU)
+                fence_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty0 + 8u * st);
                 if (++st == stages) { st = 0; ph ^= 1u; }

@@ -42,6 +42,11 @@ def hbm_bytes(B):
         "SOFTMAX": B * 1000 * 6,
         "UPDATE": PARAMS * 22,                                      # r w,v,g; w w,v fp32 + bf16 copy
         "AVERAGE": PARAMS * (32 + 4),                               # r/w w,v of both replicas + both bf16 copies
+        # the fused kernels the training step runs: a read, p + argmax written; a, dp, argmax read, da written
+        "LRN1_POOL1_FWD": B * (a1 * 2 + p1 * 3), "LRN2_POOL2_FWD": B * (a2 * 2 + p2 * 3),
+        "POOL1_LRN1_BWD": B * (a1 * 4 + p1 * 3), "POOL2_LRN2_BWD": B * (a2 * 4 + p2 * 3),
+        "UPDATE_AVERAGE": PARAMS * 44,                              # r w,v,g of both replicas; w w,v and bf16 copy of both
+        "SCALE_REFRESH": PARAMS * 6,                                # scale 1: r w, w bf16 copy
     }
     return d
 

@@ -12,7 +12,6 @@ from paper_1412_2302_b200 import synth
 pytestmark = pytest.mark.gpu
 
 SEED = synth.BASE_SEED + 5
-B = 3          # ragged: no grid is a multiple of the 128-row tile
 TOL = 2e-2
 
 
@@ -25,12 +24,16 @@ def rel(a, b):
     return np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30)
 
 
-# every operation runs three times: tile shapes from the cost model, convolutions on single CTAs only, and
-# convolutions on CTA pairs (cta_group::2) only
-@pytest.fixture(scope="module", params=[0, 16, 32], ids=["auto", "single-cta", "cta-pairs"])
+# every operation runs at batch 3 (ragged: no grid is a multiple of the 128-row tile, one or two tiles per kernel, split
+# counts at their maximum) three times: tile shapes from the cost model, convolutions on single CTAs only, and
+# convolutions on CTA pairs (cta_group::2) only; and once more at batch 40, where the persistent kernels walk several
+# rounds of their tile lists with a partial last round (conv1: 1016 row tiles, conv2: 263 per group, conv3-5: 62 with a
+# ragged last one) and the split counts follow from the batch
+@pytest.fixture(scope="module", params=[(0, 3), (16, 3), (32, 3), (0, 40)], ids=["auto", "single-cta", "cta-pairs", "auto-batch40"])
 def net(request):
     from paper_1412_2302_b200.alexnet import AlexNet
-    n = AlexNet(batch=B, replicas=2, seed=SEED, mean_image=synth.mean_image(SEED), flags=request.param)
+    flags, batch = request.param
+    n = AlexNet(batch=batch, replicas=2, seed=SEED, mean_image=synth.mean_image(SEED), flags=flags)
     yield n
     n.close()
 
@@ -50,6 +53,7 @@ CONVS = [("conv1", "X0", "A1", (3, 227, 227)), ("conv2", "P1", "A2", (96, 27, 27
 
 @pytest.mark.parametrize("name,tin,tout,shp", CONVS)
 def test_conv_forward(net, params, name, tin, tout, shp):
+    B = net.batch
     x = synth.bf16_grid(SEED, tag(name), (B,) + shp, -1, 1)
     if name == "conv1":
         x = x * 4
@@ -71,6 +75,7 @@ BWD = [("conv1", "DA1", "DX0", None, (3, 227, 227)), ("conv2", "DA2", "DP1", Non
 
 @pytest.mark.parametrize("name,tdy,tdx,tmask,shp", BWD)
 def test_conv_backward_data(net, params, name, tdy, tdx, tmask, shp):
+    B = net.batch
     c = O.CONV[name]
     ho = 55 if name == "conv1" else shp[1]
     dy = synth.bf16_grid(SEED, 7 + tag(name), (B, c["cout"], ho, ho), -1, 1)
@@ -93,6 +98,7 @@ WG = [("conv1", "X0", "DA1", (3, 227, 227), 55), ("conv2", "P1", "DA2", (96, 27,
 
 @pytest.mark.parametrize("name,tin,tdy,shp,ho", WG)
 def test_conv_backward_weight_and_bias(net, params, name, tin, tdy, shp, ho):
+    B = net.batch
     c = O.CONV[name]
     x = synth.bf16_grid(SEED, 21 + tag(name), (B,) + shp, -1, 1)
     dy = synth.bf16_grid(SEED, 22 + tag(name), (B, c["cout"], ho, ho), -1, 1)
@@ -114,6 +120,7 @@ FCS = [("fc6", "P5", "F6", "M6", 2), ("fc7", "F6", "F7", "M7", 3), ("fc8", "F7",
 
 @pytest.mark.parametrize("name,tin,tout,tm,stream", FCS)
 def test_fc_forward_with_dropout(net, params, name, tin, tout, tm, stream):
+    B = net.batch
     K, N = O.FC[name]
     x = synth.bf16_grid(SEED, 31 + tag(name), (B, K), -1, 1)
     xin = x.reshape(B, 256, 6, 6) if name == "fc6" else x
@@ -134,6 +141,7 @@ FCB = [("fc6", "DF6", "DP5", None), ("fc7", "DF7", "DF6", "F6"), ("fc8", "DZ", "
 
 @pytest.mark.parametrize("name,tdy,tdx,tmask", FCB)
 def test_fc_backward_data(net, params, name, tdy, tdx, tmask):
+    B = net.batch
     K, N = O.FC[name]
     dy = synth.bf16_grid(SEED, 41 + tag(name), (B, N), -1, 1)
     net.set_tensor(tdy, dy)
@@ -155,6 +163,7 @@ FCW = [("fc6", "P5", "DF6"), ("fc7", "F6", "DF7"), ("fc8", "F7", "DZ")]
 
 @pytest.mark.parametrize("name,tin,tdy", FCW)
 def test_fc_backward_weight_and_bias(net, params, name, tin, tdy):
+    B = net.batch
     K, N = O.FC[name]
     x = synth.bf16_grid(SEED, 51 + tag(name), (B, K), -1, 1)
     dy = synth.bf16_grid(SEED, 52 + tag(name), (B, N), -1, 1)
@@ -173,6 +182,7 @@ def test_fc_backward_weight_and_bias(net, params, name, tin, tdy):
 
 @pytest.mark.parametrize("which,ta,tn,tdn,tda,shp", [(1, "A1", "N1", "DN1", "DA1", (96, 55, 55)), (2, "A2", "N2", "DN2", "DA2", (256, 27, 27))])
 def test_lrn_forward_backward(net, which, ta, tn, tdn, tda, shp):
+    B = net.batch
     a = np.maximum(synth.bf16_grid(SEED, 60 + which, (B,) + shp, -1, 1) * 64, 0)   # post-ReLU range up to 64
     g = synth.bf16_grid(SEED, 62 + which, (B,) + shp, -1, 1)
     net.set_tensor(ta, a)
@@ -191,6 +201,7 @@ POOLS = [(1, "N1", "P1", "ARG1", "DP1", "DN1", None, (96, 55, 55)), (2, "N2", "P
 
 @pytest.mark.parametrize("which,tx,ty,targ,tdy,tdx,trelu,shp", POOLS)
 def test_pool_forward_backward(net, which, tx, ty, targ, tdy, tdx, trelu, shp):
+    B = net.batch
     x = np.maximum(synth.bf16_grid(SEED, 70 + which, (B,) + shp, -1, 1), 0)   # many exact ties at 0 and on the grid
     net.set_tensor(tx, x)
     net.run_op(f"POOL{which}_FWD")
@@ -208,7 +219,70 @@ def test_pool_forward_backward(net, which, tx, ty, targ, tdy, tdx, trelu, shp):
     assert rel(net.get_tensor(tdx), ref) < 4e-3
 
 
+def tie_heavy(seed, tag, shape, block=3, scale=8.0):
+    """Post-ReLU activations full of exact ties: piecewise constant over block x block pixels (so that the pixels of a
+    pooling window often hold identical channel vectors, whose normalised values are then identical bit for bit), about
+    half of the blocks zero."""
+    Bn, C, H, W = shape
+    hb, wb = (H + block - 1) // block, (W + block - 1) // block
+    coarse = np.maximum(synth.bf16_grid(seed, tag, (Bn, C, hb, wb), -1, 1) * scale, 0)
+    return np.repeat(np.repeat(coarse, block, axis=2), block, axis=3)[:, :, :H, :W].copy()
+
+
+FUSED = [(1, "A1", "N1", "P1", "ARG1", "DP1", "DA1", (96, 55, 55)), (2, "A2", "N2", "P2", "ARG2", "DP2", "DA2", (256, 27, 27))]
+
+
+@pytest.mark.parametrize("which,ta,tn,tp,targ,tdp,tda,shp", FUSED)
+@pytest.mark.parametrize("block", [3, 2, 1])
+def test_fused_lrn_pool_forward_argmax_bit_exact(net, which, ta, tn, tp, targ, tdp, tda, shp, block):
+    """The kernel the training step runs for LRN + pooling (integer-key maximum).  The normalised tensor it pools is the
+    one the single-operation LRN kernel writes (same device function), so pooling THAT tensor with the oracle gives the
+    exact expectation: values and argmax codes bit for bit, on inputs where most windows hold exact ties (zeros and
+    repeated non-zero values), so that any tie rule but first-maximum-in-scan-order fails."""
+    B = net.batch
+    a = tie_heavy(SEED, 90 + which + 10 * block, (B,) + shp, block)
+    net.set_tensor(ta, a)
+    net.run_op(f"LRN{which}_FWD")
+    net.sync()
+    n_gpu = net.get_tensor(tn).reshape((B,) + shp)
+    assert rel(n_gpu, O.lrn_fwd(a)) < 4e-3
+    y, arg = O.pool_fwd(n_gpu.astype(np.float64))
+    # the input must really exercise the tie rule: in many windows the maximum occurs more than once
+    cnt = sum((n_gpu[:, :, ky:ky + 2 * y.shape[2] - 1:2, kx:kx + 2 * y.shape[3] - 1:2] == y).astype(np.int32)
+              for ky in range(3) for kx in range(3))
+    assert (cnt >= 2).mean() > (0.3 if block > 1 else 0.01)
+    net.set_tensor(tp, np.full(y.shape, -1.0, np.float32))
+    net.set_tensor(targ, np.full(arg.shape, 9, np.float32))
+    net.run_op(f"LRN{which}_POOL{which}_FWD")
+    net.sync()
+    assert np.array_equal(net.get_tensor(tp).reshape(y.shape), y.astype(np.float32))
+    assert np.array_equal(net.get_tensor(targ).reshape(arg.shape).astype(np.uint8), arg)     # bit exact
+
+
+@pytest.mark.parametrize("which,ta,tn,tp,targ,tdp,tda,shp", FUSED)
+def test_fused_pool_lrn_backward(net, which, ta, tn, tp, targ, tdp, tda, shp):
+    """The fused backward kernel of the step (pooling gradient scattered in shared memory, LRN gradient, ReLU mask)
+    against the oracle's pool_bwd followed by lrn_bwd, with argmax codes that send several windows to one pixel."""
+    B = net.batch
+    a = tie_heavy(SEED, 95 + which, (B,) + shp, 2)
+    y, arg = O.pool_fwd(O.lrn_fwd(a))
+    rng = np.random.default_rng(17 + which)
+    arg = np.where(rng.random(arg.shape) < 0.5, arg, rng.integers(0, 9, size=arg.shape)).astype(np.uint8)   # any valid code
+    dp = synth.bf16_grid(SEED, 97 + which, y.shape, -1, 1)
+    net.set_tensor(ta, a)
+    net.set_tensor(targ, arg.astype(np.float32))
+    net.set_tensor(tdp, dp)
+    net.run_op(f"POOL{which}_LRN{which}_BWD")
+    net.sync()
+    dn = O.round_bf16(O.pool_bwd(dp, arg, a.shape))          # the kernel rounds the pooled gradient to bf16, as the unfused path stores it
+    ref = O.lrn_bwd(a, dn) * (a > 0)
+    got = net.get_tensor(tda).reshape(ref.shape)
+    assert rel(got, ref) < 4e-3, rel(got, ref)
+    assert (got[a <= 0] == 0).all()
+
+
 def test_softmax_xent(net):
+    B = net.batch
     z = synth.normal(SEED, 80, (B, 1000), 3.0)
     lab = synth.labels(SEED, 0, 0, B)
     img = synth.images(SEED, 0, 0, B)
@@ -228,6 +302,7 @@ def test_softmax_xent(net):
 
 
 def test_preprocess_crop_flip_bit_exact(net):
+    B = net.batch
     import torch
     for step in (5, 6):
         img = synth.images(SEED, 1, step, B)
@@ -244,6 +319,7 @@ def test_preprocess_crop_flip_bit_exact(net):
 
 
 def test_update_and_average_fp32(net):
+    B = net.batch
     rng = np.random.default_rng(3)
     n = net.param_count
     w0 = rng.standard_normal(n).astype(np.float32) * 0.05
