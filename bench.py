@@ -53,6 +53,8 @@ KERNEL_FLOP = (1.3315e9 + 1.1207e9, 1.3315e9, 0.2346e9, 0.1173e9)
 # batch-128 training step (one ncu capture of this build's kernel; the summary is kept with the other profiles)
 NCU_DRAM_BYTES_PER_CONV_LAUNCH = 32.7e6
 N_POOL = 4                          # distinct synthetic batches cycled through
+CONV_OPS = ("CONV1_FWD", "CONV2_FWD", "CONV3_FWD", "CONV4_FWD", "CONV5_FWD", "CONV2_BWD_DATA", "CONV3_BWD_DATA", "CONV4_BWD_DATA",
+            "CONV5_BWD_DATA")
 
 
 def peaks():
@@ -270,29 +272,33 @@ def run_ours(args, rank, world, local_rank):
             net.train_step(0, want_loss=False)
             exchange.exchange_and_average(rep)
 
-    loss_buf = torch.zeros(2, dtype=torch.float32).pin_memory()
-    loss_ev = [torch.cuda.Event(), torch.cuda.Event()]
+    LAG = 3                         # the host reads the loss of step i - LAG while it queues step i
+    loss_buf = torch.zeros(LAG + 1, dtype=torch.float32).pin_memory()
+    loss_ev = [torch.cuda.Event() for _ in range(LAG + 1)]
     losses = []
+
+    def read_loss(j):
+        loss_ev[j % (LAG + 1)].synchronize()
+        losses.append(float(loss_buf[j % (LAG + 1)]))
 
     def loop(pool, n, first, want_loss):
         """n overlapped steps: the load of step i+1 is issued before step i.  With want_loss every step's loss is
         copied to pinned host memory and read by the host: the copy is queued behind the step (alexnet_loss_async) and
-        read one step later, so the host never holds the GPU up."""
+        read LAG steps later, so the host never holds the GPU up; all n losses have been read when the loop returns."""
         net.load_batch_async(0, *pool[first % N_POOL], first)
         for i in range(first, first + n):
             if i + 1 < first + n:
                 net.load_batch_async(0, *pool[(i + 1) % N_POOL], i + 1)
             step()
             if want_loss:
-                k = (i - first) & 1
+                k = (i - first) % (LAG + 1)
                 net.loss_async(0, loss_buf[k:k + 1])
                 loss_ev[k].record(cs)
-                if i > first:
-                    loss_ev[k ^ 1].synchronize()
-                    losses.append(float(loss_buf[k ^ 1]))
+                if i - first >= LAG:
+                    read_loss(i - first - LAG)
         if want_loss:
-            loss_ev[(n - 1) & 1].synchronize()
-            losses.append(float(loss_buf[(n - 1) & 1]))
+            for j in range(max(0, n - LAG), n):
+                read_loss(j)
 
     def timed(body):
         barrier()
@@ -334,15 +340,13 @@ def run_ours(args, rank, world, local_rank):
                 bi, bl, _ = ld.next()
                 net.load_batch_async(0, bi, bl, i + 1)
             step()
-            k = (i - first) & 1
+            k = (i - first) % (LAG + 1)
             net.loss_async(0, loss_buf[k:k + 1])
             loss_ev[k].record(cs)
             if i > first:
-                loss_ev[k ^ 1].synchronize()   # step i-1 has run: its loss is on the host and the copy out of its ring slot is done
-                losses.append(float(loss_buf[k ^ 1]))
+                read_loss(i - first - 1)       # step i-1 has run: its loss is on the host and the copy out of its ring slot is done
                 ld.release()
-        loss_ev[(n - 1) & 1].synchronize()
-        losses.append(float(loss_buf[(n - 1) & 1]))
+        read_loss(n - 1)
         ld.release()
 
     loader_loop(3, 0)
@@ -369,6 +373,20 @@ def run_ours(args, rank, world, local_rank):
     k_ms, k_n = net.profile_read()
     net.profile(False)
     net.sync()
+    # the nine convolution launches again, each as bursts of eight back-to-back launches between two events: inside the
+    # overlapped step a launch's set-up runs under its predecessor's tail (programmatic dependent launch), which the event
+    # pairs of the pass above prevent; this is the steady-state duration of a launch
+    b2b_ms = 0.0
+    with torch.cuda.stream(cs):
+        for name in CONV_OPS:
+            net.run_op(name, iters=3)
+            ts = []
+            for _ in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(cs); net.run_op(name, iters=8); e1.record(cs)
+                ts.append((e0, e1))
+            net.sync()
+            b2b_ms += sorted(a.elapsed_time(b) for a, b in ts)[2] / 8
     net.close()
 
     if rank == 0:
@@ -417,6 +435,10 @@ def run_ours(args, rank, world, local_rank):
                          "ms_x_mhz_per_step": per_kernel["conv_kernel"]["ms_per_step"] * mhz if mhz else None,
                          "launches_per_step": per_kernel["conv_kernel"]["launches_per_step"],
                          "ms_per_step": per_kernel["conv_kernel"]["ms_per_step"], "all_tensor_kernels": per_kernel,
+                         "back_to_back": {"ms_per_step": b2b_ms, "achieved": KERNEL_FLOP[0] * BATCH / (b2b_ms * 1e-3) / 1e12,
+                                          "frac_of_burst": KERNEL_FLOP[0] * BATCH / (b2b_ms * 1e-3) / 1e12 / tf_burst,
+                                          "note": "the same nine launches, each timed as 8 back-to-back launches between two CUDA "
+                                                  "events: a launch's set-up overlaps its predecessor's tail, as inside the step"},
                          "whole_step": {"tflops": FLOP_PER_IMAGE * BATCH / (ms / K * 1e-3) / 1e12,
                                         "frac_of_burst": FLOP_PER_IMAGE * BATCH / (ms / K * 1e-3) / 1e12 / tf_burst}},
         }

@@ -108,14 +108,40 @@ def dropout_mask(seed, layer_stream, replica, step, B, width, p) -> np.ndarray:
 # ----------------------------------------------------------- layer functions
 
 
-def preprocess(img_u8, mean, cf) -> np.ndarray:
-    """img_u8 (B,256,256,3) uint8, mean (256,256,3), cf (B,3) -> X (B,3,227,227) fp64."""
+def preprocess(img_u8, mean, cf, shift=None) -> np.ndarray:
+    """img_u8 (B,256,256,3) uint8, mean (256,256,3), cf (B,3) -> X (B,3,227,227) fp64.
+    shift (B,3), optional: one RGB offset per image, added to every pixel (color_shift below)."""
     img_u8 = np.ascontiguousarray(img_u8, np.uint8)
     B = img_u8.shape[0]
     X = np.empty((B, 3, 227, 227), np.float64)
     cf = np.ascontiguousarray(cf, np.int32)
     lib().orc_preprocess(_p(img_u8), _p(_f64(mean)), _p(cf), I(B), _p(X))
+    if shift is not None:
+        X += np.asarray(shift, np.float64)[:, :, None, None]
     return X
+
+
+def normal_draws(seed, stream, replica, step, count) -> np.ndarray:
+    """count standard-normal draws from the counter hash: draw r(idx) gives u1 = (top 24 bits + 1) / 2^24 in (0, 1] and
+    u2 = (bits 16..39) / 2^24 in [0, 1); z = sqrt(-2 ln u1) cos(2 pi u2) (Box-Muller, first variate)."""
+    key = stream_key(seed, stream, replica, step)
+    z = np.empty(count, np.float64)
+    for i in range(count):
+        r = draw(key, i)
+        u1 = ((r >> 40) + 1) / 16777216.0
+        u2 = ((r >> 16) & 0xFFFFFF) / 16777216.0
+        z[i] = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+    return z
+
+
+def color_shift(seed, replica, step, B, eigvec, eigval, sigma) -> np.ndarray:
+    """The intensity augmentation of Krizhevsky et al. 2012 (section 4.1), which the paper's experiments leave out
+    ("Experiments", the sentence on the reported error rates): to every pixel of image n add
+    eigvec @ (alpha_n * eigval), where eigvec (3,3: columns are the principal components of the RGB pixel values of
+    the training set) and eigval (3,) are dataset constants and alpha_n (3,) ~ N(0, sigma^2) is drawn once per image
+    (hash stream 10, index 3 n + i).  Returns (B,3) offsets; sigma = 0 gives zeros."""
+    alpha = sigma * normal_draws(seed, 10, replica, step, 3 * B).reshape(B, 3)
+    return (alpha * np.asarray(eigval, np.float64)[None, :]) @ np.asarray(eigvec, np.float64).T
 
 
 def conv_fwd(x, w, b, stride, pad, groups):
@@ -305,6 +331,7 @@ class OracleConfig:
     wd_on_biases: bool = False
     inverted_dropout: bool = False
     bf16_aware: bool = False  # diagnostic: round where the GPU stores bf16
+    color: tuple = None       # (eigvec (3,3), eigval (3,), sigma): intensity augmentation in training passes; None = off
 
 
 @dataclass
@@ -349,7 +376,8 @@ class OracleNet:
         B = img_u8.shape[0]
         T = {}
         T["cf"] = crop_flip(c.seed, self.replica, step, B) if cf is None else np.asarray(cf, np.int32)
-        T["x0"] = q(preprocess(img_u8, mean, T["cf"]))
+        shift = color_shift(c.seed, self.replica, step, B, *c.color) if c.color else None
+        T["x0"] = q(preprocess(img_u8, mean, T["cf"], shift))
         la = self._lrn_args()
 
         def conv_block(name, x):

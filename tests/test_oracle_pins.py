@@ -364,3 +364,58 @@ def test_round_bf16():
     assert (O.round_bf16(x) == t).all()
     r = rng.standard_normal(1000) * 100
     assert (O.round_bf16(r) == torch.tensor(r, dtype=torch.float32).to(torch.bfloat16).to(torch.float64).numpy()).all()
+
+
+# ---------------------------------------------------------------- intensity augmentation (the one the paper skips)
+def test_normal_draws_are_standard_normal_and_reproducible():
+    z = O.normal_draws(7, 10, 0, 3, 60000)
+    assert np.array_equal(z, O.normal_draws(7, 10, 0, 3, 60000))
+    assert not np.array_equal(z[:100], O.normal_draws(7, 10, 1, 3, 100))            # another replica, other draws
+    # moments of N(0,1) within sampling error (60000 draws: standard errors 0.004, 0.006, 0.01, 0.02)
+    assert abs(z.mean()) < 0.02 and abs(z.var() - 1.0) < 0.03
+    assert abs((z ** 3).mean()) < 0.05 and abs((z ** 4).mean() - 3.0) < 0.12
+    # quantiles against the normal distribution function
+    from math import erf, sqrt
+    for x in (-2.0, -1.0, -0.25, 0.5, 1.5):
+        assert abs((z < x).mean() - 0.5 * (1.0 + erf(x / sqrt(2.0)))) < 0.008
+    # Box-Muller from the published hash: the first draw by hand
+    r = O.draw(O.stream_key(7, 10, 0, 3), 0)
+    u1, u2 = ((r >> 40) + 1) / 2.0 ** 24, ((r >> 16) & 0xFFFFFF) / 2.0 ** 24
+    assert 0.0 < u1 <= 1.0 and 0.0 <= u2 < 1.0
+    assert z[0] == np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2)
+
+
+def test_color_shift_special_cases():
+    B = 64
+    ident, ones = np.eye(3), np.ones(3)
+    a = O.color_shift(5, 0, 2, B, ident, ones, 0.1)
+    assert a.shape == (B, 3)
+    # identity components, unit eigenvalues: the offsets are the draws themselves, image n using draws 3n..3n+2
+    assert np.allclose(a, 0.1 * O.normal_draws(5, 10, 0, 2, 3 * B).reshape(B, 3), rtol=0, atol=1e-15)
+    assert np.array_equal(O.color_shift(5, 0, 2, B, ident, ones, 0.0), np.zeros((B, 3)))
+    # a rotation of the components preserves the length of every offset; eigenvalues scale the coordinates
+    th = 0.7
+    rot = np.array([[np.cos(th), -np.sin(th), 0.0], [np.sin(th), np.cos(th), 0.0], [0.0, 0.0, 1.0]])
+    lam = np.array([3.0, 2.0, 0.5])
+    b = O.color_shift(5, 0, 2, B, rot, lam, 0.1)
+    assert np.allclose(np.linalg.norm(b, axis=1), np.linalg.norm(a * lam, axis=1), rtol=1e-12)
+    # a single component along (1,1,1)/sqrt 3 shifts all three colours alike: a pure intensity change
+    grey = np.zeros((3, 3)); grey[:, 0] = 1.0 / np.sqrt(3.0)
+    c = O.color_shift(5, 0, 2, B, grey, np.array([4.0, 0.0, 0.0]), 0.1)
+    assert np.allclose(c[:, 0], c[:, 1]) and np.allclose(c[:, 1], c[:, 2]) and np.abs(c).max() > 0
+    # column i of eigvec is component i: with eigval e_1 only the second column matters
+    only1 = O.color_shift(5, 0, 2, B, rot, np.array([0.0, 1.0, 0.0]), 0.1)
+    assert np.allclose(only1, np.outer(a[:, 1], rot[:, 1]), atol=1e-15)
+
+
+def test_preprocess_with_shift_is_a_per_image_colour_offset():
+    rng = np.random.default_rng(4)
+    img = rng.integers(0, 256, size=(3, 256, 256, 3), dtype=np.uint8)
+    mean = rng.uniform(100, 140, size=(256, 256, 3))
+    cf = O.crop_flip(9, 0, 0, 3)
+    shift = rng.standard_normal((3, 3))
+    x0, x1 = O.preprocess(img, mean, cf), O.preprocess(img, mean, cf, shift)
+    d = x1 - x0
+    for n in range(3):
+        for c in range(3):
+            assert np.allclose(d[n, c], shift[n, c], rtol=0, atol=1e-12)
