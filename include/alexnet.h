@@ -106,6 +106,17 @@ int alexnet_destroy(alexnet_t* h);
  * consumed returns STATE. */
 int alexnet_load_batch_async(alexnet_t* h, int replica, const uint8_t* images, const int32_t* labels, uint64_t step);
 
+/* The intensity augmentation of Krizhevsky et al. 2012 (section 4.1), which the
+ * paper's experiments leave out ("Experiments", the sentence on the reported
+ * error rates): off by default; with sigma > 0 every later training load adds,
+ * to all pixels of image n, the RGB offset eigvec * (alpha_n .* eigval) with
+ * alpha_n ~ N(0, sigma^2) in R^3 drawn per image from (seed, replica, step).
+ *   host_eigvec  host fp32 [3][3], row = colour, column i = i-th principal component of the RGB values of the training set
+ *   host_eigval  host fp32 [3]
+ *   sigma        0.1 in that paper; 0 switches the augmentation off (the arrays may then be NULL)
+ * Evaluation batches are never augmented.  Takes effect for loads issued after the call.  Errors: ARG. */
+int alexnet_set_color_augmentation(alexnet_t* h, const float* host_eigvec, const float* host_eigval, float sigma);
+
 /* One SGD step of `replica` on its oldest loaded batch (paper, "Data
  * parallelism": every replica is updated on a minibatch of its own): forward,
  * softmax cross-entropy, backward, momentum update

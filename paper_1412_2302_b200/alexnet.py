@@ -37,7 +37,7 @@ EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "
            "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error", "alexnet_bias_grad_noalloc", "alexnet_loader_ring_bytes",
            "alexnet_loader_create", "alexnet_loader_next", "alexnet_loader_release", "alexnet_loader_destroy",
            "alexnet_forward_backward", "alexnet_apply_update", "alexnet_update_and_average", "alexnet_param_regions",
-           "alexnet_scale_and_refresh", "alexnet_create_error", "alexnet_debug_expire_wait"]
+           "alexnet_scale_and_refresh", "alexnet_create_error", "alexnet_debug_expire_wait", "alexnet_set_color_augmentation"]
 
 
 class Config(ctypes.Structure):
@@ -84,6 +84,7 @@ def load_library():
     L.alexnet_create_error.restype = ctypes.c_char_p
     L.alexnet_create_error.argtypes = []
     L.alexnet_debug_expire_wait.argtypes = [vp, ctypes.c_longlong]
+    L.alexnet_set_color_augmentation.argtypes = [vp, vp, vp, ctypes.c_float]
     L.alexnet_eval_batch.argtypes = [vp, i32, vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                                      ctypes.POINTER(ctypes.c_float)]
     L.alexnet_get_params.argtypes = [vp, i32, i32, vp, sz]
@@ -229,6 +230,15 @@ class AlexNet:
             off = p.value - base
             out.append(self.arena[off:off + 4 * n.value].view(self._torch.float32))
         return tuple(out)
+
+    def set_color_augmentation(self, eigvec=None, eigval=None, sigma=0.0):
+        """Intensity augmentation of training loads: eigvec (3,3), eigval (3,) of the data set's RGB values; sigma 0 = off."""
+        if sigma == 0:
+            self._ck(self.lib.alexnet_set_color_augmentation(self.h, None, None, 0.0))
+            return
+        ev = np.ascontiguousarray(eigvec, np.float32).reshape(3, 3)
+        el = np.ascontiguousarray(eigval, np.float32).reshape(3)
+        self._ck(self.lib.alexnet_set_color_augmentation(self.h, _ptr(ev), _ptr(el), float(sigma)))
 
     def debug_expire_wait(self, budget_cycles=2_000_000):
         self._ck(self.lib.alexnet_debug_expire_wait(self.h, int(budget_cycles)))

@@ -171,6 +171,7 @@ struct alexnet {
     uint64_t launches;
     int latched;
     float alpha_eff, drop_scale; uint32_t thr24;
+    kn::ColorAug color = {};      // sigma == 0: no intensity augmentation (the paper's setting)
     int sm_count;
     PFN_cuTensorMapEncodeTiled_v12000 encode;
     // optional per-launch timing of the GEMM kernel (event pairs on the launching stream)
@@ -852,8 +853,14 @@ void op_average(alexnet* h, cudaStream_t st) {
 void op_preprocess(alexnet* h, int r, int slot, uint64_t step, cudaStream_t st, bool eval = false) {
     Replica& R = h->rep[r];
     const long long total = (long long)h->B * 57 * 57 * 4;
-    launch_k(kn::preprocess_kernel, nblk(total, 256), 256, 0, st, R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
-                                                            kn::stream_key(h->cfg.seed, 1, r, step), eval ? 1 : 0);
+    kn::ColorAug aug = h->color;
+    aug.key = kn::stream_key(h->cfg.seed, 10, r, step);
+    if (aug.sigma != 0.f && !eval)
+        launch_k(kn::preprocess_kernel<true>, nblk(total, 256), 256, 0, st, R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
+                 kn::stream_key(h->cfg.seed, 1, r, step), 0, aug);
+    else
+        launch_k(kn::preprocess_kernel<false>, nblk(total, 256), 256, 0, st, R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
+                 kn::stream_key(h->cfg.seed, 1, r, step), eval ? 1 : 0, aug);
     h->launches++;
 }
 
@@ -1215,6 +1222,15 @@ int alexnet_scale_and_refresh(alexnet_t* h, int replica, float scale) {
     if (int rc = check_status(h)) return rc;
     op_scale_refresh(h, replica, scale, h->cs);
     CK(cudaGetLastError());
+    return ALEXNET_OK;
+}
+
+int alexnet_set_color_augmentation(alexnet_t* h, const float* host_eigvec, const float* host_eigval, float sigma) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (!(sigma >= 0.f) || (sigma > 0.f && (!host_eigvec || !host_eigval))) return fail(h, ALEXNET_ERR_ARG, "set_color_augmentation: bad argument");
+    h->color.sigma = sigma;
+    for (int c = 0; c < 3 && sigma > 0.f; ++c)
+        for (int i = 0; i < 3; ++i) h->color.pl[3 * c + i] = host_eigvec[3 * c + i] * host_eigval[i];
     return ALEXNET_OK;
 }
 

@@ -51,9 +51,20 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 // sy = oy + Y, sx = ox + (flip ? 226 - X : X), written as bf16 in the 4x4
 // space-to-depth layout [B][57][57][48], channel = ((Y%4)*4 + X%4)*3 + c,
 // with row/column 227 of the 228-padded image set to zero.
+// Optional intensity augmentation (Krizhevsky et al. 2012, section 4.1; the paper's experiments leave it out): every
+// pixel of image n gets the RGB offset d = sum_i pl[.][i] * alpha_i with pl[c][i] = eigvec[c][i] * eigval[i] and
+// alpha_i = sigma * z_i, z_i standard normal from the hash (stream 10, index 3 n + i, Box-Muller as in the init kernel).
+struct ColorAug { float pl[9]; float sigma; uint64_t key; };
+__device__ __forceinline__ float normal_draw(uint64_t key, uint64_t idx) {
+    const uint64_t r = draw(key, idx);
+    const float u1 = ((float)(r >> 40) + 1.f) * (1.f / 16777216.f);
+    const float u2 = (float)((r >> 16) & 0xFFFFFF) * (1.f / 16777216.f);
+    return sqrtf(-2.f * logf(u1)) * cospif(2.f * u2);
+}
+template <bool AUG>
 __global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* __restrict__ mean,
                                   __nv_bfloat16* __restrict__ out, int32_t* __restrict__ cf_out,
-                                  int B, uint64_t key, int eval_mode) {
+                                  int B, uint64_t key, int eval_mode, const ColorAug aug) {
     pdl_sync();
     // one thread per (n, by, bx, dy): 12 output values (4 dx * 3 colours) = 24 bytes
     const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -70,6 +81,13 @@ __global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* 
     const int flip = eval_mode ? 0 : (int)((r >> 32) & 1);
     if (cf_out && by == 0 && bx == 0 && dy == 0) { cf_out[3 * n] = ox; cf_out[3 * n + 1] = oy; cf_out[3 * n + 2] = flip; }
     const int Y = by * 4 + dy;
+    float shift[3] = {0.f, 0.f, 0.f};
+    if (AUG && !eval_mode) {
+        const float a0 = aug.sigma * normal_draw(aug.key, 3ull * n), a1 = aug.sigma * normal_draw(aug.key, 3ull * n + 1),
+                    a2 = aug.sigma * normal_draw(aug.key, 3ull * n + 2);
+        #pragma unroll
+        for (int c = 0; c < 3; ++c) shift[c] = aug.pl[3 * c] * a0 + aug.pl[3 * c + 1] * a1 + aug.pl[3 * c + 2] * a2;
+    }
     float v[12];
     #pragma unroll
     for (int dx = 0; dx < 4; ++dx) {
@@ -79,7 +97,7 @@ __global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* 
             const size_t s = ((size_t)sy * 256 + sx) * 3;
             const uint8_t* ip = img + (size_t)n * 196608 + s;
             #pragma unroll
-            for (int c = 0; c < 3; ++c) v[dx * 3 + c] = (float)ip[c] - mean[s + c];
+            for (int c = 0; c < 3; ++c) v[dx * 3 + c] = ((float)ip[c] - mean[s + c]) + shift[c];
         } else {
             v[dx * 3] = v[dx * 3 + 1] = v[dx * 3 + 2] = 0.f;
         }

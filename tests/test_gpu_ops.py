@@ -346,3 +346,43 @@ def test_update_and_average_fp32(net):
     net.replica_average()                                 # identical replicas: bitwise identity
     net.sync()
     assert np.array_equal(net.get_params(0, 0), before) and np.array_equal(net.get_params(1, 0), before)
+
+
+def test_preprocess_intensity_augmentation(net):
+    """The augmentation the paper's experiments leave out, as an option of the preprocessing gather: per-image RGB offsets
+    from the hash (fp32 Box-Muller on the device, fp64 in the oracle: the bf16 result may differ by one rounding step in a
+    few places), never at evaluation, and switched off again the gather is bit-exact as before."""
+    import torch
+    B = net.batch
+    th = 0.6
+    eigvec = np.array([[np.cos(th), -np.sin(th), 0.0], [np.sin(th), np.cos(th), 0.0], [0.0, 0.0, 1.0]]) @ np.array(
+        [[1.0, 0.0, 0.0], [0.0, np.cos(0.3), -np.sin(0.3)], [0.0, np.sin(0.3), np.cos(0.3)]])
+    eigval = np.array([55.0, 5.0, 1.2])                     # spread of the three components, in pixel units
+    step = 9
+    img, lab = synth.images(SEED, 0, step, B), synth.labels(SEED, 0, step, B)
+    net.set_color_augmentation(eigvec, eigval, 0.1)
+    net.load_batch_async(0, torch.from_numpy(img), torch.from_numpy(lab), step)
+    net.sync()
+    cf = O.crop_flip(SEED, 0, step, B)
+    assert np.array_equal(net.get_tensor("CROPFLIP").reshape(B, 3).astype(np.int32), cf)
+    shift = O.color_shift(SEED, 0, step, B, eigvec.astype(np.float32), eigval.astype(np.float32), 0.1)
+    assert np.abs(shift).max() > 1.0                        # a visible offset
+    ref = O.preprocess(img, synth.mean_image(SEED), cf, shift)
+    got = net.get_tensor("X0").reshape(ref.shape).astype(np.float64)
+    plain = O.preprocess(img, synth.mean_image(SEED), cf)
+    assert rel(got, ref) < 2.5e-3 and rel(got, plain) > 10 * rel(got, ref)
+    want = O.round_bf16(ref.astype(np.float32))
+    off = got != want
+    # one bf16 rounding step, or, where pixel - mean + offset nearly cancels, the fp32 rounding of terms of size 256
+    assert off.mean() < 0.01 and (np.abs(got - want)[off] <= np.abs(want[off]) * 2.0 ** -7 + 2e-4).all()
+    net.train_step(0); net.sync()
+    # evaluation never augments; and with sigma = 0 the training gather is bit-exact again
+    net.eval_batch(0, torch.from_numpy(img), torch.from_numpy(lab))       # (the parameters are whatever earlier tests left: only X0 matters)
+    x_eval = net.get_tensor("X0").reshape(ref.shape)
+    centre = O.preprocess(img, synth.mean_image(SEED), np.tile(np.array([[14, 14, 0]], np.int32), (B, 1)))
+    assert np.array_equal(x_eval, O.round_bf16(centre.astype(np.float32)).astype(np.float32))
+    net.set_color_augmentation(sigma=0.0)
+    net.load_batch_async(0, torch.from_numpy(img), torch.from_numpy(lab), step)
+    net.sync()
+    assert np.array_equal(net.get_tensor("X0").reshape(ref.shape), O.round_bf16(plain.astype(np.float32)).astype(np.float32))
+    net.train_step(0); net.sync()
