@@ -206,6 +206,22 @@ int alexnet_update_and_average(alexnet_t* h);
  * rebuilds the copies, which is what a caller needs after writing averaged
  * parameters into the arrays itself.  Asynchronous, on the compute stream. */
 int alexnet_param_regions(alexnet_t* h, int replica, float** dev_w, float** dev_v, float** dev_g, size_t* n_floats);
+
+/* The paper's own form of the exchange (the data-parallel figure: step 2, each
+ * GPU copies the other's weights, biases and momentum into receive buffers of
+ * its own; step 3, it averages them with its own): the caller has brought the
+ * other replicas' parameter and momentum arrays (alexnet_param_regions of the
+ * peers: peer copies, or an all-gather) into buffers on THIS GPU; this call
+ * replaces the replica's parameters and momentum by the mean over all `count`
+ * replicas and rebuilds the bf16 copies.  One pass: (count - 1) x 8 + 8 bytes
+ * read and 10 written per parameter index.
+ *   dev_w, dev_v  host arrays of `count` device pointers, entry r = the arrays received from the replica of rank r
+ *                 (n_floats fp32 each, 16-byte aligned, in this GPU's memory); entry `self` is ignored: the replica's
+ *                 own arrays take its place, so that every rank adds the replicas in the same (rank) order and all
+ *                 ranks end with bit-identical parameters
+ *   count         number of replicas, 1..8;  self: this replica's rank, 0 <= self < count
+ * Asynchronous, on the compute stream; the buffers must stay unchanged until it has run.  Errors: ARG, DEVICE_TIMEOUT, CUDA. */
+int alexnet_average_received(alexnet_t* h, int replica, const float* const* dev_w, const float* const* dev_v, int count, int self);
 int alexnet_scale_and_refresh(alexnet_t* h, int replica, float scale);
 
 /* Read / write a replica's parameters in the canonical order above.

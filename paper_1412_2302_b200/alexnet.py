@@ -37,7 +37,7 @@ EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "
            "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error", "alexnet_bias_grad_noalloc", "alexnet_loader_ring_bytes",
            "alexnet_loader_create", "alexnet_loader_next", "alexnet_loader_release", "alexnet_loader_destroy",
            "alexnet_forward_backward", "alexnet_apply_update", "alexnet_update_and_average", "alexnet_param_regions",
-           "alexnet_scale_and_refresh", "alexnet_create_error", "alexnet_debug_expire_wait", "alexnet_set_color_augmentation"]
+           "alexnet_scale_and_refresh", "alexnet_create_error", "alexnet_debug_expire_wait", "alexnet_set_color_augmentation", "alexnet_average_received"]
 
 
 class Config(ctypes.Structure):
@@ -85,6 +85,7 @@ def load_library():
     L.alexnet_create_error.argtypes = []
     L.alexnet_debug_expire_wait.argtypes = [vp, ctypes.c_longlong]
     L.alexnet_set_color_augmentation.argtypes = [vp, vp, vp, ctypes.c_float]
+    L.alexnet_average_received.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), i32, i32]
     L.alexnet_eval_batch.argtypes = [vp, i32, vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                                      ctypes.POINTER(ctypes.c_float)]
     L.alexnet_get_params.argtypes = [vp, i32, i32, vp, sz]
@@ -218,6 +219,17 @@ class AlexNet:
 
     def scale_and_refresh(self, replica=0, scale=1.0):
         self._ck(self.lib.alexnet_scale_and_refresh(self.h, replica, float(scale)))
+
+    def average_received(self, replica, recv_w, recv_v, self_rank):
+        """Average the replica's parameters and momentum with the copies received from the other replicas: recv_w / recv_v
+        are lists with one fp32 CUDA tensor per rank (entry self_rank may be None: the replica's own arrays stand there)."""
+        n = len(recv_w)
+        pw, pv = (ctypes.c_void_p * n)(), (ctypes.c_void_p * n)()
+        for r in range(n):
+            pw[r] = None if r == self_rank or recv_w[r] is None else recv_w[r].data_ptr()
+            pv[r] = None if r == self_rank or recv_v[r] is None else recv_v[r].data_ptr()
+        self._keep = self._keep[-8:] + [(recv_w, recv_v)]
+        self._ck(self.lib.alexnet_average_received(self.h, replica, pw, pv, n, int(self_rank)))
 
     def param_views(self, replica=0):
         """(w, v, g): fp32 torch views of the replica's parameter, momentum and gradient arrays inside the arena (the

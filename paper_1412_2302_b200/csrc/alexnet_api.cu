@@ -1234,6 +1234,27 @@ int alexnet_set_color_augmentation(alexnet_t* h, const float* host_eigvec, const
     return ALEXNET_OK;
 }
 
+int alexnet_average_received(alexnet_t* h, int replica, const float* const* dev_w, const float* const* dev_v, int count, int self) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (replica < 0 || replica >= h->cfg.replicas || count < 1 || count > 8 || self < 0 || self >= count || !dev_w || !dev_v)
+        return fail(h, ALEXNET_ERR_ARG, "average_received: bad argument (1 <= count <= 8, 0 <= self < count)");
+    if (int rc = check_status(h)) return rc;
+    Replica& R = h->rep[replica];
+    kn::RecvList rl{};
+    rl.count = count;
+    for (int r = 0; r < count; ++r) {
+        rl.w[r] = r == self ? R.w : dev_w[r];
+        rl.v[r] = r == self ? R.v : dev_v[r];
+        if (!rl.w[r] || !rl.v[r] || ((uintptr_t)rl.w[r] & 15) || ((uintptr_t)rl.v[r] & 15))
+            return fail(h, ALEXNET_ERR_ARG, "average_received: NULL or misaligned buffer");
+    }
+    launch_k(kn::average_received_kernel, 1184, 256, 0, h->cs, R.w, R.v, R.shadow, rl, h->L.n_total / 4, 1.f / (float)count);
+    h->launches++;
+    refresh_shadows(h, replica, false, h->cs);
+    CK(cudaGetLastError());
+    return ALEXNET_OK;
+}
+
 int alexnet_debug_expire_wait(alexnet_t* h, long long budget_cycles) {
     if (!h) return ALEXNET_ERR_ARG;
     if (int rc = check_status(h)) return rc;

@@ -826,6 +826,30 @@ __global__ void __launch_bounds__(256) scale_refresh_kernel(float* __restrict__ 
         ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
     }
 }
+// The paper's own form of the exchange ("Data parallelism" figure, steps 2 and 3): every replica has RECEIVED the other
+// replicas' parameters and momenta into buffers of its own GPU (peer copies or an all-gather: the caller's) and now averages.
+// slot[r] = the arrays of the replica of rank r in rank order, the local replica's own arrays at r = self (so every rank adds
+// in the same order and all ranks end bit-identical); w, v = the local arrays, overwritten; also writes the bf16 copy.
+struct RecvList { const float* w[8]; const float* v[8]; int count; };
+__global__ void __launch_bounds__(256) average_received_kernel(float* __restrict__ w, float* __restrict__ v, __nv_bfloat16* __restrict__ shadow,
+                                                               const RecvList rl, long long n4, float inv_count) {
+    pdl_sync();
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 a = ((const float4*)rl.w[0])[i], c = ((const float4*)rl.v[0])[i];
+        #pragma unroll 1
+        for (int r = 1; r < rl.count; ++r) {
+            const float4 b = ((const float4*)rl.w[r])[i], d = ((const float4*)rl.v[r])[i];
+            a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+            c.x += d.x; c.y += d.y; c.z += d.z; c.w += d.w;
+        }
+        a.x *= inv_count; a.y *= inv_count; a.z *= inv_count; a.w *= inv_count;
+        c.x *= inv_count; c.y *= inv_count; c.z *= inv_count; c.w *= inv_count;
+        ((float4*)w)[i] = a; ((float4*)v)[i] = c;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(a.x, a.y), hi = __floats2bfloat162_rn(a.z, a.w);
+        ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
+    }
+}
 __global__ void shadow_kernel(const float* __restrict__ w, __nv_bfloat16* __restrict__ shadow, long long n4) {
     pdl_sync();
     const long long stride = (long long)gridDim.x * blockDim.x;

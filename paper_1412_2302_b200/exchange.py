@@ -11,6 +11,8 @@ Two forms, equal in exact arithmetic for replicas that start the step identical 
 section; checked to 1e-5 in the tests):
 
   exchange_and_average(rep)            after train_step: all-reduce w and v (8 bytes per parameter on the wire)
+  exchange_then_average(rep)           after train_step, the paper's own two steps: every rank receives the other ranks'
+                                       w and v into buffers of its own (all-gather), then averages them with its own
   allreduce_gradients_and_update(rep)  after forward_backward: all-reduce g (4 bytes per parameter), then one update
                                        with the mean gradient
 
@@ -43,6 +45,9 @@ class LocalReplica:
     def apply_update(self, grad_scale):
         self.net.apply_update(self.replica, grad_scale)
 
+    def average_received(self, recv_w, recv_v, self_rank):
+        self.net.average_received(self.replica, recv_w, recv_v, self_rank)
+
 
 class _NoStream:
     def __enter__(self):
@@ -70,6 +75,23 @@ def exchange_and_average(rep, group=None):
             dist.all_reduce(w, op=dist.ReduceOp.SUM, group=group)
             dist.all_reduce(v, op=dist.ReduceOp.SUM, group=group)
         rep.scale_and_refresh(1.0 / world)
+
+
+def exchange_then_average(rep, group=None, buffers=None):
+    """The figure's steps as drawn: (2) every replica's weights, biases and momentum are copied to all others, into receive
+    buffers on the receiving GPU; (3) every GPU averages what it holds.  buffers = (list of w buffers, list of v buffers),
+    one per rank, kept by the caller between steps (allocated here when None).  Returns the buffers."""
+    world = _world(group)
+    rank = dist.get_rank(group) if _initialised() else 0
+    w, v, _ = rep.param_views()
+    if buffers is None:
+        buffers = ([torch.empty_like(w) for _ in range(world)], [torch.empty_like(v) for _ in range(world)])
+    with (rep.stream() if hasattr(rep, "stream") else _NoStream()):
+        if _initialised():
+            dist.all_gather(buffers[0], w, group=group)
+            dist.all_gather(buffers[1], v, group=group)
+        rep.average_received(buffers[0], buffers[1], rank)
+    return buffers
 
 
 def allreduce_gradients_and_update(rep, group=None):

@@ -33,6 +33,15 @@ class HostReplica:
         self.w.mul_(scale); self.v.mul_(scale)
         self.refreshed += 1
 
+    def average_received(self, recv_w, recv_v, self_rank):
+        n = len(recv_w)
+        sw, sv = torch.zeros_like(self.w), torch.zeros_like(self.v)
+        for r in range(n):                              # rank order, the own arrays at the own rank
+            sw += self.w if r == self_rank else recv_w[r]
+            sv += self.v if r == self_rank else recv_v[r]
+        self.w.copy_(sw * (1.0 / n)); self.v.copy_(sv * (1.0 / n))
+        self.refreshed += 1
+
     def apply_update(self, grad_scale):
         assert self.pending
         self.v.mul_(MU).add_(self.w, alpha=-LR * WD).add_(self.g * grad_scale, alpha=-LR)
@@ -69,6 +78,11 @@ def _worker(rank, world, port, out):
         # gradient form: all-reduce the gradients, one update with their mean
         b = HostReplica(w, v, g)
         exchange.allreduce_gradients_and_update(b)
+        # the figure's own two steps: receive the other replica's arrays, then average
+        c = HostReplica(w, v, g)
+        c.apply_update(1.0)
+        exchange.exchange_then_average(c)
+        assert torch.equal(c.w, a.w) and torch.equal(c.v, a.v)          # two replicas: the same sum, the same halving
         exchange.barrier(world)
         ms = exchange.max_over_ranks(10.0 + 5.0 * rank, world)          # rank 1 is the slow one
         out.put((rank, a.w.numpy().copy(), a.v.numpy().copy(), b.w.numpy().copy(), b.v.numpy().copy(), a.refreshed, ms))

@@ -36,7 +36,7 @@ def test_one_rank_nccl_exchange_equals_local_paths(nccl_group):
         net = AlexNet(batch=B, seed=seed, mean_image=synth.mean_image(seed))
         net.set_params(w)
         rep = exchange.LocalReplica(net, 0)
-        losses = []
+        losses, state = [], {}
         for step in range(3):
             img = torch.from_numpy(synth.images(seed, 0, step, B)).pin_memory()
             lab = torch.from_numpy(synth.labels(seed, 0, step, B)).pin_memory()
@@ -46,6 +46,9 @@ def test_one_rank_nccl_exchange_equals_local_paths(nccl_group):
             elif mode == "params":
                 losses.append(net.train_step(0, want_loss=True))
                 exchange.exchange_and_average(rep)
+            elif mode == "gather":
+                losses.append(net.train_step(0, want_loss=True))
+                state["buffers"] = exchange.exchange_then_average(rep, buffers=state.get("buffers"))
             else:
                 losses.append(net.forward_backward(0, want_loss=True))
                 exchange.allreduce_gradients_and_update(rep)
@@ -54,8 +57,8 @@ def test_one_rank_nccl_exchange_equals_local_paths(nccl_group):
         net.close()
         return out
 
-    plain, params, grads = run("plain"), run("params"), run("grads")
-    for other in (params, grads):
+    plain, params, grads, gather = run("plain"), run("params"), run("grads"), run("gather")
+    for other in (params, grads, gather):
         assert other[0] == plain[0]
         assert np.array_equal(other[1], plain[1]) and np.array_equal(other[2], plain[2])
     assert not np.array_equal(plain[1], w)

@@ -564,6 +564,21 @@ def test_deferred_update_forms():
     assert rel(net.get_params(0, 0), O.replica_average(wa.astype(np.float64), wb.astype(np.float64))[0]) < 1e-5
     assert rel(net.get_params(0, 1), O.replica_average(va.astype(np.float64), vb.astype(np.float64))[0]) < 1e-5
     assert rel(net.get_params(0, 0), wm) < 1e-5                     # and both forms of the exchange agree
+    # (4) the figure's own form: each replica averages its arrays with a received copy of the other's (rank order)
+    avg_w, avg_v = net.get_params(0, 0), net.get_params(0, 1)
+    net.set_params(wa, 0); net.set_params(va, 0, 1)               # back to the two separately updated replicas
+    with torch.cuda.stream(net.compute_stream):
+        ra = [t.clone() for t in net.param_views(0)[:2]]          # what replica 1 receives from replica 0, and vice versa
+        rb = [t.clone() for t in net.param_views(1)[:2]]
+    net.average_received(0, [None, rb[0]], [None, rb[1]], 0)
+    net.average_received(1, [ra[0], None], [ra[1], None], 1)
+    net.sync()
+    assert np.array_equal(net.get_params(0, 0), net.get_params(1, 0)) and np.array_equal(net.get_params(0, 1), net.get_params(1, 1))
+    assert rel(net.get_params(0, 0), O.replica_average(wa.astype(np.float64), wb.astype(np.float64))[0]) < 1e-5
+    assert np.array_equal(net.get_params(0, 0), avg_w) and np.array_equal(net.get_params(0, 1), avg_v)   # (a + b) / 2 either way
+    with pytest.raises(A.AlexNetError) as e:
+        net.average_received(0, [None] * 9, [None] * 9, 0)
+    assert e.value.code == A.ERR_ARG
     # the refreshed bf16 copies are the ones the next step computes with: one more step must match a fresh handle
     chk = make(B, seed=seed)
     chk.set_params(net.get_params(0, 0)); chk.set_params(net.get_params(0, 1), 0, 1)
@@ -650,4 +665,57 @@ def test_gradient_is_bit_for_bit_repeatable_under_overlap_batch128():
     S = torch.stack(snaps)
     assert bool((S == S[0]).all()), int((S != S[0]).any(dim=1).sum())
     assert bool(torch.isfinite(S[0]).all()) and float(S[0].abs().max()) > 0
+    net.close()
+
+
+def test_batch256_sampled_layers_and_weight_gradients():
+    """The per-layer sweep's batch (256: two row tiles per FC pass, other split counts everywhere).  Two images are
+    followed through every layer by the oracle; every weight and bias gradient is recomputed by the oracle's backward-weight
+    functions FROM the device's own activations and output gradients (exact inputs, whole batch), so each weight-gradient
+    kernel and each split reduction is checked at this batch without an fp64 step over 256 images."""
+    seed, B = BASE + 5, 256
+    net = make(B, seed=seed)
+    w = synth.init_params(seed, variance_preserving=True, bias=0.1)
+    net.set_params(w)
+    img, lab = load(net, 0, seed, 0, B)
+    loss = net.forward_backward(0, want_loss=True)
+    assert np.isfinite(loss)
+    assert_step_pooling_exact(net)
+    pick = [0, 255]
+    onet = O.OracleNet(O.OracleConfig(seed=seed), w.astype(np.float64))
+    kw = dict(cf=O.crop_flip(seed, 0, 0, B)[pick], m6=O.dropout_mask(seed, 2, 0, 0, B, 4096, 0.5)[pick],
+              m7=O.dropout_mask(seed, 3, 0, 0, B, 4096, 0.5)[pick], mean_over=B)
+    T = onet.forward_backward(img[pick], lab[pick], synth.mean_image(seed), 0, **kw)
+    gates, args = gpu_decisions(net, T, pick=pick)
+    Tb = onet.forward_backward(img[pick], lab[pick], synth.mean_image(seed), 0, gates=gates, args=args, **kw)
+    T.update({k: Tb[k] for k in GRADS})
+    G = {k: net.get_tensor(k.upper()) for k in ACTS + GRADS}
+    errs = {k: rel(G[k].reshape((B,) + T[k].shape[1:])[pick], T[k]) for k in ACTS + GRADS}
+    bad = {k: v for k, v in errs.items() if not v < TOL}
+    assert not bad, (bad, errs)
+    # weight gradients from the device's own tensors
+    g = net.get_params(0, 2)
+    off, _ = O.param_offsets()
+    shp = {"x0": (3, 227, 227), "p1": (96, 27, 27), "p2": (256, 13, 13), "a3": (384, 13, 13), "a4": (384, 13, 13)}
+    dys = {"conv1": ("x0", "da1", 55), "conv2": ("p1", "da2", 27), "conv3": ("p2", "da3", 13), "conv4": ("a3", "da4", 13), "conv5": ("a4", "da5", 13)}
+    gerr = {}
+    for name, (tx, tdy, ho) in dys.items():
+        c = O.CONV[name]
+        x = G[tx].reshape((B,) + shp[tx]).astype(np.float64)
+        dy = G[tdy].reshape(B, c["cout"], ho, ho).astype(np.float64)
+        o, n, s_ = off[name + ".W"]
+        dw, db = O.conv_bwd_weight(x, dy, s_, c["s"], c["p"], c["g"])
+        gerr[name + ".W"] = rel(g[o:o + n], dw)
+        o, n, _ = off[name + ".b"]
+        gerr[name + ".b"] = rel(g[o:o + n], db)
+    for name, tx, tdy in (("fc6", "p5", "df6"), ("fc7", "f6", "df7"), ("fc8", "f7", "dz")):
+        K, N = O.FC[name]
+        x = G[tx].reshape(B, K).astype(np.float64)
+        dy = G[tdy].reshape(B, N).astype(np.float64)
+        o, n, _ = off[name + ".W"]
+        gerr[name + ".W"] = rel(g[o:o + n], (dy.T @ x).ravel())
+        o, n, _ = off[name + ".b"]
+        gerr[name + ".b"] = rel(g[o:o + n], dy.sum(axis=0))
+    bad = {k: v for k, v in gerr.items() if not v < 1e-3}          # exact bf16 inputs, fp32 accumulation: summation order only
+    assert not bad, (bad, gerr)
     net.close()
