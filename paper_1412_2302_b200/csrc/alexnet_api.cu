@@ -674,7 +674,12 @@ void refresh_shadows(alexnet* h, int r, bool whole, cudaStream_t st) {
         launch_k(kn::shadow_kernel, 1184, 256, 0, st, R.w, R.shadow, h->L.n_total / 4);
         h->launches++;
     }
-    launch_k(kn::conv_transpose_shadow_kernel, 592, 256, 0, st, R.shadow, R.wt, h->L.tjobs);
+    launch_k(kn::conv_transpose_shadow_kernel, h->L.tjobs.tile0[5], 256, 0, st, R.shadow, R.wt, (bf16*)nullptr, h->L.tjobs);
+    h->launches++;
+}
+// after an average both replicas hold the same parameters: one launch writes both transposed copies
+void refresh_transposed_both(alexnet* h, cudaStream_t st) {
+    launch_k(kn::conv_transpose_shadow_kernel, h->L.tjobs.tile0[5], 256, 0, st, h->rep[0].shadow, h->rep[0].wt, h->rep[1].wt, h->L.tjobs);
     h->launches++;
 }
 
@@ -833,8 +838,7 @@ void op_update_average(alexnet* h, cudaStream_t st) {
     launch_k(kn::sgd_update_average_kernel, 1184, 256, 0, st, A.w, A.v, A.g, Bq.w, Bq.v, Bq.g, A.shadow, Bq.shadow, L.n_total / 4,
              nd / 4, h->cfg.lr, h->cfg.momentum, h->cfg.weight_decay);
     h->launches++;
-    refresh_shadows(h, 0, false, st);
-    refresh_shadows(h, 1, false, st);
+    refresh_transposed_both(h, st);
 }
 void op_scale_refresh(alexnet* h, int r, float scale, cudaStream_t st) {
     Replica& R = h->rep[r];
@@ -847,8 +851,7 @@ void op_average(alexnet* h, cudaStream_t st) {
     Replica &A = h->rep[0], &Bq = h->rep[1];
     launch_k(kn::replica_average_kernel, 1184, 256, 0, st, A.w, Bq.w, A.v, Bq.v, A.shadow, Bq.shadow, h->L.n_total / 4);
     h->launches++;
-    refresh_shadows(h, 0, false, st);
-    refresh_shadows(h, 1, false, st);
+    refresh_transposed_both(h, st);
 }
 void op_preprocess(alexnet* h, int r, int slot, uint64_t step, cudaStream_t st, bool eval = false) {
     Replica& R = h->rep[r];

@@ -860,22 +860,37 @@ __global__ void shadow_kernel(const float* __restrict__ w, __nv_bfloat16* __rest
     }
 }
 
-__global__ void conv_transpose_shadow_kernel(const __nv_bfloat16* __restrict__ shadow, __nv_bfloat16* __restrict__ wt,
-                                             const TransposeJobs jobs) {
+// Transposed bf16 copies of the conv filters from the bf16 copy of the weights, in the 32 x 32 tiles of
+// sgd_update_conv_kernel (8-byte reads along the input channels, 8-byte writes along the output channels through a
+// shared-memory tile); wt2 != nullptr: a second destination (the other replica's copy after an average, when both are equal).
+__global__ void __launch_bounds__(256) conv_transpose_shadow_kernel(const __nv_bfloat16* __restrict__ shadow, __nv_bfloat16* __restrict__ wt,
+                                                                    __nv_bfloat16* __restrict__ wt2, const TransposeJobs jobs) {
     pdl_sync();
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (int q = 0; q < jobs.n; ++q) {
-        const TransposeJob J = jobs.j[q];
-        const int cog = J.cout / J.groups;
-        for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < J.count; i += stride) {
-            // i indexes dst [tap][cin][cog]
-            const int co_ = (int)(i % cog);
-            long long r = i / cog;
-            const int cin = (int)(r % (J.cig * J.groups));
-            const int tap = (int)(r / (J.cig * J.groups));
-            const int grp = cin / J.cig, ci = cin % J.cig;
-            wt[J.dst_off + i] = shadow[J.src_off + ((long long)tap * J.cout + grp * cog + co_) * J.cig + ci];
-        }
+    __shared__ __nv_bfloat16 tile[32][36];       // [input channel][output channel], padded
+    int q = 0;
+    while (q + 1 < jobs.n && (int)blockIdx.x >= jobs.tile0[q + 1]) ++q;
+    const TransposeJob J = jobs.j[q];
+    const int cog = J.cout / J.groups;
+    const int ci_blocks = (J.cig + 31) / 32, co_blocks = J.cout / 32;
+    int t = (int)blockIdx.x - jobs.tile0[q];
+    const int cib = t % ci_blocks; t /= ci_blocks;
+    const int cob = t % co_blocks, tap = t / co_blocks;
+    const int r = threadIdx.x >> 3, c4 = threadIdx.x & 7;
+    const int co = cob * 32 + r, ci = cib * 32 + 4 * c4;
+    if (ci < J.cig) {                            // cig is a multiple of 4
+        const uint2 u = *(const uint2*)(shadow + J.src_off + ((long long)tap * J.cout + co) * J.cig + ci);
+        const __nv_bfloat162 lo2 = *(const __nv_bfloat162*)&u.x, hi2 = *(const __nv_bfloat162*)&u.y;
+        tile[4 * c4][r] = lo2.x; tile[4 * c4 + 1][r] = lo2.y; tile[4 * c4 + 2][r] = hi2.x; tile[4 * c4 + 3][r] = hi2.y;
+    }
+    __syncthreads();
+    const int ci2 = cib * 32 + r, cq = 4 * c4;   // now: thread (input channel r of the tile, four output channels from cq)
+    if (ci2 < J.cig) {
+        const int co0 = cob * 32 + cq, grp = co0 / cog, col = co0 - grp * cog;
+        const long long d = J.dst_off + ((long long)tap * J.cig * J.groups + grp * J.cig + ci2) * cog + col;
+        const __nv_bfloat162 a = __halves2bfloat162(tile[r][cq], tile[r][cq + 1]), b2 = __halves2bfloat162(tile[r][cq + 2], tile[r][cq + 3]);
+        const uint2 o = make_uint2(*(const uint32_t*)&a, *(const uint32_t*)&b2);
+        *(uint2*)(wt + d) = o;
+        if (wt2) *(uint2*)(wt2 + d) = o;
     }
 }
 
