@@ -163,14 +163,17 @@ def config4_leg(torch, dev, seed, repeats):
     timed `repeats` times after a checked warm-up pass, in the paper's literal form (two updates, then the average) and
     with the one-pass update + average."""
     from paper_1412_2302_b200 import synth
-    from paper_1412_2302_b200.alexnet import FLAG_FUSED_FC_UPDATE, AlexNet
+    from paper_1412_2302_b200.alexnet import FLAG_FUSED_FC_UPDATE, FLAG_SHARED_REPLICA_WEIGHTS, AlexNet
     iters = 10
     host = [[(torch.from_numpy(synth.images(seed, r, i, BATCH)).pin_memory(), torch.from_numpy(synth.labels(seed, r, i, BATCH)).pin_memory())
              for r in (0, 1)] for i in range(2)]
     out = {"workload": "2 replicas x batch 128 in one HBM, 10 x (2 loads from pinned host memory, 2 steps, 1 exchange-and-average)"}
-    for form in ("separate", "one_pass"):
+    # separate: the literal form (two updates, then the average); one_pass: both updates and the average in one pass over two
+    # copies of the parameters; shared: the same with ONE copy of the parameters for both replicas (they are equal at the
+    # start of every iteration), bit-identical results
+    for form in ("separate", "one_pass", "shared"):
         net = AlexNet(batch=BATCH, replicas=2, seed=seed, mean_image=synth.mean_image(seed), device=str(dev),
-                      flags=FLAG_FUSED_FC_UPDATE if form == "separate" else 0)
+                      flags={"separate": FLAG_FUSED_FC_UPDATE, "one_pass": 0, "shared": FLAG_SHARED_REPLICA_WEIGHTS}[form])
         w0 = synth.init_params(seed)
         net.set_params(w0, 0); net.set_params(w0, 1)
         cs = net.compute_stream
@@ -217,7 +220,7 @@ def config4_leg(torch, dev, seed, repeats):
         finite = bool(torch.isfinite(views[0][0]).all())
         med, rep = summarise(times)
         # the exchange alone
-        op, nbytes = ("AVERAGE", 36) if form == "separate" else ("UPDATE_AVERAGE", 44)
+        op, nbytes = {"separate": ("AVERAGE", 36), "one_pass": ("UPDATE_AVERAGE", 44), "shared": ("UPDATE_AVERAGE", 26)}[form]
         ts = []
         for _ in range(5):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -59,8 +59,18 @@ enum {                                /* alexnet_config_t.flags */
                                         * gradients: get_params(which = 2) is then meaningless for fc6.W / fc7.W / fc8.W,
                                         * and alexnet_run_op of an FC weight-gradient operation updates the weights */
     ALEXNET_FLAG_NO_CTA_PAIRS = 16,    /* convolution forward / backward-data never run as clusters of two CTAs */
-    ALEXNET_FLAG_ALL_CTA_PAIRS = 32    /* ... always do (default: per layer, where the cost model expects a gain);
+    ALEXNET_FLAG_ALL_CTA_PAIRS = 32,   /* ... always do (default: per layer, where the cost model expects a gain);
                                         * results do not depend on either flag beyond fp32 summation order */
+    ALEXNET_FLAG_SHARED_REPLICA_WEIGHTS = 64 /* replicas == 2: both replicas use ONE copy of parameters, momentum and their bf16
+                                        * forms.  Valid for the paper's scheme because the replicas are equal at the start of
+                                        * every iteration (same initialisation; every exchange makes them equal again).  An
+                                        * iteration is then alexnet_forward_backward on both replicas followed by
+                                        * alexnet_update_and_average, which applies each replica's update to the shared state
+                                        * and stores the average: the same arithmetic and bits as with two copies, 26 bytes of
+                                        * parameter traffic per index instead of 44, and 14 bytes per parameter less memory.
+                                        * alexnet_train_step and alexnet_apply_update return STATE (they would let one replica
+                                        * run ahead of the other); alexnet_replica_average is a no-op; get/set_params address
+                                        * the one copy through either replica index */
 };
 
 typedef struct {

@@ -15,7 +15,7 @@ from . import build as _build
 
 OK, ERR_ARG, ERR_CUDA, ERR_STATE, ERR_DEVICE_TIMEOUT, ERR_NOMEM = 0, -1, -2, -3, -4, -5
 FLAG_LRN_ALPHA_DIV_N, FLAG_WD_ON_BIASES, FLAG_INVERTED_DROPOUT, FLAG_FUSED_FC_UPDATE = 1, 2, 4, 8
-FLAG_NO_CTA_PAIRS, FLAG_ALL_CTA_PAIRS = 16, 32
+FLAG_NO_CTA_PAIRS, FLAG_ALL_CTA_PAIRS, FLAG_SHARED_REPLICA_WEIGHTS = 16, 32, 64
 
 TENSORS = ["CROPFLIP", "X0", "A1", "N1", "P1", "ARG1", "A2", "N2", "P2", "ARG2", "A3", "A4", "A5", "P5", "ARG5",
            "F6", "F7", "Z", "M6", "M7", "DZ", "DF7", "DF6", "DP5", "DA5", "DA4", "DA3", "DP2", "DN2", "DA2",

@@ -256,8 +256,14 @@ size_t carve(alexnet* h, uint8_t* base) {
     h->status = c.take<int>(16);
     for (int r = 0; r < h->cfg.replicas; ++r) {
         Replica& R = h->rep[r];
-        R.w = c.take<float>(L.n_total); R.v = c.take<float>(L.n_total); R.g = c.take<float>(L.n_total);
-        R.shadow = c.take<bf16>(L.n_total); R.wt = c.take<bf16>(L.wt_total);
+        if (r == 1 && (h->cfg.flags & ALEXNET_FLAG_SHARED_REPLICA_WEIGHTS)) {
+            // one copy of parameters, momentum and their bf16 forms for both replicas; gradients stay per replica
+            R.w = h->rep[0].w; R.v = h->rep[0].v; R.shadow = h->rep[0].shadow; R.wt = h->rep[0].wt;
+            R.g = c.take<float>(L.n_total);
+        } else {
+            R.w = c.take<float>(L.n_total); R.v = c.take<float>(L.n_total); R.g = c.take<float>(L.n_total);
+            R.shadow = c.take<bf16>(L.n_total); R.wt = c.take<bf16>(L.wt_total);
+        }
         for (int s = 0; s < 2; ++s) {
             R.stage[s] = c.take<uint8_t>((size_t)B * 196608);
             R.labels[s] = c.take<int32_t>(B);
@@ -835,6 +841,13 @@ void op_update_average(alexnet* h, cudaStream_t st) {
     Replica &A = h->rep[0], &Bq = h->rep[1];
     const Layout& L = h->L;
     const long long nd = (h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES) ? L.n_total : L.n_weights;
+    if (A.w == Bq.w) {      // shared copy
+        launch_k(kn::sgd_update_average_shared_kernel, 1184, 256, 0, st, A.w, A.v, A.g, Bq.g, A.shadow, L.n_total / 4, nd / 4,
+                 h->cfg.lr, h->cfg.momentum, h->cfg.weight_decay);
+        h->launches++;
+        refresh_shadows(h, 0, false, st);
+        return;
+    }
     launch_k(kn::sgd_update_average_kernel, 1184, 256, 0, st, A.w, A.v, A.g, Bq.w, Bq.v, Bq.g, A.shadow, Bq.shadow, L.n_total / 4,
              nd / 4, h->cfg.lr, h->cfg.momentum, h->cfg.weight_decay);
     h->launches++;
@@ -1157,9 +1170,13 @@ int alexnet_load_batch_async(alexnet_t* h, int replica, const uint8_t* images, c
     return ALEXNET_OK;
 }
 
+static bool shared_weights(const alexnet_t* h) { return h->cfg.replicas == 2 && (h->cfg.flags & ALEXNET_FLAG_SHARED_REPLICA_WEIGHTS); }
+
 static int step_impl(alexnet_t* h, int replica, float* host_loss, bool with_update) {
     if (!h) return ALEXNET_ERR_ARG;
     if (replica < 0 || replica >= h->cfg.replicas) return fail(h, ALEXNET_ERR_ARG, "train_step: bad replica");
+    if (with_update && shared_weights(h))
+        return fail(h, ALEXNET_ERR_STATE, "train_step: the replicas share one copy of the parameters; use alexnet_forward_backward on both and alexnet_update_and_average");
     if (int rc = check_status(h)) return rc;
     Replica& R = h->rep[replica];
     if (R.loaded == 0) return fail(h, ALEXNET_ERR_STATE, "train_step: no loaded batch");
@@ -1189,6 +1206,7 @@ int alexnet_apply_update(alexnet_t* h, int replica, float grad_scale) {
         return fail(h, ALEXNET_ERR_ARG, "apply_update: bad argument");
     if (int rc = check_status(h)) return rc;
     Replica& R = h->rep[replica];
+    if (shared_weights(h)) return fail(h, ALEXNET_ERR_STATE, "apply_update: the replicas share one copy of the parameters; use alexnet_update_and_average");
     if (!R.grad_pending) return fail(h, ALEXNET_ERR_STATE, "apply_update: no pending gradient (call alexnet_forward_backward first)");
     op_update(h, replica, h->cs, true, grad_scale);
     R.grad_pending = false;
@@ -1223,6 +1241,7 @@ int alexnet_scale_and_refresh(alexnet_t* h, int replica, float scale) {
     if (!h) return ALEXNET_ERR_ARG;
     if (replica < 0 || replica >= h->cfg.replicas || !(scale == scale)) return fail(h, ALEXNET_ERR_ARG, "scale_and_refresh: bad argument");
     if (int rc = check_status(h)) return rc;
+    if (shared_weights(h) && replica == 1) return ALEXNET_OK;      // replica 0's call has done the shared copy
     op_scale_refresh(h, replica, scale, h->cs);
     CK(cudaGetLastError());
     return ALEXNET_OK;
@@ -1242,6 +1261,7 @@ int alexnet_average_received(alexnet_t* h, int replica, const float* const* dev_
     if (replica < 0 || replica >= h->cfg.replicas || count < 1 || count > 8 || self < 0 || self >= count || !dev_w || !dev_v)
         return fail(h, ALEXNET_ERR_ARG, "average_received: bad argument (1 <= count <= 8, 0 <= self < count)");
     if (int rc = check_status(h)) return rc;
+    if (shared_weights(h) && replica == 1) return ALEXNET_OK;      // replica 0's call has done the shared copy
     Replica& R = h->rep[replica];
     kn::RecvList rl{};
     rl.count = count;
@@ -1313,7 +1333,7 @@ int alexnet_eval_batch(alexnet_t* h, int replica, const uint8_t* images, const i
 int alexnet_replica_average(alexnet_t* h) {
     if (!h) return ALEXNET_ERR_ARG;
     if (int rc = check_status(h)) return rc;
-    if (h->cfg.replicas < 2) return ALEXNET_OK;
+    if (h->cfg.replicas < 2 || shared_weights(h)) return ALEXNET_OK;     // one copy: nothing to average
     op_average(h, h->cs);
     CK(cudaGetLastError());
     return ALEXNET_OK;
@@ -1440,6 +1460,8 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
         return fail(h, ALEXNET_ERR_ARG, "run_op: bad argument");
     if ((op == ALEXNET_OP_AVERAGE || op == ALEXNET_OP_UPDATE_AVERAGE) && h->cfg.replicas < 2)
         return fail(h, ALEXNET_ERR_ARG, "run_op: average needs two replicas");
+    if (shared_weights(h) && (op == ALEXNET_OP_AVERAGE || op == ALEXNET_OP_UPDATE))
+        return fail(h, ALEXNET_ERR_STATE, "run_op: not while the replicas share one copy of the parameters");
     if (int rc = check_status(h)) return rc;
     Replica& R = h->rep[replica];
     const int slot = R.last_slot;

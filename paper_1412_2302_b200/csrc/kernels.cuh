@@ -811,6 +811,31 @@ __global__ void __launch_bounds__(256) sgd_update_average_kernel(float* __restri
         ((uint2*)sa)[i] = s; ((uint2*)sb)[i] = s;
     }
 }
+// The same for two replicas that SHARE one copy of parameters and momentum (they are identical at the start of every
+// iteration: identical initialisation, and every exchange makes them equal again, so one copy holds both): each replica's
+// update starts from the shared (w, v) with its own gradient, the averages go back to the shared arrays.  Same arithmetic in
+// the same order as above, hence the same bits; 16 bytes read and 10 written per index (26 instead of 44).
+__global__ void __launch_bounds__(256) sgd_update_average_shared_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ ga,
+                                                                        const float* __restrict__ gb, __nv_bfloat16* __restrict__ shadow,
+                                                                        long long n4, long long n_decay4, float lr, float mu, float wd) {
+    pdl_sync();
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 a = ((const float4*)w)[i], c = ((const float4*)v)[i];
+        float4 b = a, e = c;
+        const float4 g0 = ld_stream(ga + 4 * i), g1 = ld_stream(gb + 4 * i);
+        const float d = i < n_decay4 ? lr * wd : 0.f;
+        sgd_step(a.x, c.x, g0.x, d, lr, mu); sgd_step(a.y, c.y, g0.y, d, lr, mu);
+        sgd_step(a.z, c.z, g0.z, d, lr, mu); sgd_step(a.w, c.w, g0.w, d, lr, mu);
+        sgd_step(b.x, e.x, g1.x, d, lr, mu); sgd_step(b.y, e.y, g1.y, d, lr, mu);
+        sgd_step(b.z, e.z, g1.z, d, lr, mu); sgd_step(b.w, e.w, g1.w, d, lr, mu);
+        const float4 wn = make_float4(0.5f * (a.x + b.x), 0.5f * (a.y + b.y), 0.5f * (a.z + b.z), 0.5f * (a.w + b.w));
+        const float4 vn = make_float4(0.5f * (c.x + e.x), 0.5f * (c.y + e.y), 0.5f * (c.z + e.z), 0.5f * (c.w + e.w));
+        ((float4*)w)[i] = wn; ((float4*)v)[i] = vn;
+        __nv_bfloat162 lo = __floats2bfloat162_rn(wn.x, wn.y), hi = __floats2bfloat162_rn(wn.z, wn.w);
+        ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo, *(uint32_t*)&hi);
+    }
+}
 // After an all-reduce(sum) of parameters and momentum over R replicas on R GPUs: w <- scale w, v <- scale v (scale = 1/R:
 // the average) and the bf16 copy of w: 8 bytes read and 10 written per index.
 __global__ void __launch_bounds__(256) scale_refresh_kernel(float* __restrict__ w, float* __restrict__ v,

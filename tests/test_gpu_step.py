@@ -467,33 +467,43 @@ def test_batch128_whole_batch_fused_update_against_oracle(record_property):
 
 def test_config4_two_replicas_ten_exchanges_batch128():
     """Two replicas x batch 128, identically initialised: 10 x (2 loads, 2 steps, 1 exchange-and-average).  Replicas are
-    bitwise identical after every exchange, and (second pass) the one-pass update + average on deferred gradients gives
-    bit for bit the same parameters as two updates followed by replica_average."""
+    bitwise identical after every exchange, and the one-pass update + average on deferred gradients, with two copies of the
+    parameters or with one shared copy, gives bit for bit the same parameters as two updates followed by replica_average."""
+    from paper_1412_2302_b200 import alexnet as A
     seed, B = BASE + 4, 128
     w = synth.init_params(seed)
     batches = [[(torch.from_numpy(synth.images(seed, r, s % 2, B)).pin_memory(),
                  torch.from_numpy(synth.labels(seed, r, s % 2, B)).pin_memory()) for r in (0, 1)] for s in range(2)]
     results = []
-    for fused in (False, True):
-        net = make(B, replicas=2, seed=seed)
-        net.set_params(w, 0); net.set_params(w, 1)
+    for form in ("separate", "one_pass", "shared"):
+        net = make(B, replicas=2, seed=seed, flags=A.FLAG_SHARED_REPLICA_WEIGHTS if form == "shared" else 0)
+        net.set_params(w, 0)
+        if form != "shared":
+            net.set_params(w, 1)
         for step in range(10):
             for r in (0, 1):
                 net.load_batch_async(r, *batches[step % 2][r], step)
-            if fused:
-                net.forward_backward(0); net.forward_backward(1)
-                net.update_and_average()
-            else:
+            if form == "separate":
                 net.train_step(0); net.train_step(1)
                 net.replica_average()
+            else:
+                net.forward_backward(0); net.forward_backward(1)
+                net.update_and_average()
             net.sync()
             va, vb = net.param_views(0)[1], net.param_views(1)[1]
             wa, wb = net.param_views(0)[0], net.param_views(1)[0]
             assert torch.equal(wa, wb) and torch.equal(va, vb), step
+            assert (wa.data_ptr() == wb.data_ptr()) == (form == "shared")
         results.append((net.get_params(0, 0), net.get_params(0, 1)))
         assert np.array_equal(results[-1][0], net.get_params(1, 0))
+        if form == "shared":
+            with pytest.raises(A.AlexNetError) as e:
+                net.train_step(0)
+            assert e.value.code == A.ERR_STATE
+            net.replica_average()                  # one copy: a no-op
         net.close()
-    assert np.array_equal(results[0][0], results[1][0]) and np.array_equal(results[0][1], results[1][1])
+    for other in results[1:]:
+        assert np.array_equal(results[0][0], other[0]) and np.array_equal(results[0][1], other[1])
     assert np.isfinite(results[0][0]).all() and not np.array_equal(results[0][0], w)
 
 
