@@ -729,3 +729,39 @@ def test_batch256_sampled_layers_and_weight_gradients():
     bad = {k: v for k, v in gerr.items() if not v < 1e-3}          # exact bf16 inputs, fp32 accumulation: summation order only
     assert not bad, (bad, gerr)
     net.close()
+
+
+def test_batch1024_largest_configuration_sampled_forward():
+    """The largest batch the configuration check admits (1024: 3.3 million grid rows in conv1, activation tensors of up
+    to 640 MB, a 15 GB arena): one step runs, the first and the last image are followed through the forward pass by the
+    oracle on the tensors that are small enough to fetch (they depend on every layer below), and gradients are finite."""
+    seed, B = BASE + 6, 1024
+    net = make(B, seed=seed)
+    w = synth.init_params(seed, variance_preserving=True, bias=0.1)
+    net.set_params(w)
+    rng = np.random.default_rng(seed)
+    img = torch.from_numpy(rng.integers(0, 256, size=(B, 256, 256, 3), dtype=np.uint8)).pin_memory()
+    lab = torch.from_numpy(rng.integers(0, 1000, size=(B,), dtype=np.int32)).pin_memory()
+    net.load_batch_async(0, img, lab, 0)
+    loss = net.forward_backward(0, want_loss=True)
+    pick = [0, B - 1]
+    onet = O.OracleNet(O.OracleConfig(seed=seed), w.astype(np.float64))
+    kw = dict(cf=O.crop_flip(seed, 0, 0, B)[pick], m6=O.dropout_mask(seed, 2, 0, 0, B, 4096, 0.5)[pick],
+              m7=O.dropout_mask(seed, 3, 0, 0, B, 4096, 0.5)[pick], mean_over=B)
+    T = onet.forward_backward(img.numpy()[pick], lab.numpy()[pick], synth.mean_image(seed), 0, **kw)
+    assert np.array_equal(net.get_tensor("CROPFLIP").reshape(B, 3).astype(np.int32)[pick], kw["cf"])
+    errs = {}
+    for k in ("a5", "p5", "f6", "f7", "z", "dz"):
+        errs[k] = rel(net.get_tensor(k.upper()).reshape((B,) + T[k].shape[1:])[pick], T[k])
+    bad = {k: v for k, v in errs.items() if not v < TOL}
+    assert not bad, (bad, errs)
+    # the mean loss over 1024 images of a net with near-uniform predictions, and a finite, non-zero gradient everywhere
+    ln = net.get_tensor("LOSS")
+    assert abs(ln.mean() - loss) < 1e-4 * abs(loss) and np.isfinite(ln).all()
+    g = net.param_views(0)[2]
+    off, _ = O.param_offsets()
+    gc = net.get_params(0, 2)
+    assert bool(torch.isfinite(g).all())
+    for k, (o, n, _) in off.items():
+        assert np.abs(gc[o:o + n]).max() > 0, k
+    net.close()
