@@ -21,7 +21,9 @@ stream); the median region is reported, the spread is in `repeats`.
 With N > 1 GPUs every rank holds one replica on its own GPU and every step ends
 with the paper's exchange between replicas over NCCL (gradient form: all-reduce
 of the gradients, then one update with their mean; --exchange params runs the
-literal form: update, all-reduce of weights and momentum, scale).  `python
+literal form: update, all-reduce of weights and momentum, scale; --exchange
+grads_overlap issues the all-reduce of the FC gradients under the rest of the
+backward pass).  `python
 bench.py --gpus N` starts the N ranks itself; under torchrun it joins them.
 With --impl reference the CPU checker is the thing being timed.
 """
@@ -249,7 +251,8 @@ def run_ours(args, rank, world, local_rank):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     seed = synth.BASE_SEED + 3
-    grads_form = world > 1 and args.exchange == "grads"
+    grads_form = world > 1 and args.exchange in ("grads", "grads_overlap")
+    comm_stream = torch.cuda.Stream(dev) if args.exchange == "grads_overlap" else None
     # one GPU: the FC weight-gradient kernel applies the momentum update in its epilogue (bit-identical parameters, see the
     # tests).  Several GPUs, gradient form: the gradients are stored, all-reduced, and applied by one update pass.
     net = AlexNet(batch=BATCH, replicas=1, seed=seed, mean_image=synth.mean_image(seed), device=str(dev),
@@ -270,7 +273,10 @@ def run_ours(args, rank, world, local_rank):
             net.train_step(0, want_loss=False)
         elif grads_form:
             net.forward_backward(0)
-            exchange.allreduce_gradients_and_update(rep)
+            if comm_stream is not None:
+                exchange.allreduce_gradients_overlapped_and_update(rep, comm_stream)
+            else:
+                exchange.allreduce_gradients_and_update(rep)
         else:
             net.train_step(0, want_loss=False)
             exchange.exchange_and_average(rep)
@@ -418,7 +424,8 @@ def run_ours(args, rank, world, local_rank):
                        "timing": f"median of {R} timed regions of {K} steps each",
                        "parallelism": ("single GPU" if world == 1 else
                                        f"one replica per GPU; every step ends with the exchange between replicas over NCCL ("
-                                       + ("all-reduce of the gradients, one update with their mean"
+                                       + (("all-reduce of the gradients, one update with their mean"
+                                           + (", the FC gradients exchanged under the convolution backward pass" if comm_stream is not None else ""))
                                           if grads_form else "update, all-reduce of weights and momentum, scale by 1/N") + ")")},
             "repeats": rep_value,
             "e2e": {"value": imgs / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": BATCH * 196608 + BATCH * 4,
@@ -472,7 +479,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--repeats", type=int, default=5)
-    ap.add_argument("--exchange", default="grads", choices=["grads", "params"])
+    ap.add_argument("--exchange", default="grads", choices=["grads", "grads_overlap", "params"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

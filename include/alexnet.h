@@ -217,6 +217,23 @@ int alexnet_update_and_average(alexnet_t* h);
  * parameters into the arrays itself.  Asynchronous, on the compute stream. */
 int alexnet_param_regions(alexnet_t* h, int replica, float** dev_w, float** dev_v, float** dev_g, size_t* n_floats);
 
+/* Overlapping the exchange of gradients with the backward pass.  In the arrays
+ * of alexnet_param_regions the weights of the three FC layers (96% of all
+ * parameters) are the contiguous range [*fc_weights_begin, *fc_weights_end)
+ * (in floats; the convolution filters lie before it, all biases after it), and
+ * their gradients are complete early in the backward pass, while the
+ * convolution layers' backward pass is still to run.
+ * alexnet_stream_wait_fc_gradients makes `stream` (a cudaStream_t of the
+ * caller, e.g. the one it issues its all-reduce from) wait, on the device,
+ * until the FC weight gradients of the backward pass issued last by
+ * alexnet_forward_backward are written; work queued on `stream` afterwards
+ * then runs beside the rest of that backward pass.  (When that pass kept
+ * everything on the compute stream, i.e. with per-kernel timing on, the wait
+ * is for the whole pass.)  The caller orders its stream back before
+ * alexnet_apply_update.  Errors: ARG, DEVICE_TIMEOUT, CUDA. */
+int alexnet_param_layout(const alexnet_t* h, size_t* fc_weights_begin, size_t* fc_weights_end, size_t* n_floats);
+int alexnet_stream_wait_fc_gradients(alexnet_t* h, void* stream);
+
 /* The paper's own form of the exchange (the data-parallel figure: step 2, each
  * GPU copies the other's weights, biases and momentum into receive buffers of
  * its own; step 3, it averages them with its own): the caller has brought the

@@ -37,7 +37,8 @@ EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "
            "alexnet_launch_count", "alexnet_profile", "alexnet_profile_read", "alexnet_sync", "alexnet_last_error", "alexnet_bias_grad_noalloc", "alexnet_loader_ring_bytes",
            "alexnet_loader_create", "alexnet_loader_next", "alexnet_loader_release", "alexnet_loader_destroy",
            "alexnet_forward_backward", "alexnet_apply_update", "alexnet_update_and_average", "alexnet_param_regions",
-           "alexnet_scale_and_refresh", "alexnet_create_error", "alexnet_debug_expire_wait", "alexnet_set_color_augmentation", "alexnet_average_received"]
+           "alexnet_scale_and_refresh", "alexnet_create_error", "alexnet_debug_expire_wait", "alexnet_set_color_augmentation", "alexnet_average_received", "alexnet_param_layout",
+           "alexnet_stream_wait_fc_gradients"]
 
 
 class Config(ctypes.Structure):
@@ -86,6 +87,8 @@ def load_library():
     L.alexnet_debug_expire_wait.argtypes = [vp, ctypes.c_longlong]
     L.alexnet_set_color_augmentation.argtypes = [vp, vp, vp, ctypes.c_float]
     L.alexnet_average_received.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), i32, i32]
+    L.alexnet_param_layout.argtypes = [vp, ctypes.POINTER(sz), ctypes.POINTER(sz), ctypes.POINTER(sz)]
+    L.alexnet_stream_wait_fc_gradients.argtypes = [vp, vp]
     L.alexnet_eval_batch.argtypes = [vp, i32, vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                                      ctypes.POINTER(ctypes.c_float)]
     L.alexnet_get_params.argtypes = [vp, i32, i32, vp, sz]
@@ -230,6 +233,16 @@ class AlexNet:
             pv[r] = None if r == self_rank or recv_v[r] is None else recv_v[r].data_ptr()
         self._keep = self._keep[-8:] + [(recv_w, recv_v)]
         self._ck(self.lib.alexnet_average_received(self.h, replica, pw, pv, n, int(self_rank)))
+
+    def fc_range(self):
+        """(begin, end) of the FC weights inside the arrays of param_views, in floats."""
+        b, e = ctypes.c_size_t(), ctypes.c_size_t()
+        self._ck(self.lib.alexnet_param_layout(self.h, ctypes.byref(b), ctypes.byref(e), None))
+        return int(b.value), int(e.value)
+
+    def stream_wait_fc_gradients(self, stream):
+        """Make `stream` (a torch.cuda.Stream) wait until the FC weight gradients of the backward pass issued last exist."""
+        self._ck(self.lib.alexnet_stream_wait_fc_gradients(self.h, ctypes.c_void_p(stream.cuda_stream)))
 
     def param_views(self, replica=0):
         """(w, v, g): fp32 torch views of the replica's parameter, momentum and gradient arrays inside the arena (the

@@ -161,6 +161,9 @@ struct alexnet {
     cudaStream_t side[kBranches] = {};
     cudaEvent_t ev_side_done[kBranches] = {};
     cudaEvent_t ev_fork[kBranches] = {};   // the inputs of branch b are ready on the compute stream
+    bool fc_grads_on_branches = false;     // the last backward pass ran the FC weight gradients on branches 0-2: ev_side_done[0..2]
+                                           // then complete as soon as those gradients exist, long before the pass ends
+    cudaEvent_t ev_backward_done = nullptr;   // recorded on the compute stream after every backward pass
     size_t ws_conv_off[5] = {};            // floats: each conv layer's split partials have their own region of the workspace
     float* bias_partial = nullptr;         // [5][kBiasPartial] bias-gradient partials of the conv weight-gradient kernels
     uint8_t* arena; size_t arena_bytes;
@@ -928,6 +931,8 @@ void forward_backward(alexnet* h, int r, int slot, cudaStream_t st, bool plain_f
             cudaEventRecord(h->ev_side_done[b], h->side[b]);
             cudaStreamWaitEvent(st, h->ev_side_done[b], 0);
         }
+    h->fc_grads_on_branches = used[0] && used[1] && used[2] && !fused;
+    if (h->ev_backward_done) cudaEventRecord(h->ev_backward_done, st);
 }
 
 int check_status(alexnet* h) {
@@ -1042,6 +1047,7 @@ void teardown(alexnet* h) {
         if (h->ev_fork[b]) cudaEventDestroy(h->ev_fork[b]);
     }
     for (cudaEvent_t e : h->prof_ev) cudaEventDestroy(e);
+    if (h->ev_backward_done) cudaEventDestroy(h->ev_backward_done);
     for (int r = 0; r < h->cfg.replicas; ++r)
         for (int s = 0; s < 2; ++s) {
             if (h->rep[r].ready[s]) cudaEventDestroy(h->rep[r].ready[s]);
@@ -1118,6 +1124,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
         CKC(cudaEventCreateWithFlags(&h->ev_side_done[b], cudaEventDisableTiming));
         CKC(cudaEventCreateWithFlags(&h->ev_fork[b], cudaEventDisableTiming));
     }
+    CKC(cudaEventCreateWithFlags(&h->ev_backward_done, cudaEventDisableTiming));
     // pad positions of every grid must be zero from the start; gradients and momentum start at zero
     CKC(cudaMemsetAsync(h->arena, 0, need, h->cs));
     if (host_mean_image) CKC(cudaMemcpyAsync(h->mean, host_mean_image, 256 * 256 * 3 * sizeof(float), cudaMemcpyHostToDevice, h->cs));
@@ -1234,6 +1241,26 @@ int alexnet_param_regions(alexnet_t* h, int replica, float** dev_w, float** dev_
     if (dev_v) *dev_v = R.v;
     if (dev_g) *dev_g = R.g;
     if (n_floats) *n_floats = (size_t)h->L.n_total;
+    return ALEXNET_OK;
+}
+
+int alexnet_param_layout(const alexnet_t* h, size_t* fc_weights_begin, size_t* fc_weights_end, size_t* n_floats) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (fc_weights_begin) *fc_weights_begin = (size_t)h->L.fc[0].w_off;
+    if (fc_weights_end) *fc_weights_end = (size_t)h->L.n_weights;
+    if (n_floats) *n_floats = (size_t)h->L.n_total;
+    return ALEXNET_OK;
+}
+
+int alexnet_stream_wait_fc_gradients(alexnet_t* h, void* stream) {
+    if (!h) return ALEXNET_ERR_ARG;
+    if (int rc = check_status(h)) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (h->fc_grads_on_branches) {
+        for (int b = 0; b < 3; ++b) CK(cudaStreamWaitEvent(st, h->ev_side_done[b], 0));
+    } else {
+        CK(cudaStreamWaitEvent(st, h->ev_backward_done, 0));
+    }
     return ALEXNET_OK;
 }
 

@@ -16,6 +16,11 @@ section; checked to 1e-5 in the tests):
   allreduce_gradients_and_update(rep)  after forward_backward: all-reduce g (4 bytes per parameter), then one update
                                        with the mean gradient
 
+  allreduce_gradients_overlapped_and_update(rep, comm_stream)
+                                       the gradient form with the all-reduce of the FC weight gradients (96% of the
+                                       bytes) issued from a second stream as soon as they exist, under the convolution
+                                       layers' backward pass; only the rest is exchanged after the pass
+
 `rep` is anything with param_views() -> (w, v, g) torch tensors, scale_and_refresh(scale) and apply_update(scale):
 LocalReplica adapts an AlexNet handle; the CPU tests pass a stand-in that holds host tensors.
 """
@@ -47,6 +52,15 @@ class LocalReplica:
 
     def average_received(self, recv_w, recv_v, self_rank):
         self.net.average_received(self.replica, recv_w, recv_v, self_rank)
+
+    def fc_range(self):
+        return self.net.fc_range()
+
+    def stream_wait_fc_gradients(self, stream):
+        self.net.stream_wait_fc_gradients(stream)
+
+    def wait_stream(self, stream):
+        self.net.compute_stream.wait_stream(stream)
 
 
 class _NoStream:
@@ -102,6 +116,26 @@ def allreduce_gradients_and_update(rep, group=None):
     with (rep.stream() if hasattr(rep, "stream") else _NoStream()):
         if _initialised():
             dist.all_reduce(g, op=dist.ReduceOp.SUM, group=group)
+        rep.apply_update(1.0 / world)
+
+
+def allreduce_gradients_overlapped_and_update(rep, comm_stream, group=None):
+    """Call right after forward_backward has been issued.  The all-reduce of the FC weight gradients is queued on
+    comm_stream behind a device-side wait for those gradients and runs beside the rest of the backward pass; the
+    convolution and bias gradients are all-reduced from the compute stream after the pass; then one update with the mean
+    gradient.  Every rank issues the same collectives in the same order."""
+    world = _world(group)
+    _, _, g = rep.param_views()
+    b, e = rep.fc_range()
+    rep.stream_wait_fc_gradients(comm_stream)
+    with (torch.cuda.stream(comm_stream) if comm_stream is not None else _NoStream()):
+        if _initialised():
+            dist.all_reduce(g[b:e], op=dist.ReduceOp.SUM, group=group)
+    with (rep.stream() if hasattr(rep, "stream") else _NoStream()):
+        if _initialised():
+            dist.all_reduce(g[:b], op=dist.ReduceOp.SUM, group=group)
+            dist.all_reduce(g[e:], op=dist.ReduceOp.SUM, group=group)
+        rep.wait_stream(comm_stream)
         rep.apply_update(1.0 / world)
 
 

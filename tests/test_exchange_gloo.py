@@ -42,6 +42,15 @@ class HostReplica:
         self.w.copy_(sw * (1.0 / n)); self.v.copy_(sv * (1.0 / n))
         self.refreshed += 1
 
+    def fc_range(self):
+        return 1000, 3500                               # any split of the vector into three ranges
+
+    def stream_wait_fc_gradients(self, stream):
+        pass
+
+    def wait_stream(self, stream):
+        pass
+
     def apply_update(self, grad_scale):
         assert self.pending
         self.v.mul_(MU).add_(self.w, alpha=-LR * WD).add_(self.g * grad_scale, alpha=-LR)
@@ -78,6 +87,10 @@ def _worker(rank, world, port, out):
         # gradient form: all-reduce the gradients, one update with their mean
         b = HostReplica(w, v, g)
         exchange.allreduce_gradients_and_update(b)
+        # the gradient form with the large range exchanged apart (on a GPU: from a second stream, under the backward pass)
+        d = HostReplica(w, v, g)
+        exchange.allreduce_gradients_overlapped_and_update(d, None)
+        assert torch.equal(d.w, b.w) and torch.equal(d.v, b.v)
         # the figure's own two steps: receive the other replica's arrays, then average
         c = HostReplica(w, v, g)
         c.apply_update(1.0)

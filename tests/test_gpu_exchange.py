@@ -46,6 +46,13 @@ def test_one_rank_nccl_exchange_equals_local_paths(nccl_group):
             elif mode == "params":
                 losses.append(net.train_step(0, want_loss=True))
                 exchange.exchange_and_average(rep)
+            elif mode == "overlap":
+                losses.append(None)
+                net.forward_backward(0)
+                exchange.allreduce_gradients_overlapped_and_update(rep, state.setdefault("comm", torch.cuda.Stream()))
+                buf = state.setdefault("loss", torch.zeros(1).pin_memory())
+                net.loss_async(0, buf); net.sync()
+                losses[-1] = float(buf[0])
             elif mode == "gather":
                 losses.append(net.train_step(0, want_loss=True))
                 state["buffers"] = exchange.exchange_then_average(rep, buffers=state.get("buffers"))
@@ -57,8 +64,8 @@ def test_one_rank_nccl_exchange_equals_local_paths(nccl_group):
         net.close()
         return out
 
-    plain, params, grads, gather = run("plain"), run("params"), run("grads"), run("gather")
-    for other in (params, grads, gather):
+    plain, params, grads, gather, overlap = run("plain"), run("params"), run("grads"), run("gather"), run("overlap")
+    for other in (params, grads, gather, overlap):
         assert other[0] == plain[0]
         assert np.array_equal(other[1], plain[1]) and np.array_equal(other[2], plain[2])
     assert not np.array_equal(plain[1], w)
