@@ -666,7 +666,7 @@ void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
     h->launches++;
 }
 void colsum(alexnet* h, const bf16* dy, long long rows, int C, float* db, cudaStream_t st) {
-    if (C % 8) {
+    if (C % 8 || rows < 512) {     // few rows: one thread per column, one launch (the two-stage form would use a single split)
         launch_k(kn::colsum_scalar_kernel, nblk(C, 128), 128, 0, st, dy, (int)rows, C, db);
         h->launches++;
         return;
@@ -704,11 +704,12 @@ void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
              R.g + c.w_off, l == 0, h->bias_partial + (size_t)l * kBiasPartial, c.cout, R.g + c.b_off);
     h->launches++;
 }
-void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool eval = false) {
+void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool eval = false, bool gemm_only = false) {
     Replica& R = h->rep[r];
     const FcL& f = h->L.fc[l];
     const Plan& P = R.fc_fwd[l];
     launch_gemm(h, P, st);
+    if (gemm_only) return;     // the split reduction is part of the kernel that follows (fc8 inside the step)
     const long long total = (long long)h->B * f.N;
     bf16* outs[3] = {R.f6, R.f7, nullptr};
     uint8_t* keeps[3] = {R.m6, R.m7, nullptr};
@@ -826,6 +827,15 @@ void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
     launch_k(kn::mean_kernel, 1, 256, 0, st, R.loss_n, h->B, R.loss);
     h->launches += 2;
 }
+// fc8's split reduction + bias, softmax cross-entropy and the mean loss in one launch (the step's form; N <= 1024)
+void op_fc8_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
+    Replica& R = h->rep[r];
+    const FcL& f = h->L.fc[2];
+    const Plan& P = R.fc_fwd[2];
+    launch_k(kn::fc8_softmax_xent_kernel, h->B, 256, 0, st, h->ws, P.c.splits, P.c.split_stride, R.w + f.b_off, R.z, R.labels[slot], R.dz,
+             R.loss_n, R.loss, h->status + 8, h->B, f.N);
+    h->launches++;
+}
 void op_update(alexnet* h, int r, cudaStream_t st, bool full = false, float gscale = 1.f) {
     Replica& R = h->rep[r];
     const Layout& L = h->L;
@@ -833,8 +843,17 @@ void op_update(alexnet* h, int r, cudaStream_t st, bool full = false, float gsca
     // internal order: conv filters, FC weights, biases.  The conv filters (with their transposed bf16 copies) have a tiled
     // kernel of their own; the one-pass kernel takes the rest, minus the FC weights when the fused FC update has done them.
     const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0 && !full;
-    launch_k(kn::sgd_update_conv_kernel, L.tjobs.tile0[5], 256, 0, st, R.w, R.v, R.g, R.shadow, h->cfg.lr * h->cfg.weight_decay,
-             h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs, gscale);
+    const float d = h->cfg.lr * h->cfg.weight_decay;
+    if (fused && nd == L.n_weights) {
+        // only the biases are left beside the conv filters: extra blocks of the filter kernel take them (no decay on biases)
+        const long long b4 = L.n_weights / 4, e4 = L.n_total / 4;
+        launch_k(kn::sgd_update_conv_kernel, L.tjobs.tile0[5] + nblk(e4 - b4, 256), 256, 0, st, R.w, R.v, R.g, R.shadow, d,
+                 h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs, gscale, b4, e4, 0.f);
+        h->launches++;
+        return;
+    }
+    launch_k(kn::sgd_update_conv_kernel, L.tjobs.tile0[5], 256, 0, st, R.w, R.v, R.g, R.shadow, d,
+             h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs, gscale, 0LL, 0LL, 0.f);
     launch_k(kn::sgd_update_kernel, fused ? 148 : 1184, 256, 0, st, R.w, R.v, R.g, R.shadow, (fused ? L.n_weights : L.fc[0].w_off) / 4,
              L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum, h->cfg.weight_decay, gscale);
     h->launches += 2;
@@ -890,8 +909,8 @@ void forward(alexnet* h, int r, int slot, cudaStream_t st, bool eval) {
     op_conv_fwd(h, r, 1, slot, st); op_lrn_pool_fwd(h, r, 1, st);
     op_conv_fwd(h, r, 2, slot, st); op_conv_fwd(h, r, 3, slot, st); op_conv_fwd(h, r, 4, slot, st);
     op_pool_fwd(h, r, 2, st);
-    op_fc_fwd(h, r, 0, step, st, eval); op_fc_fwd(h, r, 1, step, st, eval); op_fc_fwd(h, r, 2, step, st, eval);
-    op_softmax(h, r, slot, st);
+    op_fc_fwd(h, r, 0, step, st, eval); op_fc_fwd(h, r, 1, step, st, eval); op_fc_fwd(h, r, 2, step, st, eval, true);
+    op_fc8_softmax(h, r, slot, st);
 }
 void forward_backward(alexnet* h, int r, int slot, cudaStream_t st, bool plain_fc = false) {
     forward(h, r, slot, st, false);

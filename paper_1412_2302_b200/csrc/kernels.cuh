@@ -642,6 +642,70 @@ __global__ void softmax_xent_kernel(const float* __restrict__ z, const int32_t* 
     }
     if (tid == 0) loss_n[n] = -(zr[lab] - mx - logf(sum));
 }
+// The training step's form of the three kernels fc_reduce_fwd (fc8), softmax_xent and mean in one launch: block n adds the
+// split-K partials of its row of logits in split order, adds the bias, stores z (fp32 logits), then softmax, loss_n and dz as
+// above; the block that finishes last (a counter in global memory, reset for the next launch) averages loss_n in index order,
+// so the result does not depend on which block that is.  Same arithmetic as the separate kernels.
+__global__ void __launch_bounds__(256) fc8_softmax_xent_kernel(const float* __restrict__ ws, int splits, long long split_stride,
+                                                               const float* __restrict__ bias, float* __restrict__ z,
+                                                               const int32_t* __restrict__ labels, __nv_bfloat16* __restrict__ dz,
+                                                               float* __restrict__ loss_n, float* __restrict__ loss_mean,
+                                                               int* __restrict__ done_counter, int B, int N) {
+    pdl_sync();
+    __shared__ float red[32];
+    __shared__ float zs[1024];
+    __shared__ int last;
+    const int n = blockIdx.x, tid = threadIdx.x;
+    float mx = -INFINITY;
+    for (int j = tid; j < N; j += 256) {
+        const long long t = (long long)n * N + j;
+        float v = 0.f;
+        for (int q = 0; q < splits; ++q) v += ws[q * split_stride + t];
+        v += bias[j];
+        z[t] = v;
+        zs[j] = v;
+        mx = fmaxf(mx, v);
+    }
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(~0u, mx, o));
+    if ((tid & 31) == 0) red[tid >> 5] = mx;
+    __syncthreads();
+    mx = red[0];
+    for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
+    __syncthreads();
+    float sum = 0.f;
+    for (int j = tid; j < N; j += 256) sum += expf(zs[j] - mx);
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(~0u, sum, o);
+    if ((tid & 31) == 0) red[tid >> 5] = sum;
+    __syncthreads();
+    sum = 0.f;
+    for (int w = 0; w < 8; ++w) sum += red[w];
+    const int lab = labels[n];
+    const float inv = 1.f / sum, invB = 1.f / (float)B;
+    for (int j = tid; j < N; j += 256) {
+        const float pj = expf(zs[j] - mx) * inv;
+        dz[(size_t)n * N + j] = __float2bfloat16_rn((pj - (j == lab ? 1.f : 0.f)) * invB);
+    }
+    if (tid == 0) {
+        loss_n[n] = -(zs[lab] - mx - logf(sum));
+        __threadfence();
+        last = atomicAdd(done_counter, 1) == B - 1;
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    float s = 0.f;
+    for (int i = tid; i < B; i += 256) s += __ldcg(loss_n + i);
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(~0u, s, o);
+    __syncthreads();
+    if ((tid & 31) == 0) red[tid >> 5] = s;
+    __syncthreads();
+    if (tid == 0) {
+        float t = 0.f;
+        for (int w = 0; w < 8; ++w) t += red[w];
+        *loss_mean = t / (float)B;
+        *done_counter = 0;
+    }
+}
 __global__ void mean_kernel(const float* __restrict__ v, int n, float* __restrict__ out) {
     pdl_sync();
     __shared__ float red[32];
@@ -724,9 +788,28 @@ __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, 
 // [tap][cin][cog] (64-byte runs; a thread that walked the source order would write single elements).  Same arithmetic as sgd_update_kernel.
 __global__ void __launch_bounds__(256) sgd_update_conv_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g,
                                                               __nv_bfloat16* __restrict__ shadow, float d, float lr, float mu,
-                                                              __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs, float gscale) {
+                                                              __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs, float gscale,
+                                                              long long tail_begin4, long long tail_end4, float tail_d) {
     pdl_sync();
     __shared__ __nv_bfloat16 tile[32][36];       // [input channel][output channel], padded
+    if ((int)blockIdx.x >= jobs.tile0[jobs.n]) {
+        // blocks past the filter tiles: the plain update of the 16-byte vectors [tail_begin4, tail_end4) (the biases, when the
+        // FC weights have been updated by their weight-gradient kernels), sgd_update_kernel's arithmetic, one launch less
+        const long long i = tail_begin4 + (long long)((int)blockIdx.x - jobs.tile0[jobs.n]) * 256 + threadIdx.x;
+        if (i < tail_end4) {
+            float4 wv = ((float4*)w)[i], vv = ((float4*)v)[i];
+            const float4 gv = ((const float4*)g)[i];
+            sgd_step(wv.x, vv.x, gscale * gv.x, tail_d, lr, mu);
+            sgd_step(wv.y, vv.y, gscale * gv.y, tail_d, lr, mu);
+            sgd_step(wv.z, vv.z, gscale * gv.z, tail_d, lr, mu);
+            sgd_step(wv.w, vv.w, gscale * gv.w, tail_d, lr, mu);
+            ((float4*)w)[i] = wv;
+            ((float4*)v)[i] = vv;
+            __nv_bfloat162 lo2 = __floats2bfloat162_rn(wv.x, wv.y), hi2 = __floats2bfloat162_rn(wv.z, wv.w);
+            ((uint2*)shadow)[i] = make_uint2(*(uint32_t*)&lo2, *(uint32_t*)&hi2);
+        }
+        return;
+    }
     int q = 0;
     while (q + 1 < jobs.n && (int)blockIdx.x >= jobs.tile0[q + 1]) ++q;
     const TransposeJob J = jobs.j[q];
