@@ -539,6 +539,7 @@ int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* ws
     const int B = h->B;
     p.kh = p.kw = 1; p.cpg = 2; p.chunks = f.K / 64 / p.cpg; p.kk = 4;   // K is a multiple of 128 in all three layers
     p.MH = 1; p.BN = fc_fwd_bn(f); p.acc_stages = 2; p.cg = 1;
+    p.epi_sets = 2;     // one tile per CTA: its epilogue is never hidden behind a next tile, so two sets of warps share the four slabs
     p.M_total = B; p.m_tiles = (B + 127) / 128; p.n_tiles = (f.N + p.BN - 1) / p.BN;
     p.groups = 1; p.splits = fc_fwd_splits(f, B);
     p.asteps_total = p.chunks;
