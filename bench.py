@@ -138,7 +138,7 @@ def run_reference(args, rank, world):
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{args.steps} train steps of {sample} images each"},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-    }))
+    }), file=RESULT)
 
 
 def cpu_baseline():
@@ -248,10 +248,15 @@ def run_ours(args, rank, world, local_rank):
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    multi = world > 1 or args.force_exchange
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    elif args.force_exchange:
+        # self-check of the multi-GPU path on one GPU: a one-rank NCCL group, every step runs the exchange code
+        s_ = socket.socket(); s_.bind(("127.0.0.1", 0)); port = s_.getsockname()[1]; s_.close()
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1, device_id=dev)
     seed = synth.BASE_SEED + 3
-    grads_form = world > 1 and args.exchange in ("grads", "grads_overlap")
+    grads_form = multi and args.exchange in ("grads", "grads_overlap")
     comm_stream = torch.cuda.Stream(dev) if args.exchange == "grads_overlap" else None
     # one GPU: the FC weight-gradient kernel applies the momentum update in its epilogue (bit-identical parameters, see the
     # tests).  Several GPUs, gradient form: the gradients are stored, all-reduced, and applied by one update pass.
@@ -269,7 +274,7 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.synchronize()
 
     def step():
-        if world == 1:
+        if not multi:
             net.train_step(0, want_loss=False)
         elif grads_form:
             net.forward_backward(0)
@@ -422,7 +427,7 @@ def run_ours(args, rank, world, local_rank):
                        "global_batch": BATCH * world, "precision": "bf16 operands, fp32 accumulate, fp32 master weights",
                        "l2": "each step streams >1 GB of parameters, momentum and bf16 copies, far above the 126 MB L2",
                        "timing": f"median of {R} timed regions of {K} steps each",
-                       "parallelism": ("single GPU" if world == 1 else
+                       "parallelism": ("single GPU" if not multi else
                                        f"one replica per GPU; every step ends with the exchange between replicas over NCCL ("
                                        + (("all-reduce of the gradients, one update with their mean"
                                            + (", the FC gradients exchanged under the convolution backward pass" if comm_stream is not None else ""))
@@ -452,11 +457,12 @@ def run_ours(args, rank, world, local_rank):
                          "whole_step": {"tflops": FLOP_PER_IMAGE * BATCH / (ms / K * 1e-3) / 1e12,
                                         "frac_of_burst": FLOP_PER_IMAGE * BATCH / (ms / K * 1e-3) / 1e12 / tf_burst}},
         }
-        if world == 1:
+        if world == 1 and not args.force_exchange:
             out["config4"] = config4_leg(torch, dev, synth.BASE_SEED + 4, R)
+        if world == 1:
             out["cpu_baseline"] = cpu_baseline()
-        print(json.dumps(out))
-    if world > 1:
+        print(json.dumps(out), file=RESULT)
+    if dist.is_initialized():
         dist.barrier()
         dist.destroy_process_group()
 
@@ -473,6 +479,18 @@ def spawn_ranks(args):
     return subprocess.call(cmd)
 
 
+RESULT = sys.stdout       # where the one JSON line goes
+
+
+def keep_stdout_for_the_result():
+    """Libraries write to file descriptor 1 on their own (NCCL prints its version there when NCCL_DEBUG is set): from here
+    on descriptor 1 is stderr, and the result line goes to a private copy of the original stdout."""
+    global RESULT
+    sys.stdout.flush()
+    RESULT = os.fdopen(os.dup(1), "w")
+    os.dup2(2, 1)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -480,6 +498,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--repeats", type=int, default=5)
     ap.add_argument("--exchange", default="grads", choices=["grads", "grads_overlap", "params"])
+    ap.add_argument("--force-exchange", action="store_true",
+                    help="with one GPU: run the multi-GPU code path (the exchange after every step) on a one-rank NCCL group")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -489,10 +509,12 @@ def main():
     rank = int(os.environ.get("RANK", 0))
     world = int(os.environ.get("WORLD_SIZE", 1))
     local_rank = int(os.environ.get("LOCAL_RANK", 0))
+    keep_stdout_for_the_result()
     if args.impl == "reference":
         run_reference(args, rank, world)
     else:
         run_ours(args, rank, world, local_rank)
+    RESULT.flush()
 
 
 if __name__ == "__main__":
