@@ -154,7 +154,10 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // The issuer WARP runs its loop convergently (uniform operands stay in uniform registers) and one elected lane
-// issues: measured about 100 cycles per instruction against 130 from a lone lane inside a divergent branch.
+// issues.  In straight-line groups one warp issues at the tensor pipe's rate (measured 64 cycles per instruction at
+// N = 128, 128 at N = 256); what an instruction costs is max(N / 2, (4096 + 32 N) / 128) cycles: its A slice (4 KB) and
+// B slice are read from shared memory at 128 bytes per cycle, so N < 128 does not get faster than about 45 cycles and
+// N = 128 leaves the shared memory no bandwidth for the TMA writes that run beside it.
 __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
     asm volatile(
         "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %4, 0;\n\telect.sync _|q, 0xffffffff;\n\t"
@@ -721,9 +724,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 // is advanced by whole 128-byte rows.  Every weight tile (BN rows x 64 channels
 // of one tap) is used by the MH row halves.  Activations and weights therefore
 // travel in separate rings: an A stage lives for kw B stages.
-// One thread issues a tcgen05.mma roughly every 100 cycles, which is slower
-// than the tensor pipe for N < 192; so each 128-row half has its own issuer
-// warp (they write disjoint accumulators) and the pipe stays fed.
+// Each 128-row half has its own issuer warp (they write disjoint accumulators
+// and share the weight tiles, which halves the weight traffic into shared
+// memory per instruction).
 // Warps: 0 and 1 = TMA producers (halos, weight groups), 2..MH+1 = MMA issuers, then four epilogue warps.
 // Accumulators: MH x BN columns per buffer, two buffers when they fit in the
 // 512 TMEM columns.
