@@ -324,6 +324,20 @@ uint64_t alexnet_launch_count(const alexnet_t* h);
 int alexnet_profile(alexnet_t* h, int enable);
 int alexnet_profile_read(alexnet_t* h, double* ms4, uint64_t* launches4);
 
+/* Per-role timeline of the convolution kernel, for the timeline tool.  Only a
+ * library built with -DALEXNET_TIMELINE records it (python -m
+ * paper_1412_2302_b200.build --timeline builds that variant next to the normal
+ * one); the normal build returns ALEXNET_ERR_STATE.  Waits for the device, then
+ * copies the record of the most recent conv_kernel launch to host_out (may be
+ * NULL): 160 CTA slots x 16 values (slot = blockIdx % 160):
+ *   [0] start, [12] set-up done, [1] predecessor complete, [13] / [14] issuer enters / leaves its main loop,
+ *   [15] last store of the first epilogue warp complete, [2] exit           (all in ns of the global timer)
+ *   [3] [4] [5] cycles the first issuer waited for activations / weights / a free accumulator, [6] cycles of its main
+ *   loop, [7] instructions it issued, [8] cycles the first epilogue warp waited for accumulators,
+ *   [10] [11] cycles the producers waited for free activation / weight stages.
+ * clear != 0 zeroes the record afterwards. */
+int alexnet_timeline_read(long long* host_out, int clear);
+
 /* Bias gradient db[c] = sum over rows of dy[row][c], for callers that cannot
  * allocate device memory when they need it.  (The paper has no counterpart of
  * this call; it is the bias-gradient reduction of the step offered on its own.)

@@ -38,7 +38,7 @@ EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "
            "alexnet_loader_create", "alexnet_loader_next", "alexnet_loader_release", "alexnet_loader_destroy",
            "alexnet_forward_backward", "alexnet_apply_update", "alexnet_update_and_average", "alexnet_param_regions",
            "alexnet_scale_and_refresh", "alexnet_create_error", "alexnet_debug_expire_wait", "alexnet_set_color_augmentation", "alexnet_average_received", "alexnet_param_layout",
-           "alexnet_stream_wait_fc_gradients"]
+           "alexnet_stream_wait_fc_gradients", "alexnet_timeline_read"]
 
 
 class Config(ctypes.Structure):
@@ -89,6 +89,7 @@ def load_library():
     L.alexnet_average_received.argtypes = [vp, i32, ctypes.POINTER(vp), ctypes.POINTER(vp), i32, i32]
     L.alexnet_param_layout.argtypes = [vp, ctypes.POINTER(sz), ctypes.POINTER(sz), ctypes.POINTER(sz)]
     L.alexnet_stream_wait_fc_gradients.argtypes = [vp, vp]
+    L.alexnet_timeline_read.argtypes = [vp, i32]
     L.alexnet_eval_batch.argtypes = [vp, i32, vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32),
                                      ctypes.POINTER(ctypes.c_float)]
     L.alexnet_get_params.argtypes = [vp, i32, i32, vp, sz]

@@ -1540,6 +1540,21 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
 
 uint64_t alexnet_launch_count(const alexnet_t* h) { return h ? h->launches : 0; }
 
+int alexnet_timeline_read(long long* host_out, int clear) {
+#ifdef ALEXNET_TIMELINE
+    if (cudaDeviceSynchronize() != cudaSuccess) return ALEXNET_ERR_CUDA;
+    if (host_out && cudaMemcpyFromSymbol(host_out, tc::g_timeline, sizeof(long long) * 160 * 16) != cudaSuccess) return ALEXNET_ERR_CUDA;
+    if (clear) {
+        static const long long zeros[160 * 16] = {0};
+        if (cudaMemcpyToSymbol(tc::g_timeline, zeros, sizeof(zeros)) != cudaSuccess) return ALEXNET_ERR_CUDA;
+    }
+    return ALEXNET_OK;
+#else
+    (void)host_out; (void)clear;
+    return ALEXNET_ERR_STATE;      // this build of the library carries no timeline instrumentation
+#endif
+}
+
 int alexnet_profile(alexnet_t* h, int enable) {
     if (!h) return ALEXNET_ERR_ARG;
     h->prof = enable != 0;

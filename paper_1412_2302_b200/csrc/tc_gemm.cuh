@@ -33,6 +33,18 @@
 
 namespace tc {
 
+// Optional per-role timeline of conv_kernel (compiled in only with -DALEXNET_TIMELINE, a separate build of the library for
+// `python -m paper_1412_2302_b200.timeline`): every CTA records when it started, when its set-up was done, when its issuer
+// entered and left the main loop and how many cycles it spent in each kind of wait, when its last store had completed and
+// when it left.  16 slots per CTA; a launch overwrites the record of the launch before.
+#ifdef ALEXNET_TIMELINE
+__device__ long long g_timeline[160 * 16];
+__device__ __forceinline__ long long gtime_ns() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define TL(...) __VA_ARGS__
+#else
+#define TL(...)
+#endif
+
 enum { MODE_KK = 0, MODE_KMN = 1, MODE_MNMN = 2 };
 enum { EPI_BF16 = 0, EPI_F32 = 1 };
 constexpr int kThreads = 192;
@@ -813,6 +825,7 @@ __device__ __forceinline__ void issue_row(uint32_t d, uint64_t ad, uint64_t bd, 
 // (rank 0) issues: one instruction covers half h of both CTAs, and its commits arrive on the barriers of both.
 template <int CG>
 __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_constant__ ConvParams p) {
+    TL(long long* tl = g_timeline + (blockIdx.x % 160) * 16; if (threadIdx.x == 0) { tl[0] = gtime_ns(); tl[8] = 0; tl[10] = 0; tl[11] = 0; tl[7] = 0; })
     kn::pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -860,7 +873,9 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     if (CG == 2) cluster_sync_all();          // the peer's barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    TL(if (threadIdx.x == 0) tl[12] = gtime_ns();)
     kn::pdl_wait();        // barriers, TMEM and descriptors are set up; global memory is touched from here on
+    TL(if (threadIdx.x == 0) tl[1] = gtime_ns();)
     const int per = p.asteps_per_split, kw = p.kw;
 
     if (warp == 0) {
@@ -882,7 +897,10 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 const int ky0 = a_begin / p.chunks, ch0 = a_begin - ky0 * p.chunks;
                 const int xa = p.a_x0 + tc.g * p.a_gx;
                 for (int i = 0; i < nsteps && ok; ++i) {
-                    if (!(ok = mbar_wait(emptyA + 8u * sa, pha ^ 1u, abort_flag))) break;
+                    TL(const long long c0 = clock64();)
+                    ok = mbar_wait(emptyA + 8u * sa, pha ^ 1u, abort_flag);
+                    TL(tl[10] += clock64() - c0;)
+                    if (!ok) break;
                     {
                         const uint32_t dst = ring_a + sa * a_bytes, fb = fullA + 8u * sa;
                         const int y = m0 + p.halo_shift[ky];
@@ -925,7 +943,10 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                     int brow = ky * kw * p.b_tap_rows + yb, bcol = ch * cpg * 64;
                     const int brow_step = cpg > 1 ? 0 : p.b_tap_rows, bcol_step = cpg > 1 ? 64 : 0;
                     for (int kx0 = 0; kx0 < gw; kx0 += p.tpg) {
-                        if (!(ok = mbar_wait(emptyB + 8u * sb, phb ^ 1u, abort_flag))) break;
+                        TL(const long long c0 = clock64();)
+                        ok = mbar_wait(emptyB + 8u * sb, phb ^ 1u, abort_flag);
+                        TL(tl[11] += clock64() - c0;)
+                        if (!ok) break;
                         const uint32_t fb = fullB + 8u * sb, dst = ring_b + sb * g_bytes;
                         const int taps = min(p.tpg, gw - kx0);
                         if (rank == 0) mbar_expect_tx(fb, (uint32_t)taps * b_bytes * CG);
@@ -955,22 +976,31 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
             const int tiles_per_split = p.m_tiles * p.n_tiles * p.groups;
             const bool b_res = p.b_res != 0;
             if (b_res && vb < p.tiles_total) ok = mbar_wait_warp(fullB, 0u, abort_flag);      // the resident filter has arrived
+            TL(long long wA = 0, wB = 0, wC = 0, nm = 0; const long long tl0 = clock64(), gl0 = gtime_ns();)
             for (int tile = vb; tile < p.tiles_total && ok; tile += vgrid) {
                 const int a_begin = z * per;
                 const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
                 int ares = a_begin + (int)((unsigned)vb % (unsigned)nsteps);      // resident filter: the producer's rotation of the filter rows
-                if (!(ok = mbar_wait_warp(acce0 + 8u * ab, aph ^ 1u, abort_flag))) break;
+                TL(const long long cc0 = clock64();)
+                ok = mbar_wait_warp(acce0 + 8u * ab, aph ^ 1u, abort_flag);
+                TL(wC += clock64() - cc0;)
+                if (!ok) break;
                 if (CG == 2) fence_acq_rel_cluster();      // the peer's epilogue arrived from the other CTA
                 tc_fence_after();
                 const uint32_t d = tmem + (uint32_t)(ab * acc_cols + h * BN);
                 uint32_t accum = 0;
                 for (int i = 0; i < nsteps && ok; ++i) {
-                    if (!(ok = mbar_wait_warp(fullA + 8u * sa, pha, abort_flag))) break;
+                    TL(const long long ca0 = clock64();)
+                    ok = mbar_wait_warp(fullA + 8u * sa, pha, abort_flag);
+                    TL(wA += clock64() - ca0;)
+                    if (!ok) break;
                     const uint64_t ad = dbase + (uint64_t)((ring_a + sa * a_bytes + (uint32_t)h * 16384u) >> 4);
                     // the MMAs of a weight group in straight-line code: the fixed cost of a loop trip with a barrier wait
                     // (a few hundred cycles) is paid once per taps*kk instructions
                     for (int kx0 = 0; kx0 < gw; kx0 += p.tpg) {
+                        TL(const long long cb0 = clock64();)
                         if (!b_res && !(ok = mbar_wait_warp(fullB + 8u * sb, phb, abort_flag))) break;
+                        TL(wB += clock64() - cb0; nm += (long long)min(p.tpg, gw - kx0) * kk;)
                         const uint64_t bd = dbase + (uint64_t)((b_res ? ring_b + (uint32_t)(ares * kw) * b_bytes : ring_b + sb * g_bytes) >> 4);
                         const int taps = min(p.tpg, gw - kx0);
                         const int* toff = p.tap_off + kx0;
@@ -1000,6 +1030,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 in_split += vgrid;
                 while (in_split >= tiles_per_split) { in_split -= tiles_per_split; ++z; }
             }
+            TL(if (h == 0 && lane == 0) { tl[3] = wA; tl[4] = wB; tl[5] = wC; tl[6] = clock64() - tl0; tl[7] = nm; tl[13] = gl0; tl[14] = gtime_ns(); })
         }
     } else {
         // ------------------------------------------------------------ epilogue
@@ -1014,7 +1045,10 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
             const int m0 = tc.m_tile * tile_rows + row0, n0 = tc.n_tile * BN, g = tc.g;
             const int a_begin = tc.z * per;
             const int nsteps = min(p.asteps_total, a_begin + per) - a_begin;
-            if (!(ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag))) break;
+            TL(const long long ce0 = clock64();)
+            ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag);
+            TL(if (ew == 0 && lane == 0) tl[8] += clock64() - ce0;)
+            if (!ok) break;
             tc_fence_after();
             // with two sets of epilogue warps, the (row half, slab) units of the tile alternate between the sets
             int unit = 0;
@@ -1053,6 +1087,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
             if (++ab == acc_stages) { ab = 0; aph ^= 1u; }
         }
         if (p.tma_store && lane == 0) bulk_wait_all();
+        TL(if (ew == 0 && lane == 0) tl[15] = gtime_ns();)
     }
     tc_fence_before();
     __syncthreads();
@@ -1064,6 +1099,7 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     }
     __syncwarp();
     if (CG == 2) cluster_sync_all();          // no CTA leaves while its peer may still arrive on its barriers
+    TL(if (threadIdx.x == 0) tl[2] = gtime_ns();)
     if (warp == 2) {
         tc_fence_after();
         if (CG == 2) tmem_dealloc_pair(tmem, ncols);
