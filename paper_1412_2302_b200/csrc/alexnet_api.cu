@@ -1339,6 +1339,18 @@ int alexnet_loss_async(alexnet_t* h, int replica, float* loss_out) {
     if (!h) return ALEXNET_ERR_ARG;
     if (replica < 0 || replica >= h->cfg.replicas || !loss_out) return fail(h, ALEXNET_ERR_ARG, "loss_async: bad argument");
     if (int rc = check_status(h)) return rc;
+    // A 4-byte cudaMemcpyAsync shares the copy engines with the 25 MB batch uploads of the loader stream and was seen to hold
+    // the compute stream up by 35 us per step behind one.  Where the destination is visible to the device (device memory, or
+    // pinned / registered host memory: the cases the header allows) a one-thread kernel stores the value instead.
+    cudaPointerAttributes at{};
+    if (cudaPointerGetAttributes(&at, loss_out) == cudaSuccess && at.devicePointer != nullptr &&
+        (at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged)) {
+        launch_k(kn::store_value_kernel, 1, 1, 0, h->cs, (const float*)h->rep[replica].loss, (float*)at.devicePointer);
+        h->launches++;
+        CK(cudaGetLastError());
+        return ALEXNET_OK;
+    }
+    cudaGetLastError();      // (an unregistered host pointer makes the query fail on some drivers: not an error here)
     CK(cudaMemcpyAsync(loss_out, h->rep[replica].loss, sizeof(float), cudaMemcpyDefault, h->cs));
     return ALEXNET_OK;
 }

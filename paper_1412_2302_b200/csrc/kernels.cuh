@@ -706,6 +706,13 @@ __global__ void __launch_bounds__(256) fc8_softmax_xent_kernel(const float* __re
         *done_counter = 0;
     }
 }
+// one float to wherever dst points (device memory, or pinned host memory mapped into the device's address space): the
+// loss read-back without a copy engine, whose queue a batch upload of 25 MB may occupy
+__global__ void store_value_kernel(const float* __restrict__ src, float* __restrict__ dst) {
+    pdl_sync();
+    *dst = *src;
+    __threadfence_system();
+}
 __global__ void mean_kernel(const float* __restrict__ v, int n, float* __restrict__ out) {
     pdl_sync();
     __shared__ float red[32];
