@@ -533,7 +533,7 @@ int plan_conv_wg(alexnet* h, Plan& P, int l, const ConvL& c, const bf16* dy, con
     P.valid = true;
     return ALEXNET_OK;
 }
-int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* wsh) {
+int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* wsh, const float* bias, bool with_epilogue) {
     memset(&P, 0, sizeof(P));
     tc::ConvParams& p = P.c;
     const int B = h->B;
@@ -554,6 +554,16 @@ int plan_fc_fwd(alexnet* h, Plan& P, const FcL& f, const bf16* x, const bf16* ws
     if ((rc = make_tm_out(h, &p.tmOut, h->ws, true, (uint64_t)f.N, (uint64_t)B, (uint64_t)p.splits, (uint64_t)f.N * 4,
                           (uint64_t)B * f.N * 4))) return rc;
     finish_conv_plan(h, P);
+    // fc6 / fc7 with one row tile (batch <= 128) and 2, 4 or 8 splits: the splits of a tile form a thread-block cluster and
+    // reduce their partial tiles through distributed shared memory, with bias, ReLU and dropout applied there (no partials in
+    // HBM, no second launch).  fc8 keeps its partials: its reduction is part of the softmax kernel.
+    const int S = p.splits;
+    if (with_epilogue && p.m_tiles == 1 && (S == 2 || S == 4 || S == 8) && p.tiles_total <= h->sm_count && f.N % 4 == 0 &&
+        (size_t)128 * tc::kZcPitch * 4 <= (size_t)p.a_stages * p.MH * p.cpg * p.a_box_rows * 128 + (size_t)p.b_stages * p.tpg * p.BN * 128) {
+        p.zcluster = S;
+        p.bias = bias;
+        P.grid = p.tiles_total;
+    }
     return ALEXNET_OK;
 }
 int plan_fc_bwd(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* wsh) {
@@ -624,7 +634,7 @@ int build_plans(alexnet* h, int r) {
     const bf16* fdy[3] = {R.df6, R.df7, R.dz};
     for (int l = 0; l < 3; ++l) {
         const FcL& f = L.fc[l];
-        if ((rc = plan_fc_fwd(h, R.fc_fwd[l], f, fx[l], R.shadow + f.w_off))) return rc;
+        if ((rc = plan_fc_fwd(h, R.fc_fwd[l], f, fx[l], R.shadow + f.w_off, R.w + f.b_off, l < 2))) return rc;
         if ((rc = plan_fc_bwd(h, R.fc_bwd[l], f, fdy[l], R.shadow + f.w_off))) return rc;
         const bool fuse = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0;
         if ((rc = plan_fc_wg(h, R.fc_wg[l], f, fdy[l], fx[l], R.g + f.w_off, R.w + f.w_off, R.v + f.w_off, R.shadow + f.w_off, fuse))) return rc;
@@ -656,6 +666,17 @@ void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
         at[1].val.programmaticStreamSerializationAllowed = 1;
         lc.attrs = at; lc.numAttrs = 2;
         cudaLaunchKernelEx(&lc, tc::conv_kernel<2>, P.c);
+    }
+    else if (P.conv && P.c.zcluster) {
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3(P.grid); lc.blockDim = dim3(tc::conv_threads(P.c)); lc.dynamicSmemBytes = P.smem; lc.stream = st;
+        cudaLaunchAttribute at[2] = {};
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = P.c.zcluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[1].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at; lc.numAttrs = 2;
+        cudaLaunchKernelEx(&lc, tc::conv_kernel<1>, P.c);
     }
     else if (P.conv) launch_k(tc::conv_kernel<1>, P.grid, tc::conv_threads(P.c), P.smem, st, P.c);
     else launch_k(tc::gemm_kernel, P.grid, tc::kThreads, P.smem, st, P.p);
@@ -708,10 +729,7 @@ void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
 void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool eval = false, bool gemm_only = false) {
     Replica& R = h->rep[r];
     const FcL& f = h->L.fc[l];
-    const Plan& P = R.fc_fwd[l];
-    launch_gemm(h, P, st);
-    if (gemm_only) return;     // the split reduction is part of the kernel that follows (fc8 inside the step)
-    const long long total = (long long)h->B * f.N;
+    Plan& P = R.fc_fwd[l];
     bf16* outs[3] = {R.f6, R.f7, nullptr};
     uint8_t* keeps[3] = {R.m6, R.m7, nullptr};
     int drop = l < 2 && h->cfg.dropout_p > 0.f;
@@ -721,6 +739,15 @@ void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool ev
         scale = (h->cfg.flags & ALEXNET_FLAG_INVERTED_DROPOUT) ? 1.f : 1.f - h->cfg.dropout_p;
     }
     const uint64_t key = kn::stream_key(h->cfg.seed, 2 + l, r, step);
+    if (P.c.zcluster) {      // reduction, bias, ReLU and dropout inside the GEMM kernel (a cluster per tile)
+        P.c.fc_relu = 1; P.c.fc_dropout = drop; P.c.fc_key = key; P.c.fc_thr24 = h->thr24; P.c.fc_scale = scale;
+        P.c.fc_out = outs[l]; P.c.fc_keep = keeps[l];
+        launch_gemm(h, P, st);
+        return;
+    }
+    launch_gemm(h, P, st);
+    if (gemm_only) return;     // the split reduction is part of the kernel that follows (fc8 inside the step)
+    const long long total = (long long)h->B * f.N;
     launch_k(kn::fc_reduce_fwd_kernel, nblk(total, 256), 256, 0, st, h->ws, P.c.splits, P.c.split_stride, R.w + f.b_off, h->B, f.N,
                                                                 l < 2, drop, key, h->thr24, scale, outs[l],
                                                                 l == 2 ? R.z : nullptr, keeps[l]);

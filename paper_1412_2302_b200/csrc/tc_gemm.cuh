@@ -775,7 +775,17 @@ struct ConvParams {
     const __nv_bfloat16* mask;
     void* out;
     int* status;
+    // FC forward with the split-K reduction inside the kernel: the `zcluster` CTAs of a thread-block cluster are the k splits
+    // of one 128-row x BN tile (one tile per CTA, m_tiles == 1).  Each leaves its fp32 partial tile in its own shared
+    // memory; after a cluster barrier CTA z adds rows [z * 128 / zcluster, ...) of all partials in split order through
+    // distributed shared memory and applies bias, ReLU and dropout (the arithmetic of fc_reduce_fwd_kernel, so the result
+    // is bit-identical to the two-launch form), writing the layer's bf16 output and its keep mask.  0: off.
+    int zcluster;
+    int fc_relu, fc_dropout;       // fc_dropout: 0 none, 1 mask from the hash, 2 evaluation (expectation of the mask)
+    uint64_t fc_key; uint32_t fc_thr24; float fc_scale;
+    __nv_bfloat16* fc_out; uint8_t* fc_keep;
 };
+constexpr int kZcPitch = 132;      // floats per row of the partial tile in shared memory (128 + 4: conflict-free float4 rows)
 
 constexpr int kConvMaxThreads = 32 * 12;
 inline int conv_threads(const ConvParams& p) { return 32 * (2 + p.MH + 4 * p.epi_sets); }
@@ -832,8 +842,12 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     const uint32_t base = (raw + 1023u) & ~1023u;
     const int MH = p.MH, BN = p.BN;
     const int rank = CG == 2 ? (int)cluster_ctarank() : 0;
-    const int vb = CG == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // position and stride in the tile list
-    const int vgrid = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    int vb = CG == 2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;       // position and stride in the tile list
+    int vgrid = CG == 2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int zc = CG == 1 ? p.zcluster : 0;
+    const int zrank = zc ? (int)cluster_ctarank() : 0;
+    const int zdiv = zc ? zc : 1;
+    if (zc) { vb = zrank * p.n_tiles + (int)blockIdx.x / zdiv; vgrid = p.tiles_total; }    // split zrank of n tile blockIdx / zc; one tile
     const int tile_rows = 128 * MH * CG, row0 = rank * 128 * MH;
     const int cpg = p.cpg, gw = cpg > 1 ? cpg : p.kw;            // weight tiles per A stage
     const uint32_t a_box_bytes = (uint32_t)p.a_box_rows * 128u, a_bytes = a_box_bytes * MH * cpg, b_bytes = (uint32_t)(BN / CG) * 128u;
@@ -1063,7 +1077,18 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
                 }
                 const long long row_off = (long long)tc.z * p.split_stride + (long long)row * p.ldo + g * p.out_gx;
                 const uint32_t t0 = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * acc_cols + h * BN);
-                if (p.tma_store) {
+                if (zc) {
+                    // the partial tile stays on chip: row r of the tile to the (idle) operand ring, 32 columns per unit
+                    for (int c = 0; c < BN; c += 32, ++unit) {
+                        if (E == 2 && (unit & 1) != eset) continue;
+                        uint32_t v[32];
+                        tmem_ld32(t0 + (uint32_t)c, v);
+                        tmem_ld_wait();
+                        const uint32_t rowp = ring_a + (uint32_t)(r * kZcPitch + c) * 4u;
+                        #pragma unroll
+                        for (int q = 0; q < 8; ++q) st_shared_v4(rowp + 16u * q, v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                    }
+                } else if (p.tma_store) {
                     const int slab = p.epi == EPI_F32 ? 32 : 64;
                     for (int c = 0; c < BN; c += slab, ++unit) {
                         if (E == 2 && (unit & 1) != eset) continue;
@@ -1086,8 +1111,50 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
             else mbar_arrive(acce0 + 8u * ab);
             if (++ab == acc_stages) { ab = 0; aph ^= 1u; }
         }
-        if (p.tma_store && lane == 0) bulk_wait_all();
+        if (p.tma_store && !zc && lane == 0) bulk_wait_all();
         TL(if (ew == 0 && lane == 0) tl[15] = gtime_ns();)
+    }
+    if (zc) {
+        // every CTA of the cluster has its partial tile in shared memory (all threads arrive: the barrier also orders the
+        // epilogue warps' stores before the peers' reads); then the epilogue warps reduce this CTA's rows across the cluster
+        __syncwarp();
+        cluster_sync_all();
+        if (warp > MH + 1) {
+            const int T = 128 * p.epi_sets, t = (warp - (MH + 2)) * 32 + lane;
+            const int rows_per = 128 / zdiv, n0 = ((int)blockIdx.x / zdiv) * BN;
+            for (int idx = t; idx < rows_per * 32; idx += T) {
+                const int row = zrank * rows_per + (idx >> 5), c4 = idx & 31;
+                const uint32_t local = ring_a + (uint32_t)(row * kZcPitch + 4 * c4) * 4u;
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int q = 0; q < zc; ++q) {
+                    float4 v;
+                    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(mapa_u32(local, (uint32_t)q)) : "memory");
+                    acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
+                }
+                if (row >= p.M_total) continue;
+                const int n = n0 + 4 * c4;
+                if (n >= p.n_valid) continue;                      // n_valid is a multiple of 4 in the layers that run this way
+                const long long tt = (long long)row * p.n_valid + n;
+                uint32_t keepw = 0x01010101u;
+                #pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    float v = acc[k] + p.bias[n + k];
+                    if (p.fc_relu) v = fmaxf(v, 0.f);
+                    if (p.fc_dropout == 2) v *= p.fc_scale;
+                    else if (p.fc_dropout) {
+                        const bool keep = (uint32_t)(kn::draw(p.fc_key, (uint64_t)(tt + k)) >> 40) >= p.fc_thr24;
+                        if (!keep) keepw &= ~(0xFFu << (8 * k));
+                        v = keep ? v * p.fc_scale : 0.f;
+                    }
+                    acc[k] = v;
+                }
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[0], acc[1]), hi = __floats2bfloat162_rn(acc[2], acc[3]);
+                *(uint2*)(p.fc_out + tt) = make_uint2(*(const uint32_t*)&lo, *(const uint32_t*)&hi);
+                if (p.fc_keep) *(uint32_t*)(p.fc_keep + tt) = keepw;
+            }
+        }
+        __syncwarp();
+        cluster_sync_all();          // no CTA leaves (and frees its shared memory) while a peer may still read its partial tile
     }
     tc_fence_before();
     __syncthreads();
