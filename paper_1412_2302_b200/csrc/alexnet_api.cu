@@ -918,14 +918,14 @@ void op_average(alexnet* h, cudaStream_t st) {
 }
 void op_preprocess(alexnet* h, int r, int slot, uint64_t step, cudaStream_t st, bool eval = false) {
     Replica& R = h->rep[r];
-    const long long total = (long long)h->B * 57 * 57 * 4;
     kn::ColorAug aug = h->color;
     aug.key = kn::stream_key(h->cfg.seed, 10, r, step);
+    const dim3 grid(57, h->B);
     if (aug.sigma != 0.f && !eval)
-        launch_k(kn::preprocess_kernel<true>, nblk(total, 256), 256, 0, st, R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
+        launch_k(kn::preprocess_kernel<true>, grid, 256, 0, st, R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
                  kn::stream_key(h->cfg.seed, 1, r, step), 0, aug);
     else
-        launch_k(kn::preprocess_kernel<false>, nblk(total, 256), 256, 0, st, R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
+        launch_k(kn::preprocess_kernel<false>, grid, 256, 0, st, R.stage[slot], h->mean, R.x0[slot], R.cf[slot], h->B,
                  kn::stream_key(h->cfg.seed, 1, r, step), eval ? 1 : 0, aug);
     h->launches++;
 }

@@ -61,26 +61,35 @@ __device__ __forceinline__ float normal_draw(uint64_t key, uint64_t idx) {
     const float u2 = (float)((r >> 16) & 0xFFFFFF) * (1.f / 16777216.f);
     return sqrtf(-2.f * logf(u1)) * cospif(2.f * u2);
 }
+// One block = one image and four rows of the 228-padded crop (one row `by` of the space-to-depth grid): the four source rows
+// of the uint8 image (768 bytes each) and of the mean image (768 floats each) come to shared memory in coalesced loads, then
+// thread (bx, dy) forms its 12 values (4 pixels x 3 colours) from there and stores 24 contiguous bytes; a warp writes 768
+// contiguous bytes.  grid: (57, B), 256 threads.
 template <bool AUG>
-__global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* __restrict__ mean,
-                                  __nv_bfloat16* __restrict__ out, int32_t* __restrict__ cf_out,
-                                  int B, uint64_t key, int eval_mode, const ColorAug aug) {
+__global__ void __launch_bounds__(256) preprocess_kernel(const uint8_t* __restrict__ img, const float* __restrict__ mean,
+                                                         __nv_bfloat16* __restrict__ out, int32_t* __restrict__ cf_out,
+                                                         int B, uint64_t key, int eval_mode, const ColorAug aug) {
     pdl_sync();
-    // one thread per (n, by, bx, dy): 12 output values (4 dx * 3 colours) = 24 bytes
-    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long total = (long long)B * 57 * 57 * 4;
-    if (t >= total) return;
-    const int dy = (int)(t & 3);
-    long long cell = t >> 2;
-    const int bx = (int)(cell % 57); cell /= 57;
-    const int by = (int)(cell % 57);
-    const int n = (int)(cell / 57);
+    __shared__ uint4 s_img[4][49];        // rows padded by 16 bytes: the four rows start in different banks
+    __shared__ float s_mean[4][769];      // row pitch = 1 mod 32 words: the warp's 8 bx x 4 dy reads (12 words apart per bx) hit 32 banks
+    const int by = blockIdx.x, n = blockIdx.y, tid = threadIdx.x;
     const uint64_t r = draw(key, (uint64_t)n);
     // evaluation: the centre 227 x 227 window, never flipped
     const int ox = eval_mode ? 14 : (int)((r & 0xFFFF) % 30), oy = eval_mode ? 14 : (int)(((r >> 16) & 0xFFFF) % 30);
     const int flip = eval_mode ? 0 : (int)((r >> 32) & 1);
-    if (cf_out && by == 0 && bx == 0 && dy == 0) { cf_out[3 * n] = ox; cf_out[3 * n + 1] = oy; cf_out[3 * n + 2] = flip; }
-    const int Y = by * 4 + dy;
+    if (cf_out && by == 0 && tid == 0) { cf_out[3 * n] = ox; cf_out[3 * n + 1] = oy; cf_out[3 * n + 2] = flip; }
+    for (int i = tid; i < 4 * 48; i += 256) {
+        const int dy = i / 48, j = i - dy * 48, Y = by * 4 + dy;
+        if (Y < 227) s_img[dy][j] = __ldg((const uint4*)(img + (size_t)n * 196608 + (size_t)(oy + Y) * 768) + j);
+    }
+    #pragma unroll
+    for (int i = tid; i < 4 * 768; i += 256) {     // one float per lane: conflict-free stores at the odd row pitch
+        const int dy = i / 768, j = i - dy * 768, Y = by * 4 + dy;
+        if (Y < 227) s_mean[dy][j] = __ldg(mean + (size_t)(oy + Y) * 768 + j);
+    }
+    __syncthreads();
+    if (tid >= 228) return;
+    const int dy = tid & 3, bx = tid >> 2;
     float shift[3] = {0.f, 0.f, 0.f};
     if (AUG && !eval_mode) {
         const float a0 = aug.sigma * normal_draw(aug.key, 3ull * n), a1 = aug.sigma * normal_draw(aug.key, 3ull * n + 1),
@@ -88,23 +97,27 @@ __global__ void preprocess_kernel(const uint8_t* __restrict__ img, const float* 
         #pragma unroll
         for (int c = 0; c < 3; ++c) shift[c] = aug.pl[3 * c] * a0 + aug.pl[3 * c + 1] * a1 + aug.pl[3 * c + 2] * a2;
     }
+    const int Y = by * 4 + dy;
+    const uint8_t* ib = (const uint8_t*)s_img[dy];
+    const float* mb = s_mean[dy];
     float v[12];
     #pragma unroll
     for (int dx = 0; dx < 4; ++dx) {
         const int X = bx * 4 + dx;
         if (Y < 227 && X < 227) {
-            const int sy = oy + Y, sx = ox + (flip ? 226 - X : X);
-            const size_t s = ((size_t)sy * 256 + sx) * 3;
-            const uint8_t* ip = img + (size_t)n * 196608 + s;
+            const int s3 = (ox + (flip ? 226 - X : X)) * 3;
             #pragma unroll
-            for (int c = 0; c < 3; ++c) v[dx * 3 + c] = ((float)ip[c] - mean[s + c]) + shift[c];
+            for (int c = 0; c < 3; ++c) v[dx * 3 + c] = ((float)ib[s3 + c] - mb[s3 + c]) + shift[c];
         } else {
             v[dx * 3] = v[dx * 3 + 1] = v[dx * 3 + 2] = 0.f;
         }
     }
-    __nv_bfloat162* o = (__nv_bfloat162*)(out + ((size_t)(n * 57 + by) * 57 + bx) * 48 + dy * 12);
+    uint2* o = (uint2*)(out + ((size_t)(n * 57 + by) * 57 + bx) * 48 + dy * 12);
     #pragma unroll
-    for (int i = 0; i < 6; ++i) o[i] = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+    for (int i = 0; i < 3; ++i) {
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v[4 * i], v[4 * i + 1]), hi = __floats2bfloat162_rn(v[4 * i + 2], v[4 * i + 3]);
+        o[i] = make_uint2(*(const uint32_t*)&lo, *(const uint32_t*)&hi);
+    }
 }
 
 // ----------------------------------------------------------------------- LRN
