@@ -61,7 +61,7 @@ enum {                                /* alexnet_config_t.flags */
     ALEXNET_FLAG_NO_CTA_PAIRS = 16,    /* convolution forward / backward-data never run as clusters of two CTAs */
     ALEXNET_FLAG_ALL_CTA_PAIRS = 32,   /* ... always do (default: per layer, where the cost model expects a gain);
                                         * results do not depend on either flag beyond fp32 summation order */
-    ALEXNET_FLAG_SHARED_REPLICA_WEIGHTS = 64 /* replicas == 2: both replicas use ONE copy of parameters, momentum and their bf16
+    ALEXNET_FLAG_SHARED_REPLICA_WEIGHTS = 64,/* replicas == 2: both replicas use ONE copy of parameters, momentum and their bf16
                                         * forms.  Valid for the paper's scheme because the replicas are equal at the start of
                                         * every iteration (same initialisation; every exchange makes them equal again).  An
                                         * iteration is then alexnet_forward_backward on both replicas followed by
@@ -71,6 +71,12 @@ enum {                                /* alexnet_config_t.flags */
                                         * alexnet_train_step and alexnet_apply_update return STATE (they would let one replica
                                         * run ahead of the other); alexnet_replica_average is a no-op; get/set_params address
                                         * the one copy through either replica index */
+    ALEXNET_FLAG_FC_CHAIN = 128        /* the three FC forward passes run as ONE cooperative launch (fc_chain_kernel) whose weight
+                                        * stream never stops at a layer boundary, where that is possible: batch <= 128 and a
+                                        * device that can hold the whole grid at once; elsewhere the flag changes nothing.
+                                        * Same units, arithmetic and summation order as the three launches: bit-identical
+                                        * activations, masks and logits.  Off by default: measured, the step is no faster
+                                        * (a layer boundary inside the launch costs what a launch boundary costs) */
 };
 
 typedef struct {
@@ -305,6 +311,8 @@ enum {
     ALEXNET_OP_UPDATE_AVERAGE,   /* the one-pass update + average of alexnet_update_and_average on whatever the gradient
                                   * arrays of the two replicas hold */
     ALEXNET_OP_SCALE_REFRESH,    /* alexnet_scale_and_refresh with scale 1 */
+    ALEXNET_OP_FC_CHAIN_FWD,     /* P5 -> F6, M6, F7, M7 and fc8's split partials in one launch (what the step runs under
+                                  * ALEXNET_FLAG_FC_CHAIN); ALEXNET_ERR_STATE where it is not available */
     ALEXNET_OP_COUNT
 };
 int alexnet_run_op(alexnet_t* h, int replica, int op, int iters);
@@ -319,8 +327,9 @@ uint64_t alexnet_launch_count(const alexnet_t* h);
  * since the last read, and clears the record.  Index 0 = conv_kernel on
  * convolutions (forward and backward-data), 1 = wgrad_kernel (convolution
  * weight gradients), 2 = gemm_kernel (FC backward-data and weight gradients),
- * 3 = conv_kernel on the FC forward passes (its 1 x 1 case, HBM-bound at batch
- * 128).  Both arrays have four entries. */
+ * 3 = the FC forward passes (fc_chain_kernel: one launch for the three layers;
+ * or conv_kernel's 1 x 1 case, one launch per layer; HBM-bound at batch 128).
+ * Both arrays have four entries. */
 int alexnet_profile(alexnet_t* h, int enable);
 int alexnet_profile_read(alexnet_t* h, double* ms4, uint64_t* launches4);
 

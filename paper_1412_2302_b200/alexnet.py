@@ -15,7 +15,7 @@ from . import build as _build
 
 OK, ERR_ARG, ERR_CUDA, ERR_STATE, ERR_DEVICE_TIMEOUT, ERR_NOMEM = 0, -1, -2, -3, -4, -5
 FLAG_LRN_ALPHA_DIV_N, FLAG_WD_ON_BIASES, FLAG_INVERTED_DROPOUT, FLAG_FUSED_FC_UPDATE = 1, 2, 4, 8
-FLAG_NO_CTA_PAIRS, FLAG_ALL_CTA_PAIRS, FLAG_SHARED_REPLICA_WEIGHTS = 16, 32, 64
+FLAG_NO_CTA_PAIRS, FLAG_ALL_CTA_PAIRS, FLAG_SHARED_REPLICA_WEIGHTS, FLAG_FC_CHAIN = 16, 32, 64, 128
 
 TENSORS = ["CROPFLIP", "X0", "A1", "N1", "P1", "ARG1", "A2", "N2", "P2", "ARG2", "A3", "A4", "A5", "P5", "ARG5",
            "F6", "F7", "Z", "M6", "M7", "DZ", "DF7", "DF6", "DP5", "DA5", "DA4", "DA3", "DP2", "DN2", "DA2",
@@ -28,7 +28,7 @@ OPS = ["CONV1_FWD", "CONV2_FWD", "CONV3_FWD", "CONV4_FWD", "CONV5_FWD",
        "FC6_BWD_WEIGHT", "FC7_BWD_WEIGHT", "FC8_BWD_WEIGHT",
        "LRN1_FWD", "LRN2_FWD", "LRN1_BWD", "LRN2_BWD", "POOL1_FWD", "POOL2_FWD", "POOL5_FWD",
        "POOL1_BWD", "POOL2_BWD", "POOL5_BWD", "SOFTMAX", "UPDATE", "AVERAGE", "PREPROCESS", "CONV1_BWD_DATA",
-       "LRN1_POOL1_FWD", "LRN2_POOL2_FWD", "POOL1_LRN1_BWD", "POOL2_LRN2_BWD", "UPDATE_AVERAGE", "SCALE_REFRESH"]
+       "LRN1_POOL1_FWD", "LRN2_POOL2_FWD", "POOL1_LRN1_BWD", "POOL2_LRN2_BWD", "UPDATE_AVERAGE", "SCALE_REFRESH", "FC_CHAIN_FWD"]
 OP = {n: i for i, n in enumerate(OPS)}
 
 EXPORTS = ["alexnet_param_count", "alexnet_workspace_bytes", "alexnet_create", "alexnet_destroy",

@@ -145,6 +145,9 @@ struct Replica {
     Plan conv_fwd[5][2], conv_bwd[5], conv_wg[5][2], fc_fwd[3], fc_bwd[3], fc_wg[3];
     Plan fc_wg_plain[3];    // the FC weight gradient stored, never fused with the update (alexnet_forward_backward)
     bool grad_pending;      // forward_backward has left a gradient that no update has consumed yet
+    // fc6 -> fc7 -> fc8 forward as one cooperative launch (tc::fc_chain_kernel); chain_mode: 0 off, 1 with programmatic
+    // dependent launch, 2 without (the launch attributes the driver accepted); chain_gate: value of the grid gate
+    tc::FcChainParams chain; int chain_mode; unsigned chain_gate;
 };
 
 }  // namespace
@@ -612,6 +615,44 @@ int plan_fc_wg(alexnet* h, Plan& P, const FcL& f, const bf16* dy, const bf16* x,
     return ALEXNET_OK;
 }
 
+// The three FC forward passes as one launch (ALEXNET_FLAG_FC_CHAIN), when every layer is one unit per CTA of the same grid: one row tile (batch
+// <= 128), 128-column tiles, fc6 / fc7 as clusters of their four splits, fc8's tiles x splits filling the same grid, and
+// the device able to hold all clusters at once (the CTAs wait for one another at the layer boundaries).
+void plan_fc_chain(alexnet* h, int r) {
+    Replica& R = h->rep[r];
+    R.chain_mode = 0; R.chain_gate = 0;
+    if (!(h->cfg.flags & ALEXNET_FLAG_FC_CHAIN)) return;
+    tc::FcChainParams& q = R.chain;
+    memset(&q, 0, sizeof(q));
+    const int grid = R.fc_fwd[0].c.tiles_total;
+    bf16* outs[3] = {R.f6, R.f7, nullptr};
+    uint8_t* keeps[3] = {R.m6, R.m7, nullptr};
+    for (int l = 0; l < 3; ++l) {
+        const tc::ConvParams& c = R.fc_fwd[l].c;
+        const FcL& f = h->L.fc[l];
+        if (!R.fc_fwd[l].valid || c.m_tiles != 1 || c.BN != 128 || c.cpg != 2 || c.kk != 4 || c.kh != 1 || c.tiles_total != grid ||
+            c.n_valid % 4 || (l < 2 ? c.zcluster != tc::kChainCluster : c.zcluster != 0)) return;
+        tc::FcChainLayer& y = q.L[l];
+        y.tmA = c.tmA; y.tmB = c.tmB;
+        y.n_tiles = c.n_tiles; y.splits = c.splits; y.per = c.asteps_per_split; y.asteps_total = c.asteps_total; y.n_valid = c.n_valid;
+        y.cluster_reduce = l < 2;
+        y.relu = l < 2; y.bias = R.w + f.b_off; y.out = outs[l]; y.keep = keeps[l];
+        y.partial = h->ws; y.split_stride = c.split_stride;
+    }
+    if (grid % tc::kChainCluster || grid > h->sm_count) return;
+    q.nlayers = 3; q.M_total = h->B; q.status = h->status; q.gate = (unsigned*)(h->status + 12 + r);
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(grid); lc.blockDim = dim3(tc::kChainThreads); lc.dynamicSmemBytes = tc::fc_chain_smem_bytes();
+    cudaLaunchAttribute at[1] = {};
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = tc::kChainCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    lc.attrs = at; lc.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, tc::fc_chain_kernel, &lc) != cudaSuccess) { cudaGetLastError(); return; }
+    if (clusters * tc::kChainCluster < grid) return;
+    R.chain_mode = 1;
+}
+
 int build_plans(alexnet* h, int r) {
     Replica& R = h->rep[r];
     const Layout& L = h->L;
@@ -640,6 +681,7 @@ int build_plans(alexnet* h, int r) {
         if ((rc = plan_fc_wg(h, R.fc_wg[l], f, fdy[l], fx[l], R.g + f.w_off, R.w + f.w_off, R.v + f.w_off, R.shadow + f.w_off, fuse))) return rc;
         if ((rc = plan_fc_wg(h, R.fc_wg_plain[l], f, fdy[l], fx[l], R.g + f.w_off, R.w + f.w_off, R.v + f.w_off, R.shadow + f.w_off, false))) return rc;
     }
+    plan_fc_chain(h, r);
     return ALEXNET_OK;
 }
 
@@ -856,6 +898,54 @@ void op_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
     h->launches += 2;
 }
 // fc8's split reduction + bias, softmax cross-entropy and the mean loss in one launch (the step's form; N <= 1024)
+// fc6 -> fc7 -> fc8 (partials) in one cooperative launch; false when the driver refuses the launch (the caller then runs the
+// three layers one by one, and the chain stays off)
+bool op_fc_chain(alexnet* h, int r, uint64_t step, cudaStream_t st, bool eval) {
+    Replica& R = h->rep[r];
+    tc::FcChainParams& q = R.chain;
+    for (int l = 0; l < 2; ++l) {
+        int drop = h->cfg.dropout_p > 0.f;
+        float scale = h->drop_scale;
+        if (eval && drop) { drop = 2; scale = (h->cfg.flags & ALEXNET_FLAG_INVERTED_DROPOUT) ? 1.f : 1.f - h->cfg.dropout_p; }
+        q.L[l].dropout = drop; q.L[l].scale = scale; q.L[l].thr24 = h->thr24;
+        q.L[l].key = kn::stream_key(h->cfg.seed, 2 + l, r, step);
+    }
+    q.gate_base = R.chain_gate;
+    const int grid = R.fc_fwd[0].c.tiles_total;
+    if (h->prof) {
+        while (h->prof_ev.size() < h->prof_used + 2) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) { h->prof = false; break; }
+            h->prof_ev.push_back(e);
+        }
+    }
+    if (h->prof) cudaEventRecord(h->prof_ev[h->prof_used], st);
+    cudaError_t e = cudaErrorUnknown;
+    for (; R.chain_mode && R.chain_mode <= 2; ++R.chain_mode) {
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3(grid); lc.blockDim = dim3(tc::kChainThreads); lc.dynamicSmemBytes = tc::fc_chain_smem_bytes(); lc.stream = st;
+        cudaLaunchAttribute at[3] = {};
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = tc::kChainCluster; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        at[1].id = cudaLaunchAttributeCooperative;
+        at[1].val.cooperative = 1;
+        at[2].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[2].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = at; lc.numAttrs = R.chain_mode == 1 ? 3 : 2;
+        e = cudaLaunchKernelEx(&lc, tc::fc_chain_kernel, q);
+        if (e == cudaSuccess) break;
+        cudaGetLastError();      // a refused launch configuration is not sticky: try the next form
+    }
+    if (e != cudaSuccess) { R.chain_mode = 0; return false; }
+    R.chain_gate += (unsigned)(q.nlayers - 1) * (unsigned)grid;
+    if (h->prof) {
+        cudaEventRecord(h->prof_ev[h->prof_used + 1], st);
+        h->prof_kind.push_back(3);
+        h->prof_used += 2;
+    }
+    h->launches++;
+    return true;
+}
 void op_fc8_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
     Replica& R = h->rep[r];
     const FcL& f = h->L.fc[2];
@@ -937,7 +1027,9 @@ void forward(alexnet* h, int r, int slot, cudaStream_t st, bool eval) {
     op_conv_fwd(h, r, 1, slot, st); op_lrn_pool_fwd(h, r, 1, st);
     op_conv_fwd(h, r, 2, slot, st); op_conv_fwd(h, r, 3, slot, st); op_conv_fwd(h, r, 4, slot, st);
     op_pool_fwd(h, r, 2, st);
-    op_fc_fwd(h, r, 0, step, st, eval); op_fc_fwd(h, r, 1, step, st, eval); op_fc_fwd(h, r, 2, step, st, eval, true);
+    if (!R.chain_mode || !op_fc_chain(h, r, step, st, eval)) {
+        op_fc_fwd(h, r, 0, step, st, eval); op_fc_fwd(h, r, 1, step, st, eval); op_fc_fwd(h, r, 2, step, st, eval, true);
+    }
     op_fc8_softmax(h, r, slot, st);
 }
 void forward_backward(alexnet* h, int r, int slot, cudaStream_t st, bool plain_fc = false) {
@@ -1156,6 +1248,7 @@ int alexnet_create(const alexnet_config_t* cfg, void* dev_arena, size_t arena_by
     CKC(cudaFuncSetAttribute(tc::conv_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::conv_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     CKC(cudaFuncSetAttribute(tc::wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    CKC(cudaFuncSetAttribute(tc::fc_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
     // (static + dynamic shared memory of both exceeds the 48 KB that need no opt-in)
     CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(true), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 48));
     CKC(cudaFuncSetAttribute(POOL_LRN_BWD_1(false), cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 55 * 12 * 48));
@@ -1572,6 +1665,10 @@ int alexnet_run_op(alexnet_t* h, int replica, int op, int iters) {
         else if (op == ALEXNET_OP_POOL1_LRN1_BWD || op == ALEXNET_OP_POOL2_LRN2_BWD) op_pool_lrn_bwd(h, replica, op - ALEXNET_OP_POOL1_LRN1_BWD, st);
         else if (op == ALEXNET_OP_UPDATE_AVERAGE) op_update_average(h, st);
         else if (op == ALEXNET_OP_SCALE_REFRESH) op_scale_refresh(h, replica, 1.f, st);
+        else if (op == ALEXNET_OP_FC_CHAIN_FWD) {
+            if (!R.chain_mode || !op_fc_chain(h, replica, R.slot_step[slot], st, false))
+                return fail(h, ALEXNET_ERR_STATE, "the FC forward chain is not available in this configuration");
+        }
     }
     CK(cudaGetLastError());
     return ALEXNET_OK;

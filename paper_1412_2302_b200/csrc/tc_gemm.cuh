@@ -1175,6 +1175,326 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
 }
 
 // ===========================================================================
+// FC forward chain: the three fully connected layers of the forward pass in ONE launch.
+//
+// At batch <= 128 an FC layer is a stream of weights (117 MB of bf16 for the three layers) against one 128-row tile of
+// activations, and a launch per layer spends as long on its set-up, first loads and exposed epilogue as on the stream.
+// Here the grid (128 CTAs, clusters of four) walks fc6 -> fc7 -> fc8 with one (128-column tile, k split) unit per CTA and
+// layer.  The weight producer never waits for a layer boundary: while a layer's epilogue and the hand-over run, the
+// ring already fills with the next layer's weights, so HBM stays busy.  Only the activation producer waits: a layer's
+// input is the previous layer's output, stored by every CTA, so the CTAs count themselves on a grid-wide gate (a counter
+// in global memory; the launch is cooperative, all CTAs are resident) and the producer reads past it with an
+// acquire load and a proxy fence before its TMA loads.  All waits are bounded.
+// fc6 / fc7: the four splits of a tile are one cluster and reduce their fp32 partial tiles through distributed shared
+// memory with bias, ReLU and dropout applied (the arithmetic and order of conv_kernel's cluster form: bit-identical);
+// fc8: fp32 partials per split to global memory, reduced by the softmax kernel that follows.
+// Unit -> (tile, split) and the rotation of the reduction order are those of the per-layer launches.
+// Warps: 0 = activation producer, 1 = weight producer, 2 = MMA issuer, 3..10 = two sets of four epilogue warps.
+struct FcChainLayer {
+    CUtensorMap tmA, tmB;        // activations [B][K], box {64, 128}; weights [N][K], box {64, 128}
+    int n_tiles, splits, per;    // 128-column tiles; k splits; steps (of 128 channels) per split
+    int asteps_total, n_valid;
+    int cluster_reduce;          // 1: the splits of a tile are the CTAs of a cluster (splits == kChainCluster)
+    int relu, dropout;           // dropout: 0 none, 1 mask from the hash, 2 evaluation (expectation of the mask)
+    uint32_t thr24; float scale; uint64_t key;
+    const float* bias; __nv_bfloat16* out; uint8_t* keep;     // cluster_reduce layers
+    float* partial; long long split_stride;                   // other layers: [split][B][n_valid] fp32
+};
+struct FcChainParams {
+    FcChainLayer L[3];
+    int nlayers, M_total;
+    int* status;
+    unsigned* gate; unsigned gate_base;     // grid gate: counter and its value when the launch starts
+};
+constexpr int kChainThreads = 32 * 11, kChainCluster = 4, kChainAStages = 3, kChainBStages = 4;
+constexpr uint32_t kChainStageBytes = 32768;      // two 64-channel boxes of 128 rows
+inline size_t fc_chain_smem_bytes() { return 1024 + (size_t)(kChainAStages + kChainBStages) * kChainStageBytes + 512; }
+
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
+    unsigned v; asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory"); return v;
+}
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kChainThreads, 1) fc_chain_kernel(const __grid_constant__ FcChainParams p) {
+    // timeline slots (ns): 0 start, 1 set up, 2 end; issuer: 3 + 2 l first operands of layer l, 4 + 2 l its last commit;
+    // first epilogue thread: 9 + 3 l accumulator of layer l ready, 10 + 3 l partial tiles of the cluster ready, 11 + 3 l stored
+    // and counted on the gate (l = 0, 1); 15: the activation producer passed the first gate
+    TL(long long* tl = g_timeline + (blockIdx.x % 160) * 16; if (threadIdx.x == 0) tl[0] = gtime_ns();)
+    kn::pdl_trigger();
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    const uint32_t ring_a = base, ring_b = base + kChainAStages * kChainStageBytes;
+    const uint32_t bar_base = ring_b + kChainBStages * kChainStageBytes;
+    // barriers: fullA[3] @0, emptyA[3] @24, fullB[4] @48, emptyB[4] @80, acc_full[2] @112, acc_empty[2] @128,
+    // partials-ready (cluster) @144, stored (gate) @152; tmem slot @160, abort flag @168
+    uint8_t* gen = smem_raw + (bar_base - raw);
+    volatile int* abort_flag = (volatile int*)(gen + 168);
+    volatile uint32_t* tmem_slot = (volatile uint32_t*)(gen + 160);
+    const uint32_t fullA = bar_base, emptyA = bar_base + 24u, fullB = bar_base + 48u, emptyB = bar_base + 80u;
+    const uint32_t accf0 = bar_base + 112u, acce0 = bar_base + 128u, xbar = bar_base + 144u, gbar = bar_base + 152u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int zrank = (int)cluster_ctarank(), cid = (int)blockIdx.x / kChainCluster;
+    constexpr uint32_t kCols = 256;      // two accumulators of 128 columns
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < kChainAStages; ++s) { mbar_init(fullA + 8u * s, 1); mbar_init(emptyA + 8u * s, 1); }
+        for (int s = 0; s < kChainBStages; ++s) { mbar_init(fullB + 8u * s, 1); mbar_init(emptyB + 8u * s, 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(accf0 + 8u * s, 1); mbar_init(acce0 + 8u * s, 256); }
+        mbar_init(xbar, 8 * kChainCluster);
+        mbar_init(gbar, 8);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int l = 0; l < p.nlayers; ++l) { tma_prefetch_desc(&p.L[l].tmA); tma_prefetch_desc(&p.L[l].tmB); }
+    }
+    if (warp == 2) tmem_alloc(smem_u32((const void*)tmem_slot), kCols);
+    tc_fence_before();
+    __syncthreads();
+    __syncwarp();
+    cluster_sync_all();          // the peers' barriers exist before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    kn::pdl_wait();
+    TL(if (threadIdx.x == 0) tl[1] = gtime_ns();)
+
+    // this CTA's unit of layer l: position vb in the layer's tile list (split-major), tile and split
+    #define CHAIN_UNIT(L) \
+        int vb, n_tile, z; \
+        if ((L).cluster_reduce) { n_tile = cid; z = zrank; vb = z * (L).n_tiles + n_tile; } \
+        else { vb = (int)blockIdx.x; n_tile = vb % (L).n_tiles; z = vb / (L).n_tiles; } \
+        const int a_begin = z * (L).per; \
+        const int nsteps = min((L).asteps_total, a_begin + (L).per) - a_begin; \
+        (void)vb; (void)n_tile;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ activations
+            int sa = 0; uint32_t pha = 0;
+            bool ok = true;
+            for (int l = 0; l < p.nlayers && ok; ++l) {
+                const FcChainLayer& L = p.L[l];
+                CHAIN_UNIT(L)
+                if (l > 0) {
+                    // the gate: every CTA has stored its part of the previous layer's output
+                    const unsigned target = p.gate_base + (unsigned)l * gridDim.x;
+                    const long long t0 = clock64();
+                    while ((int)(ld_acquire_gpu(p.gate) - target) < 0) {
+                        if (*abort_flag) { ok = false; break; }
+                        if (clock64() - t0 > kWaitBudgetCycles) { *abort_flag = 1; ok = false; break; }
+                    }
+                    if (!ok) break;
+                    TL(if (l == 1) tl[15] = gtime_ns();)
+                    fence_proxy_async_all();     // those stores (generic proxy) before this thread's TMA reads (async proxy)
+                }
+                int a = a_begin + (int)((unsigned)vb % (unsigned)nsteps);
+                for (int i = 0; i < nsteps && ok; ++i) {
+                    ok = mbar_wait(emptyA + 8u * sa, pha ^ 1u, abort_flag);
+                    if (!ok) break;
+                    const uint32_t dst = ring_a + sa * kChainStageBytes, fb = fullA + 8u * sa;
+                    mbar_expect_tx(fb, kChainStageBytes);
+                    tma_load_2d(dst, &L.tmA, a * 128, 0, fb);
+                    tma_load_2d(dst + 16384u, &L.tmA, a * 128 + 64, 0, fb);
+                    if (++sa == kChainAStages) { sa = 0; pha ^= 1u; }
+                    if (++a == a_begin + nsteps) a = a_begin;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ weights: no layer boundary
+            int sb = 0; uint32_t phb = 0;
+            bool ok = true;
+            for (int l = 0; l < p.nlayers && ok; ++l) {
+                const FcChainLayer& L = p.L[l];
+                CHAIN_UNIT(L)
+                int a = a_begin + (int)((unsigned)vb % (unsigned)nsteps);
+                for (int i = 0; i < nsteps && ok; ++i) {
+                    ok = mbar_wait(emptyB + 8u * sb, phb ^ 1u, abort_flag);
+                    if (!ok) break;
+                    const uint32_t dst = ring_b + sb * kChainStageBytes, fb = fullB + 8u * sb;
+                    mbar_expect_tx(fb, kChainStageBytes);
+                    tma_load_2d(dst, &L.tmB, a * 128, n_tile * 128, fb);
+                    tma_load_2d(dst + 16384u, &L.tmB, a * 128 + 64, n_tile * 128, fb);
+                    if (++sb == kChainBStages) { sb = 0; phb ^= 1u; }
+                    if (++a == a_begin + nsteps) a = a_begin;
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ---------------------------------------------------------------- MMA issuer (whole warp)
+        const uint32_t idesc = instr_desc(128, 0, 0, 128);
+        const uint64_t dbase = smem_desc(0, 16, 1024);
+        int sa = 0, sb = 0; uint32_t pha = 0, phb = 0;
+        int ab = 0; uint32_t aph = 0;
+        bool ok = true;
+        for (int l = 0; l < p.nlayers && ok; ++l) {
+            const FcChainLayer& L = p.L[l];
+            CHAIN_UNIT(L)
+            ok = mbar_wait_warp(acce0 + 8u * ab, aph ^ 1u, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d = tmem + (uint32_t)(ab * 128);
+            uint32_t accum = 0;
+            for (int i = 0; i < nsteps && ok; ++i) {
+                ok = mbar_wait_warp(fullA + 8u * sa, pha, abort_flag) && mbar_wait_warp(fullB + 8u * sb, phb, abort_flag);
+                if (!ok) break;
+                TL(if (i == 0 && lane == 0) tl[3 + 2 * l] = gtime_ns();)
+                const uint64_t ad = dbase + (uint64_t)((ring_a + sa * kChainStageBytes) >> 4);
+                const uint64_t bd = dbase + (uint64_t)((ring_b + sb * kChainStageBytes) >> 4);
+                #pragma unroll
+                for (int c = 0; c < 2; ++c)          // the stage's two 64-channel boxes, four K = 16 steps each
+                    #pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        umma(d, ad + (uint64_t)(c * 1024 + 2 * j), bd + (uint64_t)(c * 1024 + 2 * j), idesc, (c == 0 && j == 0) ? accum : 1u);
+                accum = 1;
+                umma_commit(emptyB + 8u * sb);
+                umma_commit(emptyA + 8u * sa);
+                if (++sa == kChainAStages) { sa = 0; pha ^= 1u; }
+                if (++sb == kChainBStages) { sb = 0; phb ^= 1u; }
+            }
+            if (!ok) break;
+            umma_commit(accf0 + 8u * ab);
+            TL(if (lane == 0) tl[4 + 2 * l] = gtime_ns();)
+            if (++ab == 2) { ab = 0; aph ^= 1u; }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue
+        const int quad = warp & 3, ew = warp - 3, eset = ew >> 2;
+        const int r = quad * 32 + lane;          // row of the tile = TMEM lane
+        const int et = ew * 32 + lane;           // 0..255
+        int ab = 0; uint32_t aph = 0, xph = 0, gph = 0;
+        bool ok = true;
+        for (int l = 0; l < p.nlayers && ok; ++l) {
+            const FcChainLayer& L = p.L[l];
+            CHAIN_UNIT(L)
+            ok = mbar_wait(accf0 + 8u * ab, aph, abort_flag);
+            if (!ok) break;
+            TL(if (et == 0 && l < 2) tl[9 + 3 * l] = gtime_ns();)
+            tc_fence_after();
+            const uint32_t t0 = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * 128);
+            const int n0 = n_tile * 128;
+            #pragma unroll 1
+            for (int unit = 0; unit < 4; ++unit) {       // 32-column units alternate between the two sets of warps
+                if ((unit & 1) != eset) continue;
+                const int c = unit * 32;
+                uint32_t v[32];
+                tmem_ld32(t0 + (uint32_t)c, v);
+                tmem_ld_wait();
+                if (nsteps <= 0) {
+                    #pragma unroll
+                    for (int k = 0; k < 32; ++k) v[k] = 0u;
+                }
+                if (L.cluster_reduce) {
+                    // the partial tile stays on chip: in the activation ring, idle until the next layer's gate opens
+                    const uint32_t rowp = ring_a + (uint32_t)(r * kZcPitch + c) * 4u;
+                    #pragma unroll
+                    for (int q = 0; q < 8; ++q) st_shared_v4(rowp + 16u * q, v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                } else if (r < p.M_total) {
+                    float* o = L.partial + (long long)z * L.split_stride + (long long)r * L.n_valid + n0 + c;
+                    #pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        if (n0 + c + 4 * q < L.n_valid)      // n_valid is a multiple of 4
+                            *(float4*)(o + 4 * q) = make_float4(__uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]),
+                                                                __uint_as_float(v[4 * q + 2]), __uint_as_float(v[4 * q + 3]));
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acce0 + 8u * ab);
+            if (++ab == 2) { ab = 0; aph ^= 1u; }
+            if (L.cluster_reduce) {
+                // the four output columns this thread finishes, and their bias (fetched while the cluster gathers)
+                const int c4 = et & 31, n = n0 + 4 * c4;
+                const float4 b4 = n < L.n_valid ? __ldg((const float4*)(L.bias + n)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                // every epilogue warp of the cluster tells all four CTAs that its rows of a partial tile are written (one
+                // arrival per warp: arrivals on one barrier are serialised, a thousand of them cost microseconds)
+                __syncwarp();
+                if (lane == 0) {
+                    #pragma unroll
+                    for (int q = 0; q < kChainCluster; ++q) mbar_arrive_cluster(mapa_u32(xbar, (uint32_t)q));
+                }
+                ok = mbar_wait(xbar, xph, abort_flag);
+                xph ^= 1u;
+                if (!ok) break;
+                TL(if (et == 0 && l < 2) tl[10 + 3 * l] = gtime_ns();)
+                fence_acq_rel_cluster();
+                // this CTA's 32 rows of the four partial tiles: all sixteen remote loads of a thread are in flight together
+                constexpr int rows_per = 128 / kChainCluster, items = rows_per * 32 / 256;
+                float4 part[items][kChainCluster];
+                #pragma unroll
+                for (int it = 0; it < items; ++it) {
+                    const int row = zrank * rows_per + (et >> 5) + 8 * it;
+                    const uint32_t local = ring_a + (uint32_t)(row * kZcPitch + 4 * c4) * 4u;
+                    #pragma unroll
+                    for (int q = 0; q < kChainCluster; ++q)
+                        asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(part[it][q].x), "=f"(part[it][q].y), "=f"(part[it][q].z), "=f"(part[it][q].w)
+                                     : "r"(mapa_u32(local, (uint32_t)q)) : "memory");
+                }
+                #pragma unroll
+                for (int it = 0; it < items; ++it) {
+                    const int row = zrank * rows_per + (et >> 5) + 8 * it;
+                    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                    #pragma unroll
+                    for (int q = 0; q < kChainCluster; ++q) {       // in split order
+                        acc[0] += part[it][q].x; acc[1] += part[it][q].y; acc[2] += part[it][q].z; acc[3] += part[it][q].w;
+                    }
+                    if (row >= p.M_total || n >= L.n_valid) continue;
+                    const long long tt = (long long)row * L.n_valid + n;
+                    const float bb[4] = {b4.x, b4.y, b4.z, b4.w};
+                    uint32_t keepw = 0x01010101u;
+                    #pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        float y = acc[k] + bb[k];
+                        if (L.relu) y = fmaxf(y, 0.f);
+                        if (L.dropout == 2) y *= L.scale;
+                        else if (L.dropout) {
+                            const bool keep = (uint32_t)(kn::draw(L.key, (uint64_t)(tt + k)) >> 40) >= L.thr24;
+                            if (!keep) keepw &= ~(0xFFu << (8 * k));
+                            y = keep ? y * L.scale : 0.f;
+                        }
+                        acc[k] = y;
+                    }
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(acc[0], acc[1]), hi = __floats2bfloat162_rn(acc[2], acc[3]);
+                    *(uint2*)(L.out + tt) = make_uint2(*(const uint32_t*)&lo, *(const uint32_t*)&hi);
+                    if (L.keep) *(uint32_t*)(L.keep + tt) = keepw;
+                }
+            }
+            if (l + 1 < p.nlayers) {
+                // this thread's shared-memory accesses (its rows of the tile, the peers' tiles) come before the TMA
+                // writes of the next layer's activations into the same ring; its global stores before the gate
+                fence_proxy_async_all();
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(gbar);
+                if (et == 0) {
+                    ok = mbar_wait(gbar, gph, abort_flag);
+                    if (ok) { __threadfence(); atomicAdd(p.gate, 1u); }
+                    TL(if (l < 2) tl[11 + 3 * l] = gtime_ns();)
+                }
+                gph ^= 1u;
+            }
+        }
+    }
+    #undef CHAIN_UNIT
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && p.status) atomicExch(p.status, 1);
+        long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) { }
+        __syncthreads();
+    }
+    __syncwarp();
+    cluster_sync_all();          // no CTA leaves while a peer may still read its partial tile or arrive on its barriers
+    TL(if (threadIdx.x == 0) tl[2] = gtime_ns();)
+    if (warp == 2) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kCols);
+    }
+}
+
+// ===========================================================================
 // Convolution weight-gradient kernel.
 //
 //   dW[ky][kx][co][ci] = sum_m dy[m][co] * x[m + shift(ky,kx)][ci]

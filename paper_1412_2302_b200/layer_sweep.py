@@ -47,6 +47,8 @@ def hbm_bytes(B):
         "POOL1_LRN1_BWD": B * (a1 * 4 + p1 * 3), "POOL2_LRN2_BWD": B * (a2 * 4 + p2 * 3),
         "UPDATE_AVERAGE": PARAMS * 44,                              # r w,v,g of both replicas; w w,v and bf16 copy of both
         "SCALE_REFRESH": PARAMS * 6,                                # scale 1: r w, w bf16 copy
+        # fc6 -> fc7 -> fc8 forward in one launch: the bf16 weights once, activations in and out, fc8's split partials
+        "FC_CHAIN_FWD": 2 * (MACS["FC6"] + MACS["FC7"] + MACS["FC8"]) + B * (9216 + 2 * 4096 * 3) + B * 1000 * 4 * 16,
     }
     return d
 
@@ -71,11 +73,11 @@ def main(argv=None):
 
     import torch
     from . import synth
-    from .alexnet import OPS, AlexNet
+    from .alexnet import FLAG_FC_CHAIN, OPS, AlexNet, AlexNetError
 
     B = args.batch
     seed = synth.BASE_SEED + 5
-    net = AlexNet(batch=B, replicas=2, seed=seed, mean_image=synth.mean_image(seed))
+    net = AlexNet(batch=B, replicas=2, seed=seed, mean_image=synth.mean_image(seed), flags=FLAG_FC_CHAIN)
     w = synth.init_params(seed, variance_preserving=True)
     net.set_params(w, 0)
     net.set_params(w, 1)
@@ -93,8 +95,13 @@ def main(argv=None):
     names = args.ops.split(",") if args.ops else OPS
     with torch.cuda.stream(cs):
         for name in names:
-            for _ in range(3):
-                net.run_op(name)
+            try:
+                for _ in range(3):
+                    net.run_op(name)
+            except AlexNetError:
+                if name != "FC_CHAIN_FWD":
+                    raise
+                continue              # the one-launch FC forward exists at batch <= 128 only
             ts = []
             for _ in range(args.iters):
                 flush.fill_(1)

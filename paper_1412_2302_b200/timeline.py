@@ -25,6 +25,15 @@ CONV_OPS = ["CONV1_FWD", "CONV2_FWD", "CONV3_FWD", "CONV4_FWD", "CONV5_FWD", "CO
             "CONV4_BWD_DATA", "CONV5_BWD_DATA", "FC6_FWD", "FC7_FWD", "FC8_FWD"]
 
 
+# fc_chain_kernel's slots, in the order the events happen
+CHAIN_SLOTS = [(1, "set up"), (3, "fc6: first operands at the issuer"), (4, "fc6: last instruction committed"),
+               (9, "fc6: accumulator at the epilogue"), (10, "fc6: the cluster's four partial tiles in shared memory"),
+               (11, "fc6: reduced, stored and counted on the gate"), (15, "gate open: fc7's activations may be loaded"),
+               (5, "fc7: first operands"), (6, "fc7: last instruction committed"), (12, "fc7: accumulator at the epilogue"),
+               (13, "fc7: the cluster's partial tiles"), (14, "fc7: reduced, stored and counted on the gate"),
+               (7, "fc8: first operands"), (8, "fc8: last instruction committed"), (2, "end")]
+
+
 def read(lib, clear):
     buf = np.zeros((160, 16), np.int64)
     rc = lib.alexnet_timeline_read(ctypes.c_void_p(buf.ctypes.data), 1 if clear else 0)
@@ -68,10 +77,10 @@ def main(argv=None):
     _build.LIB = _build.LIB_TIMELINE          # the binding loads this variant
     import torch
     from . import synth
-    from .alexnet import AlexNet
+    from .alexnet import FLAG_FC_CHAIN, AlexNet
     B = args.batch
     seed = synth.BASE_SEED + 5
-    net = AlexNet(batch=B, replicas=1, seed=seed, mean_image=synth.mean_image(seed))
+    net = AlexNet(batch=B, replicas=1, seed=seed, mean_image=synth.mean_image(seed), flags=FLAG_FC_CHAIN if B <= 128 else 0)
     net.set_params(synth.init_params(seed, variance_preserving=True))
     img = torch.from_numpy(synth.images(seed, 0, 0, B)).pin_memory()
     lab = torch.from_numpy(synth.labels(seed, 0, 0, B)).pin_memory()
@@ -93,6 +102,22 @@ def main(argv=None):
                   f"{r.get('loop_us', 0):>8.1f}{r.get('cycles_per_instruction', 0):>9.0f}{r.get('cycles_per_instruction_outside_waits', 0):>7.0f}"
                   f"{100 * w['activations']:>7.0f}/{100 * w['weights']:.0f}/{100 * w['accumulator']:.0f}"
                   f"{r.get('last_instruction_to_last_store_us', 0):>10.1f}{r.get('last_instruction_to_exit_us', 0):>9.1f}")
+    # the one-launch FC forward (ALEXNET_FLAG_FC_CHAIN): where the time between its three weight streams goes
+    if not args.ops and B <= 128:
+        print("# FC_CHAIN_FWD: us since the first CTA started, mean / min / max over the 128 CTAs")
+        for mode, n in (("single", 1), ("in a burst", 3)):
+            net.run_op("FC_CHAIN_FWD", iters=2)
+            net.sync()
+            read(net.lib, True)
+            net.run_op("FC_CHAIN_FWD", iters=n)
+            net.sync()
+            d = read(net.lib, True)
+            d = d[d[:, 0] > 0]
+            t0 = d[:, 0].min()
+            print(f"  [{mode}] span {(d[:, 2].max() - t0) / 1e3:.1f} us")
+            for k, what in CHAIN_SLOTS:
+                v = (d[:, k] - t0) / 1e3
+                print(f"    {what:<58}{v.mean():>8.2f}{v.min():>8.2f}{v.max():>8.2f}")
     net.close()
 
 

@@ -381,6 +381,47 @@ def test_fused_fc_update_gives_the_same_parameters():
     assert not np.array_equal(w0, w)
 
 
+def test_fc_forward_chain_equals_three_launches():
+    """ALEXNET_FLAG_FC_CHAIN: fc6 -> fc7 -> fc8 forward as one cooperative launch against the three per-layer launches:
+    same units, same summation order, so activations, dropout masks, logits, losses and the parameters after three steps
+    are bit-identical; also the evaluation pass; at a full and at a ragged row tile."""
+    from paper_1412_2302_b200 import alexnet as A
+    for B in (128, 40):
+        seed = BASE + 14
+        w = synth.init_params(seed, variance_preserving=True, bias=0.1)
+        res = []
+        for flags in (A.FLAG_FUSED_FC_UPDATE | A.FLAG_FC_CHAIN, A.FLAG_FUSED_FC_UPDATE):
+            net = make(B, seed=seed, flags=flags)
+            net.set_params(w)
+            losses, acts = [], None
+            for step in range(3):
+                load(net, 0, seed, step, B)
+                losses.append(net.train_step(0, want_loss=True))
+                if step == 0:
+                    acts = [net.get_tensor(t) for t in ("F6", "M6", "F7", "M7", "Z", "DZ")]
+            chain = True
+            try:
+                net.run_op("FC_CHAIN_FWD")
+            except A.AlexNetError as e:
+                chain = False
+                assert e.code == A.ERR_STATE
+            if flags & A.FLAG_FC_CHAIN and not chain:
+                net.close()
+                pytest.skip("this device cannot hold the chain's 32 clusters of four CTAs at once")
+            assert chain == bool(flags & A.FLAG_FC_CHAIN)
+            img, lab = torch.from_numpy(synth.images(seed, 0, 7, B)).cuda(), torch.from_numpy(synth.labels(seed, 0, 7, B)).cuda()
+            ev = net.eval_batch(0, img, lab)
+            res.append((losses, acts, net.get_params(0, 0), net.get_params(0, 1), ev, net.launch_count))
+            net.close()
+        (l0, a0, w0, v0, e0, n0), (l1, a1, w1, v1, e1, n1) = res
+        assert l0 == l1 and e0 == e1
+        for x, y in zip(a0, a1):
+            assert np.array_equal(x, y)
+        assert 0 < a0[1].mean() < 1                      # a real dropout mask
+        assert np.array_equal(w0, w1) and np.array_equal(v0, v1)
+        assert n0 < n1                                    # two launches fewer per forward pass
+
+
 def test_loss_async_delivers_the_step_loss():
     """alexnet_loss_async queues the copy of the last step's loss behind the step; after a sync it equals the loss
     train_step returns when it is asked to wait, and error paths are checked."""
