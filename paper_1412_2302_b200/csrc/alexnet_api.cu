@@ -688,7 +688,13 @@ int build_plans(alexnet* h, int r) {
 // ---------------------------------------------------------------- launches
 inline int nblk(long long n, int t) { return (int)((n + t - 1) / t); }
 
-void launch_gemm(alexnet* h, const Plan& P, cudaStream_t st) {
+// early_weights: the launch is part of a forward or backward pass whose earlier kernels (and whatever may still run beside
+// them) never write this layer's bf16 weights, so conv_kernel may load them before its predecessor has finished
+void launch_gemm(alexnet* h, const Plan& P0, cudaStream_t st, bool early_weights = false) {
+    Plan Pl;
+    const Plan* Pp = &P0;
+    if (early_weights && P0.conv) { Pl = P0; Pl.c.early_b = 1; Pp = &Pl; }
+    const Plan& P = *Pp;
     if (h->prof) {
         while (h->prof_ev.size() < h->prof_used + 2) {
             cudaEvent_t e;
@@ -756,8 +762,10 @@ void refresh_transposed_both(alexnet* h, cudaStream_t st) {
     h->launches++;
 }
 
-void op_conv_fwd(alexnet* h, int r, int l, int slot, cudaStream_t st) { launch_gemm(h, h->rep[r].conv_fwd[l][slot], st); }
-void op_conv_bwd(alexnet* h, int r, int l, cudaStream_t st) { launch_gemm(h, h->rep[r].conv_bwd[l], st); }
+void op_conv_fwd(alexnet* h, int r, int l, int slot, cudaStream_t st, bool early_weights = false) {
+    launch_gemm(h, h->rep[r].conv_fwd[l][slot], st, early_weights);
+}
+void op_conv_bwd(alexnet* h, int r, int l, cudaStream_t st, bool early_weights = false) { launch_gemm(h, h->rep[r].conv_bwd[l], st, early_weights); }
 void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
     Replica& R = h->rep[r];
     const ConvL& c = h->L.conv[l];
@@ -768,7 +776,8 @@ void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
              R.g + c.w_off, l == 0, h->bias_partial + (size_t)l * kBiasPartial, c.cout, R.g + c.b_off);
     h->launches++;
 }
-void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool eval = false, bool gemm_only = false) {
+void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool eval = false, bool gemm_only = false,
+               bool early_weights = false) {
     Replica& R = h->rep[r];
     const FcL& f = h->L.fc[l];
     Plan& P = R.fc_fwd[l];
@@ -784,10 +793,10 @@ void op_fc_fwd(alexnet* h, int r, int l, uint64_t step, cudaStream_t st, bool ev
     if (P.c.zcluster) {      // reduction, bias, ReLU and dropout inside the GEMM kernel (a cluster per tile)
         P.c.fc_relu = 1; P.c.fc_dropout = drop; P.c.fc_key = key; P.c.fc_thr24 = h->thr24; P.c.fc_scale = scale;
         P.c.fc_out = outs[l]; P.c.fc_keep = keeps[l];
-        launch_gemm(h, P, st);
+        launch_gemm(h, P, st, early_weights);
         return;
     }
-    launch_gemm(h, P, st);
+    launch_gemm(h, P, st, early_weights);
     if (gemm_only) return;     // the split reduction is part of the kernel that follows (fc8 inside the step)
     const long long total = (long long)h->B * f.N;
     launch_k(kn::fc_reduce_fwd_kernel, nblk(total, 256), 256, 0, st, h->ws, P.c.splits, P.c.split_stride, R.w + f.b_off, h->B, f.N,
@@ -1023,12 +1032,15 @@ void op_preprocess(alexnet* h, int r, int slot, uint64_t step, cudaStream_t st, 
 void forward(alexnet* h, int r, int slot, cudaStream_t st, bool eval) {
     Replica& R = h->rep[r];
     const uint64_t step = R.slot_step[slot];
+    // conv1 may directly follow the kernel that wrote its weights (the update of the step before): it waits in full.  Its
+    // CTAs hold every SM until it ends, so no later kernel of the pass can start (and read weights) before that writer is done.
     op_conv_fwd(h, r, 0, slot, st); op_lrn_pool_fwd(h, r, 0, st);
-    op_conv_fwd(h, r, 1, slot, st); op_lrn_pool_fwd(h, r, 1, st);
-    op_conv_fwd(h, r, 2, slot, st); op_conv_fwd(h, r, 3, slot, st); op_conv_fwd(h, r, 4, slot, st);
+    op_conv_fwd(h, r, 1, slot, st, true); op_lrn_pool_fwd(h, r, 1, st);
+    op_conv_fwd(h, r, 2, slot, st, true); op_conv_fwd(h, r, 3, slot, st, true); op_conv_fwd(h, r, 4, slot, st, true);
     op_pool_fwd(h, r, 2, st);
     if (!R.chain_mode || !op_fc_chain(h, r, step, st, eval)) {
-        op_fc_fwd(h, r, 0, step, st, eval); op_fc_fwd(h, r, 1, step, st, eval); op_fc_fwd(h, r, 2, step, st, eval, true);
+        op_fc_fwd(h, r, 0, step, st, eval, false, true); op_fc_fwd(h, r, 1, step, st, eval, false, true);
+        op_fc_fwd(h, r, 2, step, st, eval, true, true);
     }
     op_fc8_softmax(h, r, slot, st);
 }
@@ -1058,11 +1070,12 @@ void forward_backward(alexnet* h, int r, int slot, cudaStream_t st, bool plain_f
         else { op_fc_wg(h, r, l, l == 2, st); op_fc_bwd(h, r, l, st); }
     }
     op_pool_bwd(h, r, 2, st);
-    op_conv_wg(h, r, 4, slot, branch(3 + 4)); op_conv_bwd(h, r, 4, st);
-    op_conv_wg(h, r, 3, slot, branch(3 + 3)); op_conv_bwd(h, r, 3, st);
-    op_conv_wg(h, r, 2, slot, branch(3 + 2)); op_conv_bwd(h, r, 2, st);
+    // (the transposed bf16 filters that the data gradients read are written between steps only: they may load early)
+    op_conv_wg(h, r, 4, slot, branch(3 + 4)); op_conv_bwd(h, r, 4, st, true);
+    op_conv_wg(h, r, 3, slot, branch(3 + 3)); op_conv_bwd(h, r, 3, st, true);
+    op_conv_wg(h, r, 2, slot, branch(3 + 2)); op_conv_bwd(h, r, 2, st, true);
     op_pool_lrn_bwd(h, r, 1, st);
-    op_conv_wg(h, r, 1, slot, branch(3 + 1)); op_conv_bwd(h, r, 1, st);
+    op_conv_wg(h, r, 1, slot, branch(3 + 1)); op_conv_bwd(h, r, 1, st, true);
     op_pool_lrn_bwd(h, r, 0, st);
     op_conv_wg(h, r, 0, slot, branch(3 + 0));
     for (int b = 0; b < alexnet::kBranches; ++b)

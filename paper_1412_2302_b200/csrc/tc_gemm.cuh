@@ -784,6 +784,10 @@ struct ConvParams {
     int fc_relu, fc_dropout;       // fc_dropout: 0 none, 1 mask from the hash, 2 evaluation (expectation of the mask)
     uint64_t fc_key; uint32_t fc_thr24; float fc_scale;
     __nv_bfloat16* fc_out; uint8_t* fc_keep;
+    // 1: the weight producer does not wait for the kernel before this one in the stream (programmatic dependent launch):
+    // the caller knows that no kernel that may still be running writes the weights, so their first stages load while
+    // the predecessor drains.  Every other role waits as usual.
+    int early_b;
 };
 constexpr int kZcPitch = 132;      // floats per row of the partial tile in shared memory (128 + 4: conflict-free float4 rows)
 
@@ -888,7 +892,8 @@ __global__ void __launch_bounds__(kConvMaxThreads, 1) conv_kernel(const __grid_c
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
     TL(if (threadIdx.x == 0) tl[12] = gtime_ns();)
-    kn::pdl_wait();        // barriers, TMEM and descriptors are set up; global memory is touched from here on
+    // barriers, TMEM and descriptors are set up; global memory is touched from here on (the weights possibly earlier)
+    if (!(p.early_b && warp == 1)) kn::pdl_wait();
     TL(if (threadIdx.x == 0) tl[1] = gtime_ns();)
     const int per = p.asteps_per_split, kw = p.kw;
 
