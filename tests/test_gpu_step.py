@@ -422,6 +422,29 @@ def test_fc_forward_chain_equals_three_launches():
         assert n0 < n1                                    # two launches fewer per forward pass
 
 
+def test_fc_forward_chain_with_two_replicas():
+    """The chain keeps one gate per replica: two replicas stepping in turn, with the exchange between, give the same
+    parameters with and without ALEXNET_FLAG_FC_CHAIN."""
+    from paper_1412_2302_b200 import alexnet as A
+    seed, B = BASE + 15, 16
+    w = synth.init_params(seed, variance_preserving=True, bias=0.1)
+    res = []
+    for flags in (A.FLAG_FC_CHAIN, 0):
+        net = make(B, replicas=2, seed=seed, flags=flags)
+        net.set_params(w, 0)
+        net.set_params(w, 1)
+        for step in range(3):
+            for r in (0, 1):
+                load(net, r, seed, step, B)
+                net.train_step(r)
+            net.replica_average()
+        res.append((net.get_params(0, 0), net.get_params(1, 0), net.get_params(0, 1), net.launch_count))
+        net.close()
+    (a0, b0, v0, n0), (a1, b1, v1, n1) = res
+    assert np.array_equal(a0, b0) and np.array_equal(a0, a1) and np.array_equal(v0, v1)
+    assert n0 <= n1
+
+
 def test_loss_async_delivers_the_step_loss():
     """alexnet_loss_async queues the copy of the last step's loss behind the step; after a sync it equals the loss
     train_step returns when it is asked to wait, and error paths are checked."""
