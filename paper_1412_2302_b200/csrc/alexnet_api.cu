@@ -813,7 +813,7 @@ void op_fc_bwd(alexnet* h, int r, int l, cudaStream_t st) {
     bf16* outs[3] = {R.dp5, R.df6, R.df7};
     // the data gradient of layer l is the output gradient of layer l-1: its column sums are that layer's bias gradient
     float* db = l > 0 ? R.g + h->L.fc[l - 1].b_off : nullptr;
-    launch_k(kn::fc_reduce_bwd_kernel, nblk(f.K, 32), 1024, 0, st, h->ws, P.p.splits, P.p.split_stride, masks[l], h->drop_scale, h->B, f.K,
+    launch_k(kn::fc_reduce_bwd_kernel, nblk(f.K, 32), 256, 0, st, h->ws, P.p.splits, P.p.split_stride, masks[l], h->drop_scale, h->B, f.K,
                                                            outs[l], db);
     h->launches++;
 }

@@ -525,33 +525,62 @@ __global__ void fc_reduce_fwd_kernel(const float* __restrict__ ws, int splits, l
 }
 // dx[b][k] = [mask[b][k] > 0] * scale * sum_z ws[z][b][k] -> bf16 (mask = the layer input, post ReLU and dropout);
 // db[k] = sum_b dx[b][k] (of the bf16-rounded values: the bias gradient of the layer below), when db != nullptr.
-// grid: K/32 blocks of 1024 threads = 32 columns x 32 row lanes.
-__global__ void __launch_bounds__(1024) fc_reduce_bwd_kernel(const float* __restrict__ ws, int splits, long long split_stride,
-                                                             const __nv_bfloat16* __restrict__ mask, float scale, int B, int K,
-                                                             __nv_bfloat16* __restrict__ out, float* __restrict__ db) {
+// grid: K/32 blocks of 256 threads = 8 column quads x 32 row lanes; a thread owns four columns of the rows rl, rl + 32, ...
+// (batch <= 128: at most four) and has all its loads in flight together.  K is a multiple of 4; larger batches take the
+// rows in rounds of 128.
+__global__ void __launch_bounds__(256) fc_reduce_bwd_kernel(const float* __restrict__ ws, int splits, long long split_stride,
+                                                            const __nv_bfloat16* __restrict__ mask, float scale, int B, int K,
+                                                            __nv_bfloat16* __restrict__ out, float* __restrict__ db) {
     pdl_sync();
     __shared__ float red[32][33];
-    const int c = blockIdx.x * 32 + (threadIdx.x & 31), rl = threadIdx.x >> 5;
-    float acc = 0.f;
+    const int cq = threadIdx.x & 7, rl = threadIdx.x >> 3;
+    const int c = blockIdx.x * 32 + 4 * cq;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
     if (c < K) {
-        for (int b = rl; b < B; b += 32) {
-            const size_t t = (size_t)b * K + c;
-            float v = 0.f;
-            for (int z = 0; z < splits; ++z) v += ws[z * split_stride + t];
-            if (mask) v = __bfloat162float(mask[t]) > 0.f ? v * scale : 0.f;
-            const __nv_bfloat16 o = __float2bfloat16_rn(v);
-            out[t] = o;
-            acc += __bfloat162float(o);
+        for (int b0 = 0; b0 < B; b0 += 128) {
+            float4 v[4];
+            uint2 mk[4];
+            #pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int b = b0 + rl + 32 * i;
+                v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+                mk[i] = make_uint2(0u, 0u);
+                if (b < B) {
+                    const size_t t = (size_t)b * K + c;
+                    if (mask) mk[i] = __ldg((const uint2*)(mask + t));
+                    for (int z = 0; z < splits; ++z) {
+                        const float4 w = __ldg((const float4*)(ws + z * split_stride + t));
+                        v[i].x += w.x; v[i].y += w.y; v[i].z += w.z; v[i].w += w.w;
+                    }
+                }
+            }
+            #pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int b = b0 + rl + 32 * i;
+                if (b >= B) continue;
+                float f[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+                if (mask) {
+                    const __nv_bfloat162* m2 = (const __nv_bfloat162*)&mk[i];
+                    const float2 ma = __bfloat1622float2(m2[0]), mb = __bfloat1622float2(m2[1]);
+                    f[0] = ma.x > 0.f ? f[0] * scale : 0.f; f[1] = ma.y > 0.f ? f[1] * scale : 0.f;
+                    f[2] = mb.x > 0.f ? f[2] * scale : 0.f; f[3] = mb.y > 0.f ? f[3] * scale : 0.f;
+                }
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(f[0], f[1]), hi = __floats2bfloat162_rn(f[2], f[3]);
+                *(uint2*)(out + (size_t)b * K + c) = make_uint2(*(const uint32_t*)&lo, *(const uint32_t*)&hi);
+                const float2 ra = __bfloat1622float2(lo), rb = __bfloat1622float2(hi);
+                acc[0] += ra.x; acc[1] += ra.y; acc[2] += rb.x; acc[3] += rb.y;
+            }
         }
     }
     if (!db) return;
-    red[rl][threadIdx.x & 31] = acc;
+    #pragma unroll
+    for (int k = 0; k < 4; ++k) red[rl][4 * cq + k] = acc[k];
     __syncthreads();
-    if (threadIdx.x < 32 && c < K) {
+    if (threadIdx.x < 32 && blockIdx.x * 32 + threadIdx.x < K) {
         float s = 0.f;
         #pragma unroll
         for (int q = 0; q < 32; ++q) s += red[q][threadIdx.x];
-        db[c] = s;
+        db[blockIdx.x * 32 + threadIdx.x] = s;
     }
 }
 // g[i] = sum_z ws[z][i]; conv1: entries of the 12x12 zero-padded filter outside 11x11 stay zero.
