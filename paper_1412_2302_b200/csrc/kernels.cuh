@@ -695,18 +695,37 @@ __global__ void __launch_bounds__(256) fc8_softmax_xent_kernel(const float* __re
                                                                int* __restrict__ done_counter, int B, int N) {
     pdl_sync();
     __shared__ float red[32];
-    __shared__ float zs[1024];
+    __shared__ __align__(16) float zs[1024];
     __shared__ int last;
     const int n = blockIdx.x, tid = threadIdx.x;
     float mx = -INFINITY;
-    for (int j = tid; j < N; j += 256) {
-        const long long t = (long long)n * N + j;
-        float v = 0.f;
-        for (int q = 0; q < splits; ++q) v += ws[q * split_stride + t];
-        v += bias[j];
-        z[t] = v;
-        zs[j] = v;
-        mx = fmaxf(mx, v);
+    if ((N & 3) == 0) {
+        // four columns per thread, the loads of all splits in flight together (the maximum does not depend on which thread
+        // sees which column; the sums below keep the column -> thread mapping of softmax_xent_kernel)
+        for (int j = 4 * tid; j < N; j += 1024) {
+            const long long t = (long long)n * N + j;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            #pragma unroll 4
+            for (int q = 0; q < splits; ++q) {
+                const float4 w = __ldg((const float4*)(ws + q * split_stride + t));
+                v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+            }
+            const float4 b4 = __ldg((const float4*)(bias + j));
+            v.x += b4.x; v.y += b4.y; v.z += b4.z; v.w += b4.w;
+            *(float4*)(z + t) = v;
+            *(float4*)(zs + j) = v;
+            mx = fmaxf(fmaxf(mx, fmaxf(v.x, v.y)), fmaxf(v.z, v.w));
+        }
+    } else {
+        for (int j = tid; j < N; j += 256) {
+            const long long t = (long long)n * N + j;
+            float v = 0.f;
+            for (int q = 0; q < splits; ++q) v += ws[q * split_stride + t];
+            v += bias[j];
+            z[t] = v;
+            zs[j] = v;
+            mx = fmaxf(mx, v);
+        }
     }
     for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(~0u, mx, o));
     if ((tid & 31) == 0) red[tid >> 5] = mx;
