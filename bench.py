@@ -63,7 +63,7 @@ def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return d.get("bf16_tflops", 1651.8), d.get("bf16_tflops_sustained", 1391.0), d.get("hbm_gbs", 6545.9), "measured"
+        return d.get("bf16_tflops", 1685.7), d.get("bf16_tflops_sustained", 1394.1), d.get("hbm_gbs", 6451.5), "measured"
     return 1590.0, 1400.0, 6650.0, "fallback"
 
 
