@@ -766,11 +766,13 @@ void op_conv_fwd(alexnet* h, int r, int l, int slot, cudaStream_t st, bool early
     launch_gemm(h, h->rep[r].conv_fwd[l][slot], st, early_weights);
 }
 void op_conv_bwd(alexnet* h, int r, int l, cudaStream_t st, bool early_weights = false) { launch_gemm(h, h->rep[r].conv_bwd[l], st, early_weights); }
-void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st) {
+// reduce == false: the split partials stay as they are; the update that follows the pass adds them (op_update with a slot)
+void op_conv_wg(alexnet* h, int r, int l, int slot, cudaStream_t st, bool reduce = true) {
     Replica& R = h->rep[r];
     const ConvL& c = h->L.conv[l];
     const Plan& P = R.conv_wg[l][slot];
     launch_gemm(h, P, st);     // weight-gradient partials per row split, and the bias-gradient partials
+    if (!reduce) return;
     const long long total = (long long)c.taps * c.cout * c.cig;
     launch_k(kn::wgrad_reduce_kernel, nblk(total, 256), 256, 0, st, h->ws + h->ws_conv_off[l], P.w.splits, P.w.split_stride, total,
              R.g + c.w_off, l == 0, h->bias_partial + (size_t)l * kBiasPartial, c.cout, R.g + c.b_off);
@@ -963,7 +965,12 @@ void op_fc8_softmax(alexnet* h, int r, int slot, cudaStream_t st) {
              R.loss_n, R.loss, h->status + 8, h->B, f.N);
     h->launches++;
 }
-void op_update(alexnet* h, int r, cudaStream_t st, bool full = false, float gscale = 1.f) {
+// The conv split reduction may ride in the update launch when that launch takes the conv filters and every bias in one go
+bool update_can_reduce_conv(const alexnet* h) {
+    return (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) && !(h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES);
+}
+// reduce_slot >= 0: the conv weight-gradient kernels of that batch slot left their split partials unreduced (see op_conv_wg)
+void op_update(alexnet* h, int r, cudaStream_t st, bool full = false, float gscale = 1.f, int reduce_slot = -1) {
     Replica& R = h->rep[r];
     const Layout& L = h->L;
     const long long nd = (h->cfg.flags & ALEXNET_FLAG_WD_ON_BIASES) ? L.n_total : L.n_weights;
@@ -974,13 +981,26 @@ void op_update(alexnet* h, int r, cudaStream_t st, bool full = false, float gsca
     if (fused && nd == L.n_weights) {
         // only the biases are left beside the conv filters: extra blocks of the filter kernel take them (no decay on biases)
         const long long b4 = L.n_weights / 4, e4 = L.n_total / 4;
+        kn::ConvSplitSrc src;
+        memset(&src, 0, sizeof(src));
+        if (reduce_slot >= 0) {
+            src.on = 1;
+            for (int l = 0; l < 5; ++l) {
+                const tc::WgradParams& wp = R.conv_wg[l][reduce_slot].w;
+                src.splits[l] = wp.splits; src.cout[l] = L.conv[l].cout;
+                src.ws[l] = h->ws + h->ws_conv_off[l]; src.stride[l] = wp.split_stride;
+                src.bpart[l] = h->bias_partial + (size_t)l * kBiasPartial; src.b_off4[l] = L.conv[l].b_off / 4;
+            }
+        }
         launch_k(kn::sgd_update_conv_kernel, L.tjobs.tile0[5] + nblk(e4 - b4, 256), 256, 0, st, R.w, R.v, R.g, R.shadow, d,
-                 h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs, gscale, b4, e4, 0.f);
+                 h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs, gscale, b4, e4, 0.f, src);
         h->launches++;
         return;
     }
+    kn::ConvSplitSrc none;
+    memset(&none, 0, sizeof(none));
     launch_k(kn::sgd_update_conv_kernel, L.tjobs.tile0[5], 256, 0, st, R.w, R.v, R.g, R.shadow, d,
-             h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs, gscale, 0LL, 0LL, 0.f);
+             h->cfg.lr, h->cfg.momentum, R.wt, L.tjobs, gscale, 0LL, 0LL, 0.f, none);
     launch_k(kn::sgd_update_kernel, fused ? 148 : 1184, 256, 0, st, R.w, R.v, R.g, R.shadow, (fused ? L.n_weights : L.fc[0].w_off) / 4,
              L.n_total / 4, nd / 4, h->cfg.lr, h->cfg.momentum, h->cfg.weight_decay, gscale);
     h->launches += 2;
@@ -1044,7 +1064,7 @@ void forward(alexnet* h, int r, int slot, cudaStream_t st, bool eval) {
     }
     op_fc8_softmax(h, r, slot, st);
 }
-void forward_backward(alexnet* h, int r, int slot, cudaStream_t st, bool plain_fc = false) {
+void forward_backward(alexnet* h, int r, int slot, cudaStream_t st, bool plain_fc = false, bool defer_conv_reduce = false) {
     forward(h, r, slot, st, false);
     // the data gradient reads the layer's weights, so it comes first when the weight-gradient kernel updates them in place
     const bool fused = (h->cfg.flags & ALEXNET_FLAG_FUSED_FC_UPDATE) != 0 && !plain_fc;
@@ -1071,13 +1091,13 @@ void forward_backward(alexnet* h, int r, int slot, cudaStream_t st, bool plain_f
     }
     op_pool_bwd(h, r, 2, st);
     // (the transposed bf16 filters that the data gradients read are written between steps only: they may load early)
-    op_conv_wg(h, r, 4, slot, branch(3 + 4)); op_conv_bwd(h, r, 4, st, true);
-    op_conv_wg(h, r, 3, slot, branch(3 + 3)); op_conv_bwd(h, r, 3, st, true);
-    op_conv_wg(h, r, 2, slot, branch(3 + 2)); op_conv_bwd(h, r, 2, st, true);
+    op_conv_wg(h, r, 4, slot, branch(3 + 4), !defer_conv_reduce); op_conv_bwd(h, r, 4, st, true);
+    op_conv_wg(h, r, 3, slot, branch(3 + 3), !defer_conv_reduce); op_conv_bwd(h, r, 3, st, true);
+    op_conv_wg(h, r, 2, slot, branch(3 + 2), !defer_conv_reduce); op_conv_bwd(h, r, 2, st, true);
     op_pool_lrn_bwd(h, r, 1, st);
-    op_conv_wg(h, r, 1, slot, branch(3 + 1)); op_conv_bwd(h, r, 1, st, true);
+    op_conv_wg(h, r, 1, slot, branch(3 + 1), !defer_conv_reduce); op_conv_bwd(h, r, 1, st, true);
     op_pool_lrn_bwd(h, r, 0, st);
-    op_conv_wg(h, r, 0, slot, branch(3 + 0));
+    op_conv_wg(h, r, 0, slot, branch(3 + 0), !defer_conv_reduce);
     for (int b = 0; b < alexnet::kBranches; ++b)
         if (used[b]) {
             cudaEventRecord(h->ev_side_done[b], h->side[b]);
@@ -1342,10 +1362,12 @@ static int step_impl(alexnet_t* h, int replica, float* host_loss, bool with_upda
     if (R.loaded == 0) return fail(h, ALEXNET_ERR_STATE, "train_step: no loaded batch");
     const int s = R.next_train;
     CK(cudaStreamWaitEvent(h->cs, R.ready[s], 0));
-    forward_backward(h, replica, s, h->cs, !with_update);
+    // a step with its update: the conv split partials are added by the update launch (five reduction launches fewer)
+    const bool defer = with_update && update_can_reduce_conv(h);
+    forward_backward(h, replica, s, h->cs, !with_update, defer);
     CK(cudaEventRecord(R.consumed[s], h->cs));
     R.consumed_valid[s] = true;
-    if (with_update) op_update(h, replica, h->cs);
+    if (with_update) op_update(h, replica, h->cs, false, 1.f, defer ? s : -1);
     R.grad_pending = !with_update;
     R.last_slot = s; R.next_train ^= 1; R.loaded--;
     CK(cudaGetLastError());

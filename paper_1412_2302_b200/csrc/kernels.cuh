@@ -854,10 +854,20 @@ __global__ void sgd_update_kernel(float* __restrict__ w, float* __restrict__ v, 
 // 4*c4 .. 4*c4+3 of output channel r (the source order [tap][cout][cig]: 128-byte runs per row), the bf16 values cross a
 // shared-memory tile, and thread (ci, q) writes four consecutive output channels of input channel ci to the transposed copy
 // [tap][cin][cog] (64-byte runs; a thread that walked the source order would write single elements).  Same arithmetic as sgd_update_kernel.
-__global__ void __launch_bounds__(256) sgd_update_conv_kernel(float* __restrict__ w, float* __restrict__ v, const float* __restrict__ g,
+// With src.on the kernel also forms the conv gradients it consumes: the weight-gradient kernels leave fp32 partials per row
+// split (and bias-gradient partials), and instead of a reduction launch per layer the update adds them here, in split
+// order and with conv1's pad entries zeroed - wgrad_reduce_kernel's arithmetic - and stores the sums to g as that kernel does.
+struct ConvSplitSrc {
+    int on;
+    int splits[5], cout[5];
+    const float* ws[5]; long long stride[5];       // layer l: ws[l][z * stride[l] + index within the layer's filters]
+    const float* bpart[5]; long long b_off4[5];    // bias partials [z][cout]; first 16-byte vector of the layer's biases
+};
+__global__ void __launch_bounds__(256) sgd_update_conv_kernel(float* __restrict__ w, float* __restrict__ v, float* __restrict__ g,
                                                               __nv_bfloat16* __restrict__ shadow, float d, float lr, float mu,
                                                               __nv_bfloat16* __restrict__ wt, const TransposeJobs jobs, float gscale,
-                                                              long long tail_begin4, long long tail_end4, float tail_d) {
+                                                              long long tail_begin4, long long tail_end4, float tail_d,
+                                                              const ConvSplitSrc src) {
     pdl_sync();
     __shared__ __nv_bfloat16 tile[32][36];       // [input channel][output channel], padded
     if ((int)blockIdx.x >= jobs.tile0[jobs.n]) {
@@ -866,7 +876,24 @@ __global__ void __launch_bounds__(256) sgd_update_conv_kernel(float* __restrict_
         const long long i = tail_begin4 + (long long)((int)blockIdx.x - jobs.tile0[jobs.n]) * 256 + threadIdx.x;
         if (i < tail_end4) {
             float4 wv = ((float4*)w)[i], vv = ((float4*)v)[i];
-            const float4 gv = ((const float4*)g)[i];
+            float4 gv;
+            int lb = -1;
+            if (src.on) {
+                #pragma unroll
+                for (int l = 0; l < 5; ++l)
+                    if (i >= src.b_off4[l] && i < src.b_off4[l] + src.cout[l] / 4) lb = l;
+            }
+            if (lb >= 0) {                       // a conv layer's bias gradient from its partials
+                const float* bp = src.bpart[lb] + 4 * (i - src.b_off4[lb]);
+                gv = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int z = 0; z < src.splits[lb]; ++z) {
+                    const float4 t4 = __ldg((const float4*)(bp + (size_t)z * src.cout[lb]));
+                    gv.x += t4.x; gv.y += t4.y; gv.z += t4.z; gv.w += t4.w;
+                }
+                ((float4*)g)[i] = gv;
+            } else {
+                gv = ((const float4*)g)[i];
+            }
             sgd_step(wv.x, vv.x, gscale * gv.x, tail_d, lr, mu);
             sgd_step(wv.y, vv.y, gscale * gv.y, tail_d, lr, mu);
             sgd_step(wv.z, vv.z, gscale * gv.z, tail_d, lr, mu);
@@ -891,7 +918,28 @@ __global__ void __launch_bounds__(256) sgd_update_conv_kernel(float* __restrict_
     if (ci < J.cig) {                            // cig is a multiple of 4
         const long long e = J.src_off + ((long long)tap * J.cout + co) * J.cig + ci;
         float4 wv = *(float4*)(w + e), vv = *(float4*)(v + e);
-        const float4 gv = *(const float4*)(g + e);
+        float4 gv;
+        if (src.on) {
+            const long long t = e - J.src_off;
+            const float* sp = src.ws[q] + t;
+            gv = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int z = 0; z < src.splits[q]; ++z) {
+                const float4 t4 = __ldg((const float4*)(sp + z * src.stride[q]));
+                gv.x += t4.x; gv.y += t4.y; gv.z += t4.z; gv.w += t4.w;
+            }
+            if (q == 0) {                        // conv1: entries of the 12 x 12 zero-padded filter outside 11 x 11 stay zero
+                float* gp = &gv.x;
+                #pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int ch = (int)((t + k) % 48), tp = (int)((t + k) / (48 * 96));
+                    const int ky = (tp / 3) * 4 + (ch / 3) / 4, kx = (tp % 3) * 4 + (ch / 3) % 4;
+                    if (ky > 10 || kx > 10) gp[k] = 0.f;
+                }
+            }
+            *(float4*)(g + e) = gv;
+        } else {
+            gv = *(const float4*)(g + e);
+        }
         sgd_step(wv.x, vv.x, gscale * gv.x, d, lr, mu);
         sgd_step(wv.y, vv.y, gscale * gv.y, d, lr, mu);
         sgd_step(wv.z, vv.z, gscale * gv.z, d, lr, mu);
