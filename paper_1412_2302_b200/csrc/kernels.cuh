@@ -470,14 +470,23 @@ __global__ void __launch_bounds__(NT) pool_lrn_bwd_kernel(const __nv_bfloat16* _
                 #pragma unroll
                 for (int i = 0; i < 8; ++i) tt[i] = 0.f;
             }
-            float4* eb = edge[it & 1];
-            eb[threadIdx.x] = make_float4(tt[0], tt[1], tt[6], tt[7]);
-            __syncthreads();
+            // tt of channels c0-2, c0-1 (left neighbour's two highest) and c0+8, c0+9 (right neighbour's two lowest)
+            float4 l, r;
+            if (CPR == 32) {
+                // a pixel is exactly one warp: the neighbours are the adjacent lanes, no shared memory and no block barrier
+                l.z = __shfl_up_sync(0xffffffffu, tt[6], 1); l.w = __shfl_up_sync(0xffffffffu, tt[7], 1);
+                r.x = __shfl_down_sync(0xffffffffu, tt[0], 1); r.y = __shfl_down_sync(0xffffffffu, tt[1], 1);
+                if (ch == 0) { l.z = 0.f; l.w = 0.f; }
+                if (ch == CPR - 1) { r.x = 0.f; r.y = 0.f; }
+            } else {
+                float4* eb = edge[it & 1];
+                eb[threadIdx.x] = make_float4(tt[0], tt[1], tt[6], tt[7]);
+                __syncthreads();
+                l = ch > 0 ? eb[threadIdx.x - 1] : make_float4(0, 0, 0, 0);
+                r = ch < CPR - 1 ? eb[threadIdx.x + 1] : make_float4(0, 0, 0, 0);
+            }
             if (valid) {
-                // tt of channels c0-2, c0-1 (left neighbour's two highest) and c0+8, c0+9 (right neighbour's two lowest)
                 float te[12];
-                const float4 l = ch > 0 ? eb[threadIdx.x - 1] : make_float4(0, 0, 0, 0);
-                const float4 r = ch < CPR - 1 ? eb[threadIdx.x + 1] : make_float4(0, 0, 0, 0);
                 te[0] = l.z; te[1] = l.w; te[10] = r.x; te[11] = r.y;
                 #pragma unroll
                 for (int i = 0; i < 8; ++i) te[2 + i] = tt[i];
